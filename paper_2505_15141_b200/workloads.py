@@ -1,0 +1,256 @@
+"""Seeded synthetic inputs for the batched speculative-verification round.
+
+This module only *makes inputs*: logits, drafted tokens and the uniform random
+numbers a round consumes.  It contains none of the verification or bandit
+arithmetic and loads no native code, so the CUDA path and the CPU checker can
+both be fed from it without sharing anything else.
+
+The inputs stand in for LLM decoding traffic (real models and prompt sets are
+not available here): batch sizes 4..256, vocabularies 1024 / 32000 / 128256 /
+152064, speculation lengths up to 8, bf16 or fp32 logits.
+
+Random numbers
+--------------
+All uniforms come from Philox4x32-10 (Salmon et al., "Parallel random numbers:
+as easy as 1, 2, 3", SC'11), a counter-based generator:
+
+    key     = (seed & 0xffffffff, seed >> 32)
+    counter = (round, sequence b, block, stream tag)
+    u       = ((word >> 9) + 0.5) * 2**-23      in (0, 1), exact in fp32 (24 significant bits)
+
+Stream tags: 0 = accept uniforms (position j uses word j%4 of block j//4),
+1 = resample uniform (block 0, word 0), 2 = arm uniform (block 0, word 0),
+3 = drafting uniforms (same indexing as tag 0).
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import Optional, Sequence, Tuple
+
+import numpy as np
+import torch
+
+TAG_ACCEPT, TAG_RESAMPLE, TAG_ARM, TAG_DRAFT = 0, 1, 2, 3
+
+_M0 = np.uint64(0xD2511F53)
+_M1 = np.uint64(0xCD9E8D57)
+_W0 = 0x9E3779B9
+_W1 = 0xBB67AE85
+_LO = np.uint64(0xFFFFFFFF)
+_S32 = np.uint64(32)
+
+
+def philox4x32_10(counter: np.ndarray, key: Tuple[int, int]) -> np.ndarray:
+    """Philox4x32 with 10 rounds.
+
+    counter: integer array [..., 4] (each word < 2**32); key: two 32-bit words.
+    Returns uint32 array [..., 4].
+    """
+    c = np.asarray(counter).astype(np.uint64)
+    c0, c1, c2, c3 = c[..., 0], c[..., 1], c[..., 2], c[..., 3]
+    k0, k1 = int(key[0]) & 0xFFFFFFFF, int(key[1]) & 0xFFFFFFFF
+    for _ in range(10):
+        p0 = _M0 * c0
+        p1 = _M1 * c2
+        hi0, lo0 = p0 >> _S32, p0 & _LO
+        hi1, lo1 = p1 >> _S32, p1 & _LO
+        c0, c1, c2, c3 = hi1 ^ c1 ^ np.uint64(k0), lo1, hi0 ^ c3 ^ np.uint64(k1), lo0
+        k0 = (k0 + _W0) & 0xFFFFFFFF
+        k1 = (k1 + _W1) & 0xFFFFFFFF
+    return np.stack([c0, c1, c2, c3], axis=-1).astype(np.uint32)
+
+
+def words_to_uniform(words: np.ndarray) -> np.ndarray:
+    """Map 32-bit words to fp32 uniforms strictly inside (0, 1)."""
+    return ((words >> np.uint32(9)).astype(np.float64) + 0.5).astype(np.float32) * np.float32(2.0 ** -23)
+
+
+def _stream(seed: int, rnd: int, B: int, n: int, tag: int) -> np.ndarray:
+    """n uniforms per sequence from the stream `tag`: array [B, n] fp32."""
+    nblk = max(1, (n + 3) // 4)
+    ctr = np.zeros((B, nblk, 4), dtype=np.uint64)
+    ctr[..., 0] = rnd & 0xFFFFFFFF
+    ctr[..., 1] = np.arange(B, dtype=np.uint64)[:, None]
+    ctr[..., 2] = np.arange(nblk, dtype=np.uint64)[None, :]
+    ctr[..., 3] = tag
+    w = philox4x32_10(ctr, (seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF))
+    return words_to_uniform(w.reshape(B, nblk * 4)[:, :n])
+
+
+@dataclass
+class RoundUniforms:
+    u_accept: np.ndarray    # [B, Gmax] fp32
+    u_resample: np.ndarray  # [B] fp32
+    u_arm: np.ndarray       # [B] fp32
+    u_draft: np.ndarray     # [B, Gmax] fp32
+
+
+def round_uniforms(seed: int, rnd: int, B: int, Gmax: int) -> RoundUniforms:
+    """All uniforms round `rnd` consumes, for every sequence."""
+    g = max(Gmax, 1)
+    return RoundUniforms(
+        u_accept=_stream(seed, rnd, B, g, TAG_ACCEPT)[:, :Gmax].copy(),
+        u_resample=_stream(seed, rnd, B, 1, TAG_RESAMPLE)[:, 0].copy(),
+        u_arm=_stream(seed, rnd, B, 1, TAG_ARM)[:, 0].copy(),
+        u_draft=_stream(seed, rnd, B, g, TAG_DRAFT)[:, :Gmax].copy(),
+    )
+
+
+# --------------------------------------------------------------------------
+# Workload presets
+# --------------------------------------------------------------------------
+
+@dataclass(frozen=True)
+class Workload:
+    name: str
+    B: int
+    V: int
+    arm_gamma: Tuple[int, ...]      # speculation length of each arm
+    dtype: str                      # "f32" | "bf16"
+    temperature: float              # 0.0 = greedy
+    rounds: int
+    seed: int
+    alg: Optional[str]              # "ucb" | "exp3" | None (fixed arm 0)
+    target_std: float = 3.0
+    boost_prob: float = 0.05        # Bernoulli probability of a +boost entry
+    boost: float = 8.0
+    sigma: str = "fixed"            # "fixed" | "per_seq" | "per_arm_phase"
+    sigma_fixed: float = 1.0
+    sigma_range: Tuple[float, float] = (0.3, 2.0)
+    sigma_arms: Tuple[float, ...] = (0.3, 0.8, 1.5, 3.0)
+    phase_len: int = 200
+    delta: float = 0.5
+
+    @property
+    def K(self) -> int:
+        return len(self.arm_gamma)
+
+    @property
+    def Gmax(self) -> int:
+        return max(self.arm_gamma)
+
+    @property
+    def torch_dtype(self) -> torch.dtype:
+        return torch.float32 if self.dtype == "f32" else torch.bfloat16
+
+    @property
+    def elem_size(self) -> int:
+        return 4 if self.dtype == "f32" else 2
+
+
+WORKLOADS = {
+    # tiny: iid N(0, 2^2) target, no boosted entries, draft = target + N(0, 0.5^2)
+    "tiny_ucb": Workload("tiny_ucb", B=4, V=1024, arm_gamma=(2, 4, 6), dtype="f32",
+                         temperature=1.0, rounds=64, seed=0, alg="ucb",
+                         target_std=2.0, boost_prob=0.0, sigma_fixed=0.5),
+    "tiny_ucb_greedy": Workload("tiny_ucb_greedy", B=4, V=1024, arm_gamma=(2, 4, 6), dtype="f32",
+                                temperature=0.0, rounds=64, seed=0, alg="ucb",
+                                target_std=2.0, boost_prob=0.0, sigma_fixed=0.5),
+    # 32000-entry vocabulary, fixed speculation length 5
+    "llama2_fixed": Workload("llama2_fixed", B=32, V=32000, arm_gamma=(5,), dtype="bf16",
+                             temperature=0.7, rounds=200, seed=1, alg=None),
+    # 128256-entry vocabulary, UCBSpec over four speculation lengths, ragged per sequence
+    "llama3_ucb": Workload("llama3_ucb", B=64, V=128256, arm_gamma=(2, 4, 6, 8), dtype="bf16",
+                           temperature=1.0, rounds=500, seed=2, alg="ucb", sigma="per_seq"),
+    # 152064-entry vocabulary, EXP3Spec, draft quality per arm rotates every 200 rounds
+    "qwen_exp3": Workload("qwen_exp3", B=256, V=152064, arm_gamma=(1, 3, 5, 8), dtype="f32",
+                          temperature=1.0, rounds=1000, seed=4, alg="exp3", sigma="per_arm_phase"),
+}
+
+
+def torch_generator(seed: int, rnd: int, device) -> torch.Generator:
+    g = torch.Generator(device=device)
+    g.manual_seed((seed * 1_000_003 + rnd * 7919 + 12345) & 0x7FFFFFFFFFFFFFFF)
+    return g
+
+
+def per_sequence_sigma(w: Workload) -> np.ndarray:
+    """Draft-noise scale per sequence for sigma == "per_seq" (fixed for the run)."""
+    rs = np.random.RandomState(w.seed + 977)
+    lo, hi = w.sigma_range
+    return rs.uniform(lo, hi, size=w.B).astype(np.float32)
+
+
+def round_sigma(w: Workload, rnd: int, arm: Optional[np.ndarray]) -> np.ndarray:
+    """Draft-noise scale of every sequence in round `rnd` (1-based) given its arm."""
+    if w.sigma == "fixed":
+        return np.full(w.B, w.sigma_fixed, dtype=np.float32)
+    if w.sigma == "per_seq":
+        return per_sequence_sigma(w)
+    if w.sigma == "per_arm_phase":
+        assert arm is not None
+        phase = (rnd - 1) // w.phase_len
+        tab = np.asarray(w.sigma_arms, dtype=np.float32)
+        return tab[(np.asarray(arm) + phase) % len(tab)]
+    raise ValueError(w.sigma)
+
+
+def make_logits(w: Workload, rnd: int, sigma: np.ndarray, device="cpu",
+                B: Optional[int] = None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Target logits [B, Gmax+1, V] and draft logits [B, Gmax, V] in w's dtype.
+
+    target = N(0, std^2) + boost * Bernoulli(boost_prob)   (fp32, then rounded)
+    draft  = (fp32 target before rounding) + sigma_b * N(0, 1), then rounded
+    """
+    B = w.B if B is None else B
+    G, V = w.Gmax, w.V
+    g = torch_generator(w.seed, rnd, device)
+    t = torch.empty(B, G + 1, V, dtype=torch.float32, device=device)
+    t.normal_(0.0, w.target_std, generator=g)
+    if w.boost_prob > 0.0:
+        mask = torch.empty(B, G + 1, V, dtype=torch.float32, device=device).uniform_(generator=g)
+        t += w.boost * (mask < w.boost_prob).to(torch.float32)
+        del mask
+    d = torch.empty(B, G, V, dtype=torch.float32, device=device)
+    d.normal_(0.0, 1.0, generator=g)
+    s = torch.as_tensor(np.asarray(sigma, dtype=np.float32)[:B], device=device).view(B, 1, 1)
+    d.mul_(s).add_(t[:, :G, :])
+    return t.to(w.torch_dtype), d.to(w.torch_dtype)
+
+
+def draw_draft_tokens(draft_logits: torch.Tensor, temperature: float,
+                      u_draft: np.ndarray) -> torch.Tensor:
+    """Drafted tokens [B, Gmax] int32: position j is drawn from softmax(draft row j / T)
+    by inverse CDF with the uniform u_draft[b, j]; at temperature 0 it is the row argmax.
+    (Input generation only: rows are independent "contexts", see make_logits.)"""
+    B, G, V = draft_logits.shape
+    if G == 0:
+        return torch.zeros(B, 0, dtype=torch.int32, device=draft_logits.device)
+    if temperature == 0.0:
+        return draft_logits.float().argmax(dim=-1).to(torch.int32)
+    dev = draft_logits.device
+    acc = torch.float64 if dev.type == "cpu" else torch.float32
+    out = torch.empty(B, G, dtype=torch.int32, device=dev)
+    u = torch.as_tensor(np.asarray(u_draft, dtype=np.float32), device=dev).to(acc)
+    for j in range(G):  # one position at a time bounds the temporary to [B, V]
+        pr = torch.softmax(draft_logits[:, j, :].to(acc) / temperature, dim=-1)
+        cdf = torch.cumsum(pr, dim=-1)
+        tgt = (u[:, j] * cdf[:, -1]).unsqueeze(-1)
+        idx = torch.searchsorted(cdf, tgt, right=True).squeeze(-1).clamp_(max=V - 1)
+        out[:, j] = idx.to(torch.int32)
+    return out
+
+
+@dataclass
+class RoundInputs:
+    target: torch.Tensor        # [B, Gmax+1, V]
+    draft: torch.Tensor         # [B, Gmax, V]
+    tokens: torch.Tensor        # [B, Gmax] int32
+    gamma: np.ndarray           # [B] int32
+    uniforms: RoundUniforms
+    sigma: np.ndarray = field(default_factory=lambda: np.zeros(0, np.float32))
+
+
+def make_round(w: Workload, rnd: int, arm: Optional[np.ndarray] = None,
+               device="cpu") -> RoundInputs:
+    """Everything one verification round reads, for round `rnd` (1-based).
+    `arm` [B] is the arm each sequence plays (None = arm 0 for all)."""
+    if arm is None:
+        arm = np.zeros(w.B, dtype=np.int32)
+    arm = np.asarray(arm, dtype=np.int32)
+    gamma = np.asarray(w.arm_gamma, dtype=np.int32)[arm]
+    sig = round_sigma(w, rnd, arm)
+    t, d = make_logits(w, rnd, sig, device=device)
+    un = round_uniforms(w.seed, rnd, w.B, w.Gmax)
+    tok = draw_draft_tokens(d, w.temperature, un.u_draft)
+    return RoundInputs(target=t, draft=d, tokens=tok, gamma=gamma, uniforms=un, sigma=sig)
