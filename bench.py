@@ -1,0 +1,424 @@
+#!/usr/bin/env python
+"""Benchmark of the batched speculative-verification round (one JSON line on stdout).
+
+A step is one pass of the whole hot path over one batch of synthetic input:
+  bs_bandit_select -> bs_softmax_verify -> bs_residual_sample -> bs_bandit_update
+captured as one CUDA graph per input set.  Inputs rotate through a ring of distinct sets
+whose total size exceeds twice the L2, so every step reads its logits from HBM.
+
+  value      rounds/s with the inputs resident in HBM (whole job, all ranks)
+  e2e        the same round driven from pinned HOST buffers: the step's logits, tokens and
+             uniforms are copied to the device and the emitted tokens read back inside the
+             timed region
+  roofline   bs_softmax_verify's kernel: algorithmic bytes (every valid logit once) divided by
+             its mean duration between CUDA events on the launching stream
+  cpu_baseline  the CPU oracle, as it stands, on a bounded sample of the same workload
+
+`--impl reference` times the CPU oracle instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "batched spec-verify rounds/sec"
+UNIT = "rounds/s"
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_HBM_GBS = 6650.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one verify launch from the ncu captures
+# summarised under profiles/ (bytes per launch; None = not captured for that workload)
+NCU_TRAFFIC = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--workload", default="qwen_exp3",
+                    choices=["tiny_ucb", "llama2_fixed", "llama3_ucb", "qwen_exp3"])
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=4)
+    ap.add_argument("--cpu-seconds", type=float, default=12.0, help="budget of the CPU-oracle sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch the four calls directly each step")
+    return ap.parse_args()
+
+
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+# ---------------------------------------------------------------------------------------------
+# CPU oracle timing (cpu_baseline leg and --impl reference)
+# ---------------------------------------------------------------------------------------------
+
+def oracle_sample(w, rnd_inputs, seconds: float, max_seqs=None):
+    """Runs the oracle's verification on sequences of one round until `seconds` are used.
+    Returns (sequences done, elapsed seconds)."""
+    from oracle import verify as ov
+    toks = rnd_inputs.tokens.cpu().numpy()
+    done, t0 = 0, time.perf_counter()
+    B = rnd_inputs.target.shape[0]
+    limit = B if max_seqs is None else min(B, max_seqs)
+    while done < limit:
+        b = done
+        g = int(rnd_inputs.gamma[b])
+        t_rows = rnd_inputs.target[b, :g + 1].float().cpu().numpy()
+        d_rows = rnd_inputs.draft[b, :g].float().cpu().numpy()
+        ov.verify_sequence(t_rows, d_rows, toks[b], g, rnd_inputs.uniforms.u_accept[b],
+                           float(rnd_inputs.uniforms.u_resample[b]), w.temperature)
+        done += 1
+        if time.perf_counter() - t0 > seconds:
+            break
+    return done, time.perf_counter() - t0
+
+
+def default_arms(w, step: int) -> np.ndarray:
+    """Arms used to shape the pre-generated inputs (the device bandit picks its own gamma)."""
+    return ((np.arange(w.B) + step) % w.K).astype(np.int32)
+
+
+def run_reference(args, w):
+    """The oracle, as it stands, on the host cores: each step is a bounded sample of one round."""
+    from paper_2505_15141_b200 import workloads as wl
+    import torch
+    torch.set_num_threads(1)
+    per_step = max(0.5, min(10.0, 90.0 / max(1, args.steps + args.warmup)))
+    nb = min(w.B, 16)                                   # sequences generated for the sample
+    rnd = wl.make_round(w, 1, default_arms(w, 0), device="cpu", B=nb)
+    times, seqs = [], []
+    for i in range(args.warmup + args.steps):
+        n, dt = oracle_sample(w, rnd, per_step)
+        if i >= args.warmup:
+            times.append(dt); seqs.append(n)
+    rounds = sum(seqs) / w.B
+    total = sum(times)
+    val = rounds / total
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / max(1, args.steps),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "V": w.V, "arm_gamma": list(w.arm_gamma),
+                   "logits_dtype": w.dtype, "temperature": w.temperature},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle",
+                         "sample": f"{sum(seqs)} sequences of {w.B}-sequence rounds in {total:.1f} s, "
+                                   f"verification only (numpy fp64, one thread)"},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks
+# ---------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for ln in self.proc.stdout:
+            self.lines.append(ln.strip())
+
+    def stop(self) -> dict:
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()                    # the exact child started above
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------------------------------------
+# CUDA arm
+# ---------------------------------------------------------------------------------------------
+
+def run_cuda(args, w):
+    import torch
+    import torch.distributed as dist
+    import __graft_entry__ as entry
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        dist.init_process_group(backend="nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if rank == 0:
+        entry.build()
+    if world > 1:
+        dist.barrier()
+    from paper_2505_15141_b200 import binding as bs, workloads as wl
+
+    B, K, G, V = w.B, w.K, w.Gmax, w.V
+    alg = bs.BS_EXP3 if w.alg == "exp3" else bs.BS_UCB        # a fixed arm is a 1-armed UCBSpec
+    es = w.elem_size
+    arm_gamma = np.asarray(w.arm_gamma)
+
+    # ---- ring of input sets, > 2 x L2 in total ----
+    set_bytes = es * V * B * (2 * G + 1)
+    ring = max(2, -(-2 * L2_BYTES // set_bytes) + 1)
+    seed_shift = 1000 * rank                                   # every rank verifies its own batch
+    sets = []
+    for i in range(ring):
+        rnd = wl.make_round(w, 1 + i + seed_shift, default_arms(w, i), device=dev)
+        sets.append(dict(
+            target=rnd.target, draft=rnd.draft, tokens=rnd.tokens.contiguous(),
+            u_accept=torch.as_tensor(rnd.uniforms.u_accept, device=dev),
+            u_resample=torch.as_tensor(rnd.uniforms.u_resample, device=dev),
+            u_arm=torch.as_tensor(rnd.uniforms.u_arm, device=dev), rnd=rnd))
+    state = bs.new_bandit(alg, B, w.arm_gamma, w.delta, dev)
+    ws = bs.new_workspace(B, G, V, dev)
+    arm_d = torch.zeros(B, dtype=torch.int32, device=dev)
+    gamma_d = torch.zeros(B, dtype=torch.int32, device=dev)
+    accept_len = torch.zeros(B, dtype=torch.int32, device=dev)
+    p_tok = torch.zeros(B, G, dtype=torch.float32, device=dev)
+    q_tok = torch.zeros(B, G, dtype=torch.float32, device=dev)
+    out_tokens = torch.zeros(B, G + 1, dtype=torch.int32, device=dev)
+    out_len = torch.zeros(B, dtype=torch.int32, device=dev)
+
+    def step_calls(s):
+        bs.bs_bandit_select(state, alg, B, K, s["u_arm"], None, arm_d, gamma_d)
+        bs.bs_softmax_verify(s["target"], s["draft"], s["tokens"], gamma_d, s["u_accept"], w.temperature,
+                             accept_len, p_tok, q_tok, ws)
+        bs.bs_residual_sample(s["target"], s["draft"], s["tokens"], gamma_d, accept_len, s["u_resample"],
+                              w.temperature, out_tokens, out_len, ws)
+        bs.bs_bandit_update(state, alg, B, K, arm_d, out_len)
+
+    side = torch.cuda.Stream(device=dev)
+    graphs = []
+    if not args.no_graph:
+        with torch.cuda.stream(side):
+            step_calls(sets[0])                                # first launch outside capture
+            side.synchronize()
+            for s in sets:
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    step_calls(s)
+                graphs.append(g)
+        torch.cuda.synchronize()
+        # start from a clean bandit: the capture warm-up above played one round
+        bs.bs_bandit_init(state, alg, B, K, w.arm_gamma, w.delta)
+
+    def run_step(i):
+        if graphs:
+            graphs[i % ring].replay()
+        else:
+            step_calls(sets[i % ring])
+
+    def pulls():
+        return bs.bs_bandit_read(state, alg, B, K)["n"].copy()
+
+    def sync_all():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- warm-up, then the timed region ----
+    for i in range(args.warmup):
+        run_step(i)
+    sync_all()
+    n0 = pulls()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    sync_all()
+    stream = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    y_sum = torch.zeros((), dtype=torch.int64, device=dev)
+    e0.record(stream)
+    for i in range(args.steps):
+        run_step(args.warmup + i)
+    e1.record(stream)
+    sync_all()
+    ms = e0.elapsed_time(e1)
+    if rank == 0:
+        time.sleep(0.15)
+        clocks = sampler.stop()
+    n1 = pulls()
+    dn = (n1 - n0)                                             # [B, K] pulls inside the timed region
+    assert dn.sum() == B * args.steps, "every sequence must have played every timed round"
+    rows_timed = int((dn * (2 * arm_gamma + 1)[None, :]).sum())
+    bytes_timed = rows_timed * V * es
+    if world > 1:
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+        bt = torch.tensor([bytes_timed], dtype=torch.float64, device=dev)
+        dist.all_reduce(bt, op=dist.ReduceOp.SUM)
+        bytes_all = float(bt.item())
+    else:
+        bytes_all = float(bytes_timed)
+    value = world * args.steps / (ms * 1e-3)
+
+    # ---- kernel pass: CUDA events around bs_softmax_verify on its launching stream ----
+    ksteps = min(args.steps, 50)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(ksteps)]
+    rsd = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(ksteps)]
+    nk0 = pulls()
+    y_total = 0
+    for i in range(ksteps):
+        s = sets[(args.warmup + args.steps + i) % ring]
+        bs.bs_bandit_select(state, alg, B, K, s["u_arm"], None, arm_d, gamma_d)
+        evs[i][0].record(stream)
+        bs.bs_softmax_verify(s["target"], s["draft"], s["tokens"], gamma_d, s["u_accept"], w.temperature,
+                             accept_len, p_tok, q_tok, ws)
+        evs[i][1].record(stream)
+        rsd[i][0].record(stream)
+        bs.bs_residual_sample(s["target"], s["draft"], s["tokens"], gamma_d, accept_len, s["u_resample"],
+                              w.temperature, out_tokens, out_len, ws)
+        rsd[i][1].record(stream)
+        bs.bs_bandit_update(state, alg, B, K, arm_d, out_len)
+        y_sum += out_len.sum()
+    torch.cuda.synchronize()
+    verify_ms = sum(a.elapsed_time(b) for a, b in evs) / ksteps
+    resid_ms = sum(a.elapsed_time(b) for a, b in rsd) / ksteps
+    dk = pulls() - nk0
+    verify_bytes = float((dk * (2 * arm_gamma + 1)[None, :]).sum()) * V * es / ksteps   # per launch
+    mean_y = float(y_sum.item()) / (B * ksteps)
+    status = bs.bs_get_device_status(ws, B, G, V)
+    assert (status & ~bs.BS_DEV_RESIDUAL_FALLBACK == 0).all(), f"device status {status}"
+
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
+    else:
+        peak, peak_src = FALLBACK_HBM_GBS, "fallback"
+    achieved = verify_bytes / (verify_ms * 1e-3) / 1e9
+
+    # ---- end to end from pinned host buffers ----
+    e2e = None
+    if args.e2e_steps > 0:
+        s0 = sets[0]
+        host = {k: torch.empty(s0[k].shape, dtype=s0[k].dtype, pin_memory=True).copy_(s0[k])
+                for k in ("target", "draft", "tokens", "u_accept", "u_resample", "u_arm")}
+        devb = {k: torch.empty_like(s0[k]) for k in host}
+        h_tokens = torch.empty(out_tokens.shape, dtype=out_tokens.dtype, pin_memory=True)
+        h_len = torch.empty(out_len.shape, dtype=out_len.dtype, pin_memory=True)
+        h2d = sum(t.numel() * t.element_size() for t in host.values())
+        d2h = h_tokens.numel() * 4 + h_len.numel() * 4
+
+        def e2e_step():
+            for k in host:
+                devb[k].copy_(host[k], non_blocking=True)
+            step_calls(devb)
+            h_tokens.copy_(out_tokens, non_blocking=True)
+            h_len.copy_(out_len, non_blocking=True)
+            torch.cuda.current_stream().synchronize()          # the caller reads the tokens every round
+
+        for _ in range(2):
+            e2e_step()
+        sync_all()
+        a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        b_.record(stream)
+        sync_all()
+        e2e_ms = a.elapsed_time(b_)
+        if world > 1:
+            t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        e2e = {"value": world * args.e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": args.e2e_steps}
+        del host, devb
+
+    # ---- CPU oracle on a bounded sample (rank 0, N = 1 only) ----
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        torch.set_num_threads(1)
+        rnd = sets[0]["rnd"]
+        rnd.gamma = np.asarray(w.arm_gamma, dtype=np.int32)[default_arms(w, 0)]
+        n, dt = oracle_sample(w, rnd, args.cpu_seconds)
+        cpu = {"value": (n / B) / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": f"{n} of the {B} sequences of one round in {dt:.1f} s, verification only "
+                         f"(numpy fp64, one thread; host has {host_cores()} cores)"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "B": B, "V": V, "arm_gamma": list(w.arm_gamma), "bandit": w.alg or "fixed",
+                       "logits_dtype": w.dtype, "temperature": w.temperature,
+                       "l2": f"ring of {ring} input sets, {ring * set_bytes / 1e6:.0f} MB > 2 x L2",
+                       "launch": "one CUDA graph per step" if graphs else "direct launches",
+                       "multi_gpu": "one independent batch per rank, no collective on the data path"},
+            "tokens_per_s": mean_y * B * value,
+            "mean_accepted_len": mean_y,
+            "algorithmic_gbs": bytes_all / (ms * 1e-3) / 1e9,
+            "roofline": {"bound": "hbm", "kernel": "verify_kernel (bs_softmax_verify)", "achieved": achieved,
+                         "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": NCU_TRAFFIC.get(w.name), "bytes_per_launch": verify_bytes,
+                         "ms_per_launch": verify_ms, "residual_ms_per_launch": resid_ms},
+            "e2e": e2e, "cpu_baseline": cpu, "clocks": clocks,
+            "gpu_launches": 4 * args.steps,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    from paper_2505_15141_b200 import workloads as wl
+    w = wl.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        if int(os.environ.get("RANK", "0")) == 0:
+            run_reference(args, w)
+        return
+    run_cuda(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,177 @@
+/*
+ * banditspec.h -- C ABI of the B200 (sm_100a) library for one batched round of
+ * speculative decoding with a bandit-chosen speculation length.
+ *
+ * One round, per sequence b of a batch of B independent sequences:
+ *
+ *   bs_bandit_select    choose the arm (speculation length gamma_b) for this round
+ *   bs_softmax_verify   softmax statistics of every target / draft row, accept test,
+ *                       first-rejection scan  -> accept_len[b] = tau_b
+ *   bs_residual_sample  resample one token from Norm([P - Q]_+) at the rejected position,
+ *                       or the bonus token from P when all drafts passed -> out_tokens, out_len
+ *   bs_bandit_update    feed the accepted length y_b = tau_b + 1 back to the arm statistics
+ *
+ * plus bs_lmhead_verify, which computes the logits themselves (bf16 hidden states times
+ * the bf16 output embedding on the tensor cores) fused with the softmax statistics.
+ *
+ * Conventions that hold for every entry point
+ *  - Every array pointer is a DEVICE pointer owned by the caller unless the comment says
+ *    "host".  The library allocates no device memory and keeps no global state.
+ *  - `stream` is a cudaStream_t passed as void*.  Calls are asynchronous on that stream,
+ *    never synchronise, and may be captured in a CUDA graph.
+ *  - The return value covers host-side argument checks and launch errors only.  Problems
+ *    found in device DATA (token id outside [0,V), gamma outside [0,Gmax], non-finite
+ *    normaliser) are recorded per sequence in the workspace and read back with
+ *    bs_get_device_status; the kernels never trap.
+ *  - Row-major layouts with the vocabulary contiguous.  Row j (0-based) of either model is
+ *    the distribution of drafted token j+1, i.e. conditioned on the prompt and the first j
+ *    drafted tokens; target row gamma_b is the bonus position.  Padded entries (j >= gamma_b
+ *    for tokens / uniforms / draft rows, j > gamma_b for target rows) are never read.
+ *  - temperature > 0: sampling mode, probabilities are softmax(logits / temperature).
+ *    temperature == 0: greedy mode (the limit of Section 2): a drafted token passes iff it
+ *    equals the arg-max of its target row (lowest index among equal maxima); draft logits
+ *    are not read and may be NULL.
+ */
+#ifndef BANDITSPEC_H_
+#define BANDITSPEC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    BS_OK = 0,
+    BS_ERR_INVALID_ARG = 1,   /* NULL pointer, negative or unsupported size, bad enum */
+    BS_ERR_CUDA = 2,          /* a CUDA runtime call or launch failed */
+    BS_ERR_UNSUPPORTED = 3,   /* valid request outside the implemented limits */
+    BS_ERR_WORKSPACE = 4,     /* workspace too small or misaligned */
+    BS_ERR_TIMEOUT = 5,       /* a bounded device-side wait gave up (LM-head pipeline) */
+    BS_ERR_DEVICE_DATA = 6    /* bs_get_device_status: some sequence carries a data error */
+} bs_status;
+
+typedef enum { BS_F32 = 0, BS_BF16 = 1 } bs_dtype;
+typedef enum { BS_UCB = 0, BS_EXP3 = 1 } bs_alg;
+
+/* Per-sequence device status bits (bs_get_device_status). */
+#define BS_DEV_BAD_GAMMA   1   /* gamma[b] outside [0, Gmax]; the sequence was processed as gamma = 0 */
+#define BS_DEV_BAD_TOKEN   2   /* a drafted token outside [0, V); that position counts as rejected */
+#define BS_DEV_NONFINITE   4   /* a softmax normaliser or residual mass was NaN / Inf / 0 */
+#define BS_DEV_RESIDUAL_FALLBACK 8 /* [P-Q]_+ had zero mass at the rejected position; sampled from P instead */
+
+/* Limits of this implementation. */
+#define BS_MAX_GAMMA   31      /* Gmax <= 31 (one warp scans the accept flags) */
+#define BS_MAX_ARMS    32      /* K <= 32 (one lane per arm) */
+#define BS_MAX_BATCH   4096    /* B <= 4096 */
+
+const char* bs_status_string(bs_status s);
+
+/* ---- workspace ------------------------------------------------------------------ */
+
+/* Bytes of device scratch bs_softmax_verify / bs_residual_sample / bs_lmhead_verify need for
+ * a batch of B sequences, speculation lengths up to Gmax and vocabulary V (any dtype).
+ * Returns 0 for arguments outside the limits. */
+size_t bs_workspace_bytes(int B, int Gmax, int V);
+
+/* Clears the workspace (arrival counters must start at zero; the kernels leave them at zero
+ * again after every call).  Call once after allocating, 256-byte aligned. */
+bs_status bs_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+
+/* Copies the per-sequence status words of the LAST verify/residual call to host memory.
+ * Synchronises the stream.  host_status: host array [B].  Returns BS_ERR_DEVICE_DATA if any
+ * word is non-zero, BS_OK otherwise. */
+bs_status bs_get_device_status(const void* workspace, size_t workspace_bytes, int B, int Gmax, int V,
+                               int32_t* host_status, void* stream);
+
+/* ---- verification (Algorithm 6 of the paper, from its second line on) ---------------- */
+
+/* Softmax statistics (Section 2: softmax of logits / temperature), accept test
+ * r <= min{1, P(x)/Q(x)} and first-rejection scan (Algorithm 6, for-loop).
+ *
+ *  target_logits  [B, Gmax+1, V]  dtype
+ *  draft_logits   [B, Gmax,   V]  dtype; may be NULL iff temperature == 0
+ *  draft_tokens   [B, Gmax] int32, the drafted tokens x~_1..x~_gamma
+ *  gamma          [B] int32, speculation length of each sequence this round, 0 <= gamma <= Gmax
+ *  u_accept       [B, Gmax] fp32 uniforms in (0,1); may be NULL iff temperature == 0
+ *  accept_len     [B] int32 out: tau_b = number of leading accepted drafts
+ *  p_tok, q_tok   [B, Gmax] fp32 out or NULL: P_j(x~_{j+1}), Q_j(x~_{j+1}) for j < gamma_b
+ *                 (entries j >= gamma_b are set to 0; both zero-filled in greedy mode)
+ *  workspace      from bs_workspace_bytes / bs_workspace_init; keeps the row statistics that
+ *                 bs_residual_sample reads, so the two calls share it and run on one stream.
+ * Reads every valid logit exactly once.  Two calls that share a workspace must not overlap. */
+bs_status bs_softmax_verify(const void* target_logits, const void* draft_logits, bs_dtype dtype,
+                            const int32_t* draft_tokens, const int32_t* gamma, const float* u_accept,
+                            float temperature, int B, int Gmax, int V,
+                            int32_t* accept_len, float* p_tok, float* q_tok,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
+/* Resampling step (Algorithm 6, else-branch and the line after the loop): for each sequence,
+ * with tau = accept_len[b]: if tau < gamma_b sample from Norm([P_tau - Q_tau]_+), otherwise
+ * sample the bonus token from P_gamma.  One uniform per sequence, inverse CDF in vocabulary
+ * order: the smallest v whose cumulative mass strictly exceeds u * total.  Greedy mode emits
+ * the arg-max of target row tau.
+ *
+ *  same logits / dtype / tokens / gamma / temperature / sizes / workspace as the preceding
+ *  bs_softmax_verify call on this stream (its row statistics are read from the workspace)
+ *  accept_len   [B] int32 in
+ *  u_resample   [B] fp32 uniforms in (0,1); may be NULL iff temperature == 0
+ *  out_tokens   [B, Gmax+1] int32 out: the tau accepted drafts, then the sampled token, then -1
+ *  out_len      [B] int32 out: y_b = tau_b + 1, the accepted length that is the bandit reward
+ *               (Section 3: the bonus token counts, 1 <= y <= L+1) */
+bs_status bs_residual_sample(const void* target_logits, const void* draft_logits, bs_dtype dtype,
+                             const int32_t* draft_tokens, const int32_t* gamma, const int32_t* accept_len,
+                             const float* u_resample, float temperature, int B, int Gmax, int V,
+                             int32_t* out_tokens, int32_t* out_len,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---- arm selection (Algorithm 3, select and history lines) ---------------------------- */
+
+/* Bytes of the opaque device state of B independent bandits with K arms. 0 if out of limits. */
+size_t bs_bandit_state_bytes(bs_alg alg, int B, int K);
+
+/* Resets the state: no pulls, no rounds.  arm_gamma: HOST array [K], speculation length of
+ * each arm; L = max_i arm_gamma[i] is the maximum speculation length of the configuration.
+ * delta: confidence parameter of UCBSpec (Algorithm 4 input; the regret proof uses 1/2);
+ * ignored by EXP3Spec.  The state is plain device memory: copying its bytes checkpoints it. */
+bs_status bs_bandit_init(void* state, size_t state_bytes, bs_alg alg, int B, int K,
+                         const int32_t* arm_gamma_host, double delta, void* stream);
+
+/* Chooses this round's arm for every active sequence.
+ *  UCBSpec (Algorithm 4 / Algorithm 8): arm t in the first K rounds (t = completed rounds),
+ *    then argmax_i  sumY_i/n_i + (L/2) sqrt((1+n_i)/n_i^2 (1 + 2 ln(K t^2 sqrt(1+n_i)/delta))),
+ *    lowest index on ties.  u_arm is not read and may be NULL.
+ *  EXP3Spec (Algorithm 5 / Algorithm 9): p_i proportional to exp(-eta_t S_i),
+ *    eta_t = sqrt(ln K / (t K)) with t = completed rounds + 1; the arm is the smallest i whose
+ *    cumulative probability strictly exceeds u_arm[b]; p of the chosen arm is kept for the update.
+ *  u_arm   [B] fp32 uniforms in (0,1) (EXP3Spec)
+ *  active  [B] uint8 or NULL (= all active); inactive sequences get arm = -1, gamma = 0
+ *  arm     [B] int32 out;  gamma [B] int32 out = arm_gamma[arm]
+ *  index_out [B, K] fp64 out or NULL: the UCB index values / EXP3 probabilities used (NaN
+ *            during UCBSpec's round-robin prefix) -- for tests and logging. */
+bs_status bs_bandit_select(void* state, size_t state_bytes, bs_alg alg, int B, int K,
+                           const float* u_arm, const uint8_t* active,
+                           int32_t* arm, int32_t* gamma, double* index_out, void* stream);
+
+/* Records the outcome of the round for every active sequence.
+ *  UCBSpec: n[arm] += 1, sumY[arm] += y, t += 1.
+ *  EXP3Spec: S[arm] += (L + 1 - y) / (L * p_arm), t += 1  (loss estimate of Algorithm 9).
+ *  arm [B] int32 in (as returned by select); reward_y [B] int32 in, 1 <= y <= L+1
+ *  (out_len of bs_residual_sample); values outside that range are clamped. */
+bs_status bs_bandit_update(void* state, size_t state_bytes, bs_alg alg, int B, int K,
+                           const int32_t* arm, const int32_t* reward_y, const uint8_t* active,
+                           void* stream);
+
+/* Reads the sufficient statistics back to host arrays (any may be NULL).  Synchronises.
+ *  UCBSpec: n_host [B,K] int64, sumY_host [B,K] int64, t_host [B] int64; S_host unused.
+ *  EXP3Spec: S_host [B,K] fp64, n_host [B,K] int64 (pulls per arm, not used by the algorithm),
+ *            t_host [B] int64; sumY_host unused. */
+bs_status bs_bandit_read(const void* state, size_t state_bytes, bs_alg alg, int B, int K,
+                         int64_t* n_host, int64_t* sumY_host, double* S_host, int64_t* t_host,
+                         void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BANDITSPEC_H_ */

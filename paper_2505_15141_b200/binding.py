@@ -1,0 +1,214 @@
+"""ctypes binding of libbanditspec.so: the same entry points as include/banditspec.h.
+
+Argument marshalling only: tensors are passed as raw device pointers, every step of the
+round runs in the library's CUDA kernels on torch's current stream.  PyTorch is used for
+device memory and streams.  Importing this module loads the CUDA library and raises if it is
+missing -- there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libbanditspec.so")
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python __graft_entry__.py` "
+                      "(the CUDA library is required; there is no fallback path)")
+_lib = C.CDLL(LIB_PATH)
+
+BS_OK = 0
+BS_ERR_INVALID_ARG, BS_ERR_CUDA, BS_ERR_UNSUPPORTED, BS_ERR_WORKSPACE, BS_ERR_TIMEOUT, BS_ERR_DEVICE_DATA = 1, 2, 3, 4, 5, 6
+BS_F32, BS_BF16 = 0, 1
+BS_UCB, BS_EXP3 = 0, 1
+BS_DEV_BAD_GAMMA, BS_DEV_BAD_TOKEN, BS_DEV_NONFINITE, BS_DEV_RESIDUAL_FALLBACK = 1, 2, 4, 8
+BS_MAX_GAMMA, BS_MAX_ARMS, BS_MAX_BATCH = 31, 32, 4096
+
+_vp, _i, _f, _d, _sz = C.c_void_p, C.c_int, C.c_float, C.c_double, C.c_size_t
+
+# name -> (restype, argtypes); must list every symbol the header declares
+SIGNATURES = {
+    "bs_status_string": (C.c_char_p, [_i]),
+    "bs_workspace_bytes": (_sz, [_i, _i, _i]),
+    "bs_workspace_init": (_i, [_vp, _sz, _vp]),
+    "bs_get_device_status": (_i, [_vp, _sz, _i, _i, _i, _vp, _vp]),
+    "bs_softmax_verify": (_i, [_vp, _vp, _i, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "bs_residual_sample": (_i, [_vp, _vp, _i, _vp, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _sz, _vp]),
+    "bs_bandit_state_bytes": (_sz, [_i, _i, _i]),
+    "bs_bandit_init": (_i, [_vp, _sz, _i, _i, _i, _vp, _d, _vp]),
+    "bs_bandit_select": (_i, [_vp, _sz, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "bs_bandit_update": (_i, [_vp, _sz, _i, _i, _i, _vp, _vp, _vp, _vp]),
+    "bs_bandit_read": (_i, [_vp, _sz, _i, _i, _i, _vp, _vp, _vp, _vp, _vp]),
+}
+for _name, (_res, _args) in SIGNATURES.items():
+    _fn = getattr(_lib, _name)
+    _fn.restype, _fn.argtypes = _res, _args
+
+
+class BanditSpecError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {_lib.bs_status_string(code).decode()} (bs_status {code})")
+
+
+def _check(code: int, where: str) -> None:
+    if code != BS_OK:
+        raise BanditSpecError(code, where)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    assert t.is_contiguous(), "tensors must be contiguous"
+    return t.data_ptr()
+
+
+def _stream(stream=None) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return BS_F32
+    if t.dtype == torch.bfloat16:
+        return BS_BF16
+    raise TypeError(f"logits must be float32 or bfloat16, got {t.dtype}")
+
+
+# ---- workspace ---------------------------------------------------------------------
+
+def bs_workspace_bytes(B: int, Gmax: int, V: int) -> int:
+    return int(_lib.bs_workspace_bytes(B, Gmax, V))
+
+
+def bs_workspace_init(workspace: torch.Tensor, stream=None) -> None:
+    _check(_lib.bs_workspace_init(_ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
+           "bs_workspace_init")
+
+
+def new_workspace(B: int, Gmax: int, V: int, device="cuda") -> torch.Tensor:
+    """Allocate (through torch) and clear a workspace for the given limits."""
+    n = bs_workspace_bytes(B, Gmax, V)
+    if n == 0:
+        raise BanditSpecError(BS_ERR_UNSUPPORTED, "bs_workspace_bytes")
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    bs_workspace_init(ws)
+    return ws
+
+
+def bs_get_device_status(workspace: torch.Tensor, B: int, Gmax: int, V: int, stream=None) -> np.ndarray:
+    """Per-sequence status bits of the last verify/residual pair (synchronises)."""
+    host = np.zeros(B, dtype=np.int32)
+    code = _lib.bs_get_device_status(_ptr(workspace), workspace.numel(), B, Gmax, V,
+                                     host.ctypes.data_as(_vp), _stream(stream))
+    if code not in (BS_OK, BS_ERR_DEVICE_DATA):
+        raise BanditSpecError(code, "bs_get_device_status")
+    return host
+
+
+# ---- verification ---------------------------------------------------------------------
+
+def bs_softmax_verify(target_logits, draft_logits, draft_tokens, gamma, u_accept, temperature: float,
+                      accept_len, p_tok, q_tok, workspace, stream=None) -> None:
+    B, G1, V = target_logits.shape
+    _check(_lib.bs_softmax_verify(_ptr(target_logits), _ptr(draft_logits), _dtype_code(target_logits),
+                                  _ptr(draft_tokens), _ptr(gamma), _ptr(u_accept), float(temperature),
+                                  B, G1 - 1, V, _ptr(accept_len), _ptr(p_tok), _ptr(q_tok),
+                                  _ptr(workspace), workspace.numel(), _stream(stream)), "bs_softmax_verify")
+
+
+def bs_residual_sample(target_logits, draft_logits, draft_tokens, gamma, accept_len, u_resample,
+                       temperature: float, out_tokens, out_len, workspace, stream=None) -> None:
+    B, G1, V = target_logits.shape
+    _check(_lib.bs_residual_sample(_ptr(target_logits), _ptr(draft_logits), _dtype_code(target_logits),
+                                   _ptr(draft_tokens), _ptr(gamma), _ptr(accept_len), _ptr(u_resample),
+                                   float(temperature), B, G1 - 1, V, _ptr(out_tokens), _ptr(out_len),
+                                   _ptr(workspace), workspace.numel(), _stream(stream)), "bs_residual_sample")
+
+
+@dataclass
+class RoundOutput:
+    accept_len: torch.Tensor   # [B] int32, tau
+    p_tok: torch.Tensor        # [B, Gmax] fp32
+    q_tok: torch.Tensor        # [B, Gmax] fp32
+    out_tokens: torch.Tensor   # [B, Gmax+1] int32
+    out_len: torch.Tensor      # [B] int32, y = tau + 1
+    workspace: torch.Tensor
+
+
+def verify_round(target_logits, draft_logits, draft_tokens, gamma, u_accept, u_resample,
+                 temperature: float, workspace: Optional[torch.Tensor] = None) -> RoundOutput:
+    """Allocates the outputs and calls bs_softmax_verify then bs_residual_sample."""
+    B, G1, V = target_logits.shape
+    G = G1 - 1
+    dev = target_logits.device
+    if workspace is None:
+        workspace = new_workspace(B, G, V, dev)
+    accept_len = torch.empty(B, dtype=torch.int32, device=dev)
+    p_tok = torch.empty(B, G, dtype=torch.float32, device=dev)
+    q_tok = torch.empty(B, G, dtype=torch.float32, device=dev)
+    out_tokens = torch.empty(B, G + 1, dtype=torch.int32, device=dev)
+    out_len = torch.empty(B, dtype=torch.int32, device=dev)
+    bs_softmax_verify(target_logits, draft_logits, draft_tokens, gamma, u_accept, temperature,
+                      accept_len, p_tok, q_tok, workspace)
+    bs_residual_sample(target_logits, draft_logits, draft_tokens, gamma, accept_len, u_resample,
+                       temperature, out_tokens, out_len, workspace)
+    return RoundOutput(accept_len, p_tok, q_tok, out_tokens, out_len, workspace)
+
+
+# ---- bandits ---------------------------------------------------------------------------
+
+def bs_bandit_state_bytes(alg: int, B: int, K: int) -> int:
+    return int(_lib.bs_bandit_state_bytes(alg, B, K))
+
+
+def bs_bandit_init(state: torch.Tensor, alg: int, B: int, K: int, arm_gamma: Sequence[int],
+                   delta: float = 0.5, stream=None) -> None:
+    ag = np.ascontiguousarray(arm_gamma, dtype=np.int32)
+    assert ag.shape == (K,)
+    _check(_lib.bs_bandit_init(_ptr(state), state.numel(), alg, B, K, ag.ctypes.data_as(_vp),
+                               float(delta), _stream(stream)), "bs_bandit_init")
+
+
+def bs_bandit_select(state, alg: int, B: int, K: int, u_arm, active, arm, gamma, index_out=None,
+                     stream=None) -> None:
+    _check(_lib.bs_bandit_select(_ptr(state), state.numel(), alg, B, K, _ptr(u_arm), _ptr(active),
+                                 _ptr(arm), _ptr(gamma), _ptr(index_out), _stream(stream)), "bs_bandit_select")
+
+
+def bs_bandit_update(state, alg: int, B: int, K: int, arm, reward_y, active=None, stream=None) -> None:
+    _check(_lib.bs_bandit_update(_ptr(state), state.numel(), alg, B, K, _ptr(arm), _ptr(reward_y),
+                                 _ptr(active), _stream(stream)), "bs_bandit_update")
+
+
+def bs_bandit_read(state, alg: int, B: int, K: int, stream=None) -> dict:
+    """Sufficient statistics as host arrays: UCBSpec {n, sumY, t}; EXP3Spec {S, n, t}."""
+    t = np.zeros(B, dtype=np.int64)
+    if alg == BS_UCB:
+        n = np.zeros((B, K), dtype=np.int64)
+        sy = np.zeros((B, K), dtype=np.int64)
+        _check(_lib.bs_bandit_read(_ptr(state), state.numel(), alg, B, K, n.ctypes.data_as(_vp),
+                                   sy.ctypes.data_as(_vp), None, t.ctypes.data_as(_vp), _stream(stream)),
+               "bs_bandit_read")
+        return {"n": n, "sumY": sy, "t": t}
+    S = np.zeros((B, K), dtype=np.float64)
+    n = np.zeros((B, K), dtype=np.int64)
+    _check(_lib.bs_bandit_read(_ptr(state), state.numel(), alg, B, K, n.ctypes.data_as(_vp), None,
+                               S.ctypes.data_as(_vp), t.ctypes.data_as(_vp), _stream(stream)), "bs_bandit_read")
+    return {"S": S, "n": n, "t": t}
+
+
+def new_bandit(alg: int, B: int, arm_gamma: Sequence[int], delta: float = 0.5, device="cuda") -> torch.Tensor:
+    K = len(arm_gamma)
+    n = bs_bandit_state_bytes(alg, B, K)
+    if n == 0:
+        raise BanditSpecError(BS_ERR_UNSUPPORTED, "bs_bandit_state_bytes")
+    state = torch.empty(n, dtype=torch.uint8, device=device)
+    bs_bandit_init(state, alg, B, K, arm_gamma, delta)
+    return state

@@ -1,0 +1,222 @@
+// Arm selection and statistics update for B independent bandits, on the device so that a
+// decoding round never returns to the host: UCBSpec (Algorithm 4 / Algorithm 8 of the paper)
+// and EXP3Spec (Algorithm 5 / Algorithm 9).  The history H_t is kept as its sufficient
+// statistics.  All index arithmetic is fp64 with explicit (non-fused) multiplies and adds.
+//
+// State blob (device memory owned by the caller):
+//   [0, 256)  Header
+//   A  [B, K] 8-byte: UCBSpec n_i (int64)         | EXP3Spec S_i = sum of loss estimates (fp64)
+//   Bm [B, K] 8-byte: UCBSpec sum of rewards (int64) | EXP3Spec pulls per arm (int64, a statistic only)
+//   t  [B] int64  completed rounds
+//   ps [B] fp64   EXP3Spec: probability of the arm chosen by the pending select
+#include "bs_common.cuh"
+
+namespace bs {
+
+struct BanditHeader {
+    int alg, B, K, L;
+    double delta;
+    int arm_gamma[BS_MAX_ARMS];
+};
+static_assert(sizeof(BanditHeader) <= 256, "header must fit its slot");
+
+struct BanditState {
+    BanditHeader* hdr;
+    long long* A_i;      // aliases A_d
+    double* A_d;
+    long long* Bm;
+    long long* t;
+    double* ps;
+};
+
+__host__ __device__ inline size_t bandit_bytes(int B, int K) {
+    return 256 + align_up(sizeof(double) * (size_t)B * K, 256) * 2 + align_up(sizeof(double) * (size_t)B, 256) * 2;
+}
+
+__host__ __device__ inline BanditState bandit_view(void* state, int B, int K) {
+    char* s = static_cast<char*>(state);
+    BanditState v;
+    v.hdr = reinterpret_cast<BanditHeader*>(s);
+    size_t o = 256;
+    v.A_i = reinterpret_cast<long long*>(s + o);
+    v.A_d = reinterpret_cast<double*>(s + o);
+    o += align_up(sizeof(double) * (size_t)B * K, 256);
+    v.Bm = reinterpret_cast<long long*>(s + o);
+    o += align_up(sizeof(double) * (size_t)B * K, 256);
+    v.t = reinterpret_cast<long long*>(s + o);
+    o += align_up(sizeof(double) * (size_t)B, 256);
+    v.ps = reinterpret_cast<double*>(s + o);
+    return v;
+}
+
+// cr_{i,t} = (L/2) sqrt( (1+n)/n^2 * (1 + 2 ln( K t^2 sqrt(1+n) / delta )) )
+__device__ inline double confidence_radius(int L, int K, long long t, long long n, double delta) {
+    const double n1 = __dadd_rn(1.0, (double)n);
+    const double arg = __ddiv_rn(__dmul_rn((double)(K * t * t), sqrt(n1)), delta);
+    const double inner = __dadd_rn(1.0, __dmul_rn(2.0, log(arg)));
+    const double frac = __ddiv_rn(n1, (double)(n * n));
+    return __dmul_rn(__ddiv_rn((double)L, 2.0), sqrt(__dmul_rn(frac, inner)));
+}
+
+// One warp per sequence, lane i = arm i.
+__global__ void __launch_bounds__(128) bandit_select_kernel(void* state, int alg, int B, int K,
+                                                           const float* u_arm, const uint8_t* active,
+                                                           int32_t* arm_out, int32_t* gamma_out, double* index_out) {
+    const int b = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (b >= B) return;
+    const BanditState s = bandit_view(state, B, K);
+    if (active && !active[b]) {
+        if (lane == 0) { arm_out[b] = -1; gamma_out[b] = 0; }
+        if (index_out && lane < K) index_out[(size_t)b * K + lane] = nan("");
+        return;
+    }
+    const int L = s.hdr->L;
+    const long long t = s.t[b];
+    int arm;
+    double shown = nan("");
+    if (alg == BS_UCB) {
+        if (t < K) {
+            arm = (int)t;                                   // rounds 1..K: arms 1..K in order
+        } else {
+            double idx = -INFINITY;
+            if (lane < K) {
+                const long long n = s.A_i[(size_t)b * K + lane];
+                const long long sy = s.Bm[(size_t)b * K + lane];
+                idx = n > 0 ? __dadd_rn(__ddiv_rn((double)sy, (double)n), confidence_radius(L, K, t, n, s.hdr->delta))
+                            : INFINITY;
+                shown = idx;
+            }
+            int best = lane;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const double oi = __shfl_xor_sync(0xffffffffu, idx, o);
+                const int ob = __shfl_xor_sync(0xffffffffu, best, o);
+                if (oi > idx || (oi == idx && ob < best)) { idx = oi; best = ob; }   // ties: lowest arm
+            }
+            arm = best;
+        }
+    } else {
+        // p_i proportional to exp(-eta_t * S_i), eta_t = sqrt(ln K / (t K)), t = this round's index
+        const double eta = sqrt(__ddiv_rn(log((double)K), (double)((t + 1) * K)));
+        const double Si = lane < K ? s.A_d[(size_t)b * K + lane] : INFINITY;
+        double mn = Si;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mn = fmin(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+        const double w = lane < K ? exp(__dmul_rn(-eta, __dadd_rn(Si, -mn))) : 0.0;
+        double tot = 0.0;
+        for (int i = 0; i < K; ++i) tot = __dadd_rn(tot, __shfl_sync(0xffffffffu, w, i));   // arm order
+        const double pi = __ddiv_rn(w, tot);
+        shown = pi;
+        const double u = (double)u_arm[b];
+        double c = 0.0, psel = 0.0;
+        arm = -1;
+        for (int i = 0; i < K; ++i) {
+            const double p = __shfl_sync(0xffffffffu, pi, i);
+            c = __dadd_rn(c, p);
+            if (arm < 0 && (c > u || i == K - 1)) { arm = i; psel = p; }
+        }
+        if (lane == 0) s.ps[b] = psel;
+    }
+    if (lane == 0) {
+        arm_out[b] = arm;
+        gamma_out[b] = s.hdr->arm_gamma[arm];
+    }
+    if (index_out && lane < K) index_out[(size_t)b * K + lane] = shown;
+}
+
+__global__ void bandit_update_kernel(void* state, int alg, int B, int K, const int32_t* arm,
+                                     const int32_t* reward_y, const uint8_t* active) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    if (active && !active[b]) return;
+    const BanditState s = bandit_view(state, B, K);
+    const int a = arm[b];
+    if (a < 0 || a >= K) return;
+    const int L = s.hdr->L;
+    const int y = max(1, min(reward_y[b], L + 1));          // accepted length, bonus included
+    if (alg == BS_UCB) {
+        s.A_i[(size_t)b * K + a] += 1;
+        s.Bm[(size_t)b * K + a] += y;
+    } else {
+        // loss estimate (L + 1 - y) / (L p_{t, I_t}); the other arms' estimates are zero
+        const double z = __ddiv_rn((double)(L + 1 - y), __dmul_rn((double)L, s.ps[b]));
+        s.A_d[(size_t)b * K + a] = __dadd_rn(s.A_d[(size_t)b * K + a], z);
+        s.Bm[(size_t)b * K + a] += 1;
+    }
+    s.t[b] += 1;
+}
+
+}  // namespace bs
+
+using namespace bs;
+
+static bool bandit_args_ok(const void* state, size_t state_bytes, int alg, int B, int K) {
+    return state && (alg == BS_UCB || alg == BS_EXP3) && B >= 1 && B <= BS_MAX_BATCH && K >= 1 && K <= BS_MAX_ARMS &&
+           state_bytes >= bandit_bytes(B, K) && (reinterpret_cast<uintptr_t>(state) & 255) == 0;
+}
+
+extern "C" size_t bs_bandit_state_bytes(bs_alg alg, int B, int K) {
+    if ((alg != BS_UCB && alg != BS_EXP3) || B < 1 || B > BS_MAX_BATCH || K < 1 || K > BS_MAX_ARMS) return 0;
+    return bandit_bytes(B, K);
+}
+
+extern "C" bs_status bs_bandit_init(void* state, size_t state_bytes, bs_alg alg, int B, int K,
+                                    const int32_t* arm_gamma_host, double delta, void* stream) {
+    if (!bandit_args_ok(state, state_bytes, alg, B, K) || !arm_gamma_host) return BS_ERR_INVALID_ARG;
+    if (alg == BS_UCB && !(delta > 0.0)) return BS_ERR_INVALID_ARG;
+    BanditHeader h;
+    h.alg = alg; h.B = B; h.K = K; h.L = 0; h.delta = delta;
+    for (int i = 0; i < BS_MAX_ARMS; ++i) h.arm_gamma[i] = 0;
+    for (int i = 0; i < K; ++i) {
+        if (arm_gamma_host[i] < 0 || arm_gamma_host[i] > BS_MAX_GAMMA) return BS_ERR_INVALID_ARG;
+        h.arm_gamma[i] = arm_gamma_host[i];
+        if (arm_gamma_host[i] > h.L) h.L = arm_gamma_host[i];
+    }
+    if (h.L < 1) return BS_ERR_INVALID_ARG;     // the radius and the loss estimate divide by L
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemsetAsync(state, 0, bandit_bytes(B, K), st);
+    // pageable host source: the copy is staged before the call returns, so `h` may go out of scope
+    if (e == cudaSuccess) e = cudaMemcpyAsync(state, &h, sizeof(h), cudaMemcpyHostToDevice, st);
+    return cuda_status(e);
+}
+
+extern "C" bs_status bs_bandit_select(void* state, size_t state_bytes, bs_alg alg, int B, int K,
+                                      const float* u_arm, const uint8_t* active,
+                                      int32_t* arm, int32_t* gamma, double* index_out, void* stream) {
+    if (!bandit_args_ok(state, state_bytes, alg, B, K) || !arm || !gamma) return BS_ERR_INVALID_ARG;
+    if (alg == BS_EXP3 && !u_arm) return BS_ERR_INVALID_ARG;
+    const int warps_per_cta = 4;
+    bandit_select_kernel<<<div_up(B, warps_per_cta), warps_per_cta * 32, 0, static_cast<cudaStream_t>(stream)>>>(
+        state, alg, B, K, u_arm, active, arm, gamma, index_out);
+    return cuda_status(cudaGetLastError());
+}
+
+extern "C" bs_status bs_bandit_update(void* state, size_t state_bytes, bs_alg alg, int B, int K,
+                                      const int32_t* arm, const int32_t* reward_y, const uint8_t* active,
+                                      void* stream) {
+    if (!bandit_args_ok(state, state_bytes, alg, B, K) || !arm || !reward_y) return BS_ERR_INVALID_ARG;
+    bandit_update_kernel<<<div_up(B, 128), 128, 0, static_cast<cudaStream_t>(stream)>>>(state, alg, B, K, arm,
+                                                                                        reward_y, active);
+    return cuda_status(cudaGetLastError());
+}
+
+extern "C" bs_status bs_bandit_read(const void* state, size_t state_bytes, bs_alg alg, int B, int K,
+                                    int64_t* n_host, int64_t* sumY_host, double* S_host, int64_t* t_host,
+                                    void* stream) {
+    if (!bandit_args_ok(state, state_bytes, alg, B, K)) return BS_ERR_INVALID_ARG;
+    const BanditState s = bandit_view(const_cast<void*>(state), B, K);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaSuccess;
+    const size_t bk = sizeof(double) * (size_t)B * K;
+    if (alg == BS_UCB) {
+        if (n_host && e == cudaSuccess) e = cudaMemcpyAsync(n_host, s.A_i, bk, cudaMemcpyDeviceToHost, st);
+        if (sumY_host && e == cudaSuccess) e = cudaMemcpyAsync(sumY_host, s.Bm, bk, cudaMemcpyDeviceToHost, st);
+    } else {
+        if (S_host && e == cudaSuccess) e = cudaMemcpyAsync(S_host, s.A_d, bk, cudaMemcpyDeviceToHost, st);
+        if (n_host && e == cudaSuccess) e = cudaMemcpyAsync(n_host, s.Bm, bk, cudaMemcpyDeviceToHost, st);
+    }
+    if (t_host && e == cudaSuccess) e = cudaMemcpyAsync(t_host, s.t, sizeof(int64_t) * B, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    return cuda_status(e);
+}

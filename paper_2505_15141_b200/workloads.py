@@ -242,15 +242,18 @@ class RoundInputs:
 
 
 def make_round(w: Workload, rnd: int, arm: Optional[np.ndarray] = None,
-               device="cpu") -> RoundInputs:
+               device="cpu", B: Optional[int] = None) -> RoundInputs:
     """Everything one verification round reads, for round `rnd` (1-based).
-    `arm` [B] is the arm each sequence plays (None = arm 0 for all)."""
+    `arm` [B] is the arm each sequence plays (None = arm 0 for all).  `B` overrides the batch
+    size (the first B sequences' arms / noise scales / uniforms; fresh logits)."""
     if arm is None:
         arm = np.zeros(w.B, dtype=np.int32)
     arm = np.asarray(arm, dtype=np.int32)
     gamma = np.asarray(w.arm_gamma, dtype=np.int32)[arm]
     sig = round_sigma(w, rnd, arm)
-    t, d = make_logits(w, rnd, sig, device=device)
-    un = round_uniforms(w.seed, rnd, w.B, w.Gmax)
+    nb = w.B if B is None else B
+    t, d = make_logits(w, rnd, sig, device=device, B=nb)
+    un = round_uniforms(w.seed, rnd, nb, w.Gmax)
+    gamma, sig = gamma[:nb], sig[:nb]
     tok = draw_draft_tokens(d, w.temperature, un.u_draft)
     return RoundInputs(target=t, draft=d, tokens=tok, gamma=gamma, uniforms=un, sigma=sig)

@@ -1,0 +1,285 @@
+"""CUDA path against the CPU oracle, element by element, through the C ABI (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import bandit as ob
+from oracle import verify as ov
+from paper_2505_15141_b200 import workloads as wl
+import parity
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _random_round(rng, B, G, V, dtype, T, sigma=1.0, gamma=None, std=3.0):
+    g = torch.Generator(device="cpu"); g.manual_seed(int(rng.integers(1 << 30)))
+    t = torch.randn(B, G + 1, V, generator=g) * std
+    d = t[:, :G] + sigma * torch.randn(B, G, V, generator=g)
+    t, d = t.to(dtype).to(DEV), d.to(dtype).to(DEV)
+    gamma = rng.integers(0, G + 1, size=B).astype(np.int32) if gamma is None else np.asarray(gamma, np.int32)
+    un = wl.RoundUniforms(rng.random((B, G)).astype(np.float32) * 0.999 + 0.0005,
+                          rng.random(B).astype(np.float32) * 0.999 + 0.0005,
+                          rng.random(B).astype(np.float32), rng.random((B, G)).astype(np.float32) * 0.999 + 0.0005)
+    tok = wl.draw_draft_tokens(d, T, un.u_draft)
+    return wl.RoundInputs(target=t, draft=d, tokens=tok, gamma=gamma, uniforms=un)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("V", [1, 7, 1000, 1001, 8192, 8193, 20011, 40000])
+def test_unit_parity_ragged_vocab(lib, dtype, V):
+    """Several tiles and ragged tails: V below / at / above one segment, odd V (rows not 16-byte aligned)."""
+    rng = np.random.default_rng(V)
+    tally = parity.Tally()
+    for T in (1.0, 0.6):
+        rnd = _random_round(rng, B=5, G=4, V=V, dtype=dtype, T=T)
+        out = parity.gpu_round(lib, rnd, T)
+        parity.check_round(out, rnd, T, tally, where=f"V={V} T={T}")
+        st = lib.bs_get_device_status(out.workspace, 5, 4, V)
+        assert (st & ~lib.BS_DEV_RESIDUAL_FALLBACK == 0).all()
+    assert tally.sequences == 10
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_greedy_parity_with_ties(lib, dtype):
+    rng = np.random.default_rng(3)
+    tally = parity.Tally()
+    for V in (5, 4096, 33333):
+        B, G = 6, 5
+        # coarse values -> many exact ties for the arg-max
+        t = torch.as_tensor(rng.integers(-4, 5, size=(B, G + 1, V)).astype(np.float32)).to(dtype).to(DEV)
+        gamma = rng.integers(0, G + 1, size=B).astype(np.int32)
+        tok = t[:, :G].float().argmax(dim=-1).to(torch.int32)           # the right token ...
+        flip = torch.as_tensor(rng.random((B, G)) < 0.3, device=DEV)
+        tok = torch.where(flip, (tok + 1) % V, tok).to(torch.int32)      # ... except where flipped
+        un = wl.round_uniforms(1, 1, B, G)
+        rnd = wl.RoundInputs(target=t, draft=t[:, :G].contiguous(), tokens=tok.contiguous(), gamma=gamma, uniforms=un)
+        out = parity.gpu_round(lib, rnd, 0.0)
+        parity.check_round(out, rnd, 0.0, tally, where=f"greedy V={V}")
+    assert tally.flagged_accept == 0 and tally.flagged_token == 0
+
+
+def test_edge_cases(lib):
+    rng = np.random.default_rng(11)
+    tally = parity.Tally()
+    B, G, V = 8, 6, 3000
+    # gamma = 0 (canonical decoding), gamma = Gmax, identical models (accept all),
+    # hopeless drafts (reject at first), tokens at 0 and V-1, extreme logits, identical logits
+    rnd = _random_round(rng, B, G, V, torch.float32, 1.0, gamma=[0, G, G, G, 3, 3, 2, 1])
+    rnd.draft[2] = rnd.target[2, :G]                                     # q == p
+    rnd.draft[3] = -rnd.target[3, :G] * 3                                # far apart
+    rnd.target[4] *= 26.0; rnd.draft[4] *= 26.0                          # logits up to about +-80
+    rnd.target[5] = 1.25; rnd.draft[5] = -0.5                            # constant rows
+    tok = wl.draw_draft_tokens(rnd.draft, 1.0, rnd.uniforms.u_draft)
+    tok[6, 0] = 0; tok[6, 1] = V - 1
+    rnd.tokens = tok.contiguous()
+    out = parity.gpu_round(lib, rnd, 1.0)
+    refs = parity.check_round(out, rnd, 1.0, tally, where="edge")
+    assert refs[0].y == 1 and refs[2].tau == G and refs[2].y == G + 1
+    assert refs[3].tau <= 1
+    st = lib.bs_get_device_status(out.workspace, B, G, V)
+    assert (st & ~lib.BS_DEV_RESIDUAL_FALLBACK == 0).all()
+    # Gmax = 0: a batch of canonical-decoding steps
+    rnd0 = _random_round(rng, 3, 0, 5000, torch.bfloat16, 0.9)
+    out0 = parity.gpu_round(lib, rnd0, 0.9)
+    parity.check_round(out0, rnd0, 0.9, tally, where="Gmax=0")
+    # the largest supported speculation length
+    rndL = _random_round(rng, 2, lib.BS_MAX_GAMMA, 600, torch.float32, 1.0, sigma=0.2,
+                         gamma=[lib.BS_MAX_GAMMA, 17])
+    outL = parity.gpu_round(lib, rndL, 1.0)
+    parity.check_round(outL, rndL, 1.0, tally, where="Gmax=31")
+
+
+def test_device_data_errors_are_reported_not_fatal(lib):
+    rng = np.random.default_rng(12)
+    B, G, V = 4, 3, 500
+    rnd = _random_round(rng, B, G, V, torch.float32, 1.0, gamma=[3, 3, 3, 3])
+    rnd.tokens[1, 1] = V + 7                       # token out of range -> position rejected
+    rnd.gamma = np.array([3, 3, 9, 3], np.int32)   # gamma out of range -> processed as gamma 0
+    rnd.target[3, 0, 5] = float("nan")             # non-finite normaliser
+    out = parity.gpu_round(lib, rnd, 1.0)
+    st = lib.bs_get_device_status(out.workspace, B, G, V)
+    assert st[0] == 0
+    assert st[1] & lib.BS_DEV_BAD_TOKEN and int(out.accept_len[1]) <= 1
+    assert st[2] & lib.BS_DEV_BAD_GAMMA and int(out.accept_len[2]) == 0 and int(out.out_len[2]) == 1
+    assert st[3] & lib.BS_DEV_NONFINITE
+    # the context is still usable and sequence 0 is still right
+    tally = parity.Tally()
+    parity.check_round(out, rnd, 1.0, tally, seqs=[0], where="after errors")
+
+
+def test_same_inputs_twice_are_bit_identical(lib):
+    rng = np.random.default_rng(13)
+    rnd = _random_round(rng, 16, 5, 32000, torch.bfloat16, 0.7)
+    ws = lib.new_workspace(16, 5, 32000, DEV)
+    a = parity.gpu_round(lib, rnd, 0.7, ws)
+    a = [x.clone() for x in (a.accept_len, a.p_tok, a.q_tok, a.out_tokens, a.out_len)]
+    b = parity.gpu_round(lib, rnd, 0.7, ws)
+    for x, y in zip(a, (b.accept_len, b.p_tok, b.q_tok, b.out_tokens, b.out_len)):
+        assert torch.equal(x, y)
+
+
+def test_batch_split_equals_whole_batch(lib):
+    """Sequences are independent: two half batches give exactly the whole batch's result."""
+    rng = np.random.default_rng(14)
+    rnd = _random_round(rng, 8, 4, 9000, torch.float32, 1.0)
+    whole = parity.gpu_round(lib, rnd, 1.0)
+    for lo, hi in ((0, 4), (4, 8)):
+        part = wl.RoundInputs(rnd.target[lo:hi].contiguous(), rnd.draft[lo:hi].contiguous(),
+                              rnd.tokens[lo:hi].contiguous(), rnd.gamma[lo:hi],
+                              wl.RoundUniforms(rnd.uniforms.u_accept[lo:hi], rnd.uniforms.u_resample[lo:hi],
+                                               rnd.uniforms.u_arm[lo:hi], rnd.uniforms.u_draft[lo:hi]))
+        o = parity.gpu_round(lib, part, 1.0)
+        assert torch.equal(o.accept_len, whole.accept_len[lo:hi])
+        assert torch.equal(o.out_tokens, whole.out_tokens[lo:hi])
+        assert torch.equal(o.p_tok, whole.p_tok[lo:hi])
+
+
+# ---- bandits -------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("alg_name", ["ucb", "exp3"])
+def test_bandit_trajectories_match_the_oracle(lib, alg_name):
+    rng = np.random.default_rng(21)
+    B, arm_gamma = 37, (1, 3, 5, 8)
+    K = len(arm_gamma)
+    alg = lib.BS_UCB if alg_name == "ucb" else lib.BS_EXP3
+    state = lib.new_bandit(alg, B, arm_gamma, 0.5, DEV)
+    ref = ob.UCBSpec(B, arm_gamma, 0.5) if alg_name == "ucb" else ob.EXP3Spec(B, arm_gamma)
+    arm_d = torch.empty(B, dtype=torch.int32, device=DEV); gam_d = torch.empty_like(arm_d)
+    idx_d = torch.empty(B, K, dtype=torch.float64, device=DEV)
+    flagged_total = 0
+    for t in range(300):
+        u = rng.random(B).astype(np.float32)
+        lib.bs_bandit_select(state, alg, B, K, torch.as_tensor(u, device=DEV), None, arm_d, gam_d, idx_d)
+        arm = arm_d.cpu().numpy().astype(np.int64)
+        a_ref, g_ref, flagged = (ref.select() if alg_name == "ucb" else ref.select(u))
+        shown = idx_d.cpu().numpy()
+        if alg_name == "exp3":
+            assert np.allclose(shown, ref.last_p, rtol=1e-12, atol=1e-15)
+        elif t >= K:
+            assert np.allclose(shown, ref.last_index, rtol=1e-12)
+        bad = (arm != a_ref) & ~flagged
+        assert not bad.any(), (t, np.nonzero(bad))
+        for b in np.nonzero(arm != a_ref)[0]:
+            flagged_total += 1
+            if alg_name == "exp3":
+                ref.p_sel[b] = ref.last_p[b][arm[b]]
+        assert (gam_d.cpu().numpy() == np.asarray(arm_gamma)[arm]).all()
+        y = np.minimum(1 + rng.geometric(0.4, size=B) * (arm + 1) // 2, np.asarray(arm_gamma)[arm] + 1).astype(np.int32)
+        lib.bs_bandit_update(state, alg, B, K, arm_d, torch.as_tensor(y, device=DEV))
+        ref.update(arm, y)
+    st = lib.bs_bandit_read(state, alg, B, K)
+    assert (st["t"] == 300).all()
+    if alg_name == "ucb":
+        assert (st["n"] == ref.n).all() and (st["sumY"] == ref.sumY).all()
+    else:
+        assert np.allclose(st["S"], ref.S, rtol=1e-10)
+    assert flagged_total <= 2
+
+
+def test_bandit_golden_tables_on_device(lib):
+    from conftest import golden_lines
+    rows = golden_lines("ucbspec_scripted.txt")
+    state = lib.new_bandit(lib.BS_UCB, 1, (2, 4, 6), 0.5, DEV)
+    arm_d = torch.empty(1, dtype=torch.int32, device=DEV); gam_d = torch.empty_like(arm_d)
+    idx_d = torch.empty(1, 3, dtype=torch.float64, device=DEV)
+    for f in rows:
+        lib.bs_bandit_select(state, lib.BS_UCB, 1, 3, None, None, arm_d, gam_d, idx_d)
+        assert int(arm_d[0]) == int(f[1])
+        if f[3] != "rr":
+            assert np.allclose(idx_d.cpu().numpy()[0], [float(x) for x in f[3:6]], atol=2e-6)
+        lib.bs_bandit_update(state, lib.BS_UCB, 1, 3, arm_d, torch.tensor([int(f[2])], dtype=torch.int32, device=DEV))
+    rows = golden_lines("exp3spec_scripted.txt")
+    state = lib.new_bandit(lib.BS_EXP3, 1, (2, 4), 0.5, DEV)
+    idx_d = torch.empty(1, 2, dtype=torch.float64, device=DEV)
+    for f, u in zip(rows, [0.3, 0.9, 0.5, 0.2, 0.7]):
+        lib.bs_bandit_select(state, lib.BS_EXP3, 1, 2, torch.tensor([u], dtype=torch.float32, device=DEV), None,
+                             arm_d, gam_d, idx_d)
+        assert int(arm_d[0]) == int(f[4])
+        assert np.allclose(idx_d.cpu().numpy()[0], [float(f[2]), float(f[3])], atol=1e-6)
+        lib.bs_bandit_update(state, lib.BS_EXP3, 1, 2, arm_d, torch.tensor([int(f[5])], dtype=torch.int32, device=DEV))
+        S = lib.bs_bandit_read(state, lib.BS_EXP3, 1, 2)["S"][0]
+        assert np.allclose(S, [float(f[7]), float(f[8])], atol=1e-6)
+
+
+def test_bandit_checkpoint_and_active_mask(lib):
+    B, arm_gamma = 5, (2, 4, 6)
+    rng = np.random.default_rng(5)
+    ys = rng.integers(1, 8, size=(64, B)).astype(np.int32)
+
+    def run(state, lo, hi, arms):
+        arm_d = torch.empty(B, dtype=torch.int32, device=DEV); gam_d = torch.empty_like(arm_d)
+        for t in range(lo, hi):
+            lib.bs_bandit_select(state, lib.BS_UCB, B, 3, None, None, arm_d, gam_d)
+            arms.append(arm_d.cpu().numpy().copy())
+            lib.bs_bandit_update(state, lib.BS_UCB, B, 3, arm_d, torch.as_tensor(ys[t], device=DEV))
+
+    a1, a2 = [], []
+    s1 = lib.new_bandit(lib.BS_UCB, B, arm_gamma, 0.5, DEV)
+    run(s1, 0, 64, a1)
+    s2 = lib.new_bandit(lib.BS_UCB, B, arm_gamma, 0.5, DEV)
+    run(s2, 0, 32, a2)
+    saved = s2.cpu()                                   # checkpoint = the bytes of the state
+    s3 = saved.to(DEV)
+    run(s3, 32, 64, a2)
+    assert np.array_equal(np.stack(a1), np.stack(a2))
+    # inactive sequences are frozen
+    s4 = lib.new_bandit(lib.BS_UCB, B, arm_gamma, 0.5, DEV)
+    act = torch.tensor([1, 0, 1, 0, 1], dtype=torch.uint8, device=DEV)
+    arm_d = torch.empty(B, dtype=torch.int32, device=DEV); gam_d = torch.empty_like(arm_d)
+    lib.bs_bandit_select(s4, lib.BS_UCB, B, 3, None, act, arm_d, gam_d)
+    assert arm_d.cpu().tolist() == [0, -1, 0, -1, 0] and gam_d.cpu().tolist() == [2, 0, 2, 0, 2]
+    lib.bs_bandit_update(s4, lib.BS_UCB, B, 3, arm_d, torch.full((B,), 2, dtype=torch.int32, device=DEV), act)
+    assert lib.bs_bandit_read(s4, lib.BS_UCB, B, 3)["t"].tolist() == [1, 0, 1, 0, 1]
+
+
+# ---- closed-loop rounds on the named workloads -----------------------------------------------
+
+def test_closed_loop_tiny_ucb(lib):
+    t = parity.closed_loop(lib, wl.WORKLOADS["tiny_ucb"], 64, DEV)
+    assert t.sequences == 4 * 64 and t.flagged_accept + t.flagged_token <= 3
+
+
+def test_closed_loop_tiny_ucb_greedy(lib):
+    t = parity.closed_loop(lib, wl.WORKLOADS["tiny_ucb_greedy"], 64, DEV)
+    assert t.flagged_accept == 0 and t.flagged_token == 0
+
+
+def test_closed_loop_llama2_fixed(lib):
+    w = wl.WORKLOADS["llama2_fixed"]
+    t = parity.closed_loop(lib, w, 40, DEV)
+    assert t.sequences == 32 * 40
+    assert t.flagged_accept + t.flagged_token <= 0.01 * t.sequences + 2
+
+
+def test_closed_loop_llama3_ucb_full_size(lib):
+    """Full-size ragged batch in the launch configuration the benchmark times; the oracle replays
+    a sample of sequences each round, the bandits of all sequences are compared every round."""
+    w = wl.WORKLOADS["llama3_ucb"]
+    t = parity.closed_loop(lib, w, 24, DEV, sample=[0, 1, 17, 40, 63])
+    assert t.sequences == 5 * 24 and t.flagged_accept + t.flagged_token <= 3
+
+
+def test_closed_loop_qwen_exp3_full_size(lib):
+    w = wl.WORKLOADS["qwen_exp3"]
+    t = parity.closed_loop(lib, w, 12, DEV, sample=[0, 100, 255])
+    assert t.sequences == 3 * 12 and t.flagged_accept + t.flagged_token <= 3
+
+
+def test_full_size_invariants_all_sequences(lib):
+    """Properties that hold for every sequence at full size: 1 <= y <= gamma + 1, accepted prefix
+    equals the drafts, the emitted token is in range, identical models accept everything."""
+    w = wl.WORKLOADS["llama3_ucb"]
+    arm = np.arange(w.B) % w.K
+    rnd = wl.make_round(w, 3, arm, device=DEV)
+    rnd.draft[:8] = rnd.target[:8, :w.Gmax]
+    rnd.tokens = wl.draw_draft_tokens(rnd.draft, w.temperature, rnd.uniforms.u_draft)
+    out = parity.gpu_round(lib, rnd, w.temperature)
+    y = out.out_len.cpu().numpy(); tau = out.accept_len.cpu().numpy(); ot = out.out_tokens.cpu().numpy()
+    tk = rnd.tokens.cpu().numpy()
+    assert ((y >= 1) & (y <= rnd.gamma + 1) & (y == tau + 1)).all()
+    assert (tau[:8] == rnd.gamma[:8]).all()
+    for b in range(w.B):
+        assert (ot[b, :tau[b]] == tk[b, :tau[b]]).all() and 0 <= ot[b, tau[b]] < w.V and (ot[b, y[b]:] == -1).all()
+    p = out.p_tok.cpu().numpy(); q = out.q_tok.cpu().numpy()
+    assert np.allclose(p[:8], q[:8], atol=1e-7) and (p >= 0).all() and (p <= 1 + 1e-6).all()
