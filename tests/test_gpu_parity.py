@@ -155,9 +155,9 @@ def test_bandit_trajectories_match_the_oracle(lib, alg_name):
         a_ref, g_ref, flagged = (ref.select() if alg_name == "ucb" else ref.select(u))
         shown = idx_d.cpu().numpy()
         if alg_name == "exp3":
-            assert np.allclose(shown, ref.last_p, rtol=1e-12, atol=1e-15)
+            assert np.allclose(shown, ref.last_p, rtol=1e-9, atol=1e-15)
         elif t >= K:
-            assert np.allclose(shown, ref.last_index, rtol=1e-12)
+            assert np.allclose(shown, ref.last_index, rtol=1e-11)
         bad = (arm != a_ref) & ~flagged
         assert not bad.any(), (t, np.nonzero(bad))
         for b in np.nonzero(arm != a_ref)[0]:
