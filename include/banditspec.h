@@ -65,8 +65,13 @@ typedef enum { BS_UCB = 0, BS_EXP3 = 1 } bs_alg;
 #define BS_MAX_GAMMA   31      /* Gmax <= 31 (one warp scans the accept flags) */
 #define BS_MAX_ARMS    32      /* K <= 32 (one lane per arm) */
 #define BS_MAX_BATCH   4096    /* B <= 4096 */
+#define BS_MAX_VOCAB   (1 << 20) /* V <= 1048576 */
 
 const char* bs_status_string(bs_status s);
+
+/* Text of the last CUDA runtime error that made a call on this thread return BS_ERR_CUDA
+ * (diagnostics only; "no error" if there was none). */
+const char* bs_last_cuda_error(void);
 
 /* ---- workspace ------------------------------------------------------------------ */
 

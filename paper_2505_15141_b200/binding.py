@@ -34,6 +34,7 @@ _vp, _i, _f, _d, _sz = C.c_void_p, C.c_int, C.c_float, C.c_double, C.c_size_t
 # name -> (restype, argtypes); must list every symbol the header declares
 SIGNATURES = {
     "bs_status_string": (C.c_char_p, [_i]),
+    "bs_last_cuda_error": (C.c_char_p, []),
     "bs_workspace_bytes": (_sz, [_i, _i, _i]),
     "bs_workspace_init": (_i, [_vp, _sz, _vp]),
     "bs_get_device_status": (_i, [_vp, _sz, _i, _i, _i, _vp, _vp]),
@@ -53,7 +54,8 @@ for _name, (_res, _args) in SIGNATURES.items():
 class BanditSpecError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
-        super().__init__(f"{where}: {_lib.bs_status_string(code).decode()} (bs_status {code})")
+        detail = f" [{_lib.bs_last_cuda_error().decode()}]" if code == BS_ERR_CUDA else ""
+        super().__init__(f"{where}: {_lib.bs_status_string(code).decode()} (bs_status {code}){detail}")
 
 
 def _check(code: int, where: str) -> None:

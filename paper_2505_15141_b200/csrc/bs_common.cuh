@@ -12,7 +12,7 @@ namespace bs {
 
 constexpr int kThreads = 256;              // threads per CTA of the streaming kernels
 constexpr int kWarps = kThreads / 32;
-constexpr int kSegBytes = 32768;           // bytes of one row segment = one work item
+constexpr int kSegBytes = 16384;           // bytes of one row segment = one work item = one pipeline stage
 constexpr int kSegElemsMin = kSegBytes / 4;  // segment length of the widest dtype (fp32)
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -21,15 +21,18 @@ __host__ __device__ inline int div_up(int a, int b) { return (a + b - 1) / b; }
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // Workspace regions (all offsets multiples of 256 bytes).
-//   ticket_verify [B] u32   arrival counters of the statistics kernel (zero between calls)
-//   ticket_resid  [B] u32   arrival counters of the resampling kernel (zero between calls)
-//   status        [B] i32   device-data status bits of the last call pair
+//   ticket_verify [B] u32     per-sequence arrival counters of the statistics kernel (zero between calls)
+//   ticket_resid  [B] u32     per-sequence arrival counters of the resampling kernel (zero between calls)
+//   ticket_row    [B, R] u32  per-row arrival counters of the statistics kernel (zero between calls)
+//   status        [B] i32     device-data status bits of the last call pair
+//   abort         [1] i32     set when a bounded pipeline wait gave up (reported as BS_ERR_TIMEOUT)
 //   row_stats     [B, R, 2] f32, R = 2*Gmax+1: (raw max logit, Z) per row; greedy: (max, arg-max bits)
 //                 rows 0..Gmax are target rows, rows Gmax+1..2*Gmax are draft rows
-//   partial       [B, R, S, 2] f32, S = ceil(V / 8192): per-segment (max, Z) / (max, arg-max)
+//   partial       [B, R, S, 2] f32, S = ceil(V / 4096): per-segment (max, Z) / (max, arg-max)
 //   resid_partial [B, S] f32  per-segment residual mass
 struct Workspace {
-    size_t off_ticket_verify, off_ticket_resid, off_status, off_row_stats, off_partial, off_resid_partial, total;
+    size_t off_ticket_verify, off_ticket_resid, off_ticket_row, off_status, off_abort, off_row_stats, off_partial,
+        off_resid_partial, total;
     int R, S;
 };
 
@@ -40,7 +43,9 @@ __host__ __device__ inline Workspace workspace_layout(int B, int Gmax, int V) {
     size_t o = 0;
     w.off_ticket_verify = o; o = align_up(o + sizeof(uint32_t) * (size_t)B, 256);
     w.off_ticket_resid = o;  o = align_up(o + sizeof(uint32_t) * (size_t)B, 256);
+    w.off_ticket_row = o;    o = align_up(o + sizeof(uint32_t) * (size_t)B * w.R, 256);
     w.off_status = o;        o = align_up(o + sizeof(int32_t) * (size_t)B, 256);
+    w.off_abort = o;         o = align_up(o + sizeof(int32_t), 256);
     w.off_row_stats = o;     o = align_up(o + sizeof(float) * 2 * (size_t)B * w.R, 256);
     w.off_partial = o;       o = align_up(o + sizeof(float) * 2 * (size_t)B * w.R * w.S, 256);
     w.off_resid_partial = o; o = align_up(o + sizeof(float) * (size_t)B * w.S, 256);
@@ -115,7 +120,13 @@ __device__ __forceinline__ float rescale(float m_from, float m_to, float c) {
     return (m_from == -INFINITY) ? 0.f : ex2((m_from - m_to) * c);
 }
 
-inline bs_status cuda_status(cudaError_t e) { return e == cudaSuccess ? BS_OK : BS_ERR_CUDA; }
+extern thread_local int g_last_cuda_error;      // last failing cudaError_t seen by this thread (diagnostics only)
+inline bs_status cuda_status(cudaError_t e) {
+    if (e == cudaSuccess) return BS_OK;
+    g_last_cuda_error = (int)e;
+    cudaGetLastError();                          // clear the sticky launch error
+    return BS_ERR_CUDA;
+}
 
 int sm_count();            // SMs of the current device (cached per device)
 

@@ -3,15 +3,19 @@
 // [.]_+ and Norm(.) as defined in the notation paragraph before Algorithm 6.
 //
 // One uniform per sequence, inverse CDF in vocabulary order.  Two levels, nobody waits:
-//   level 1  a work item is one 32 KB segment of the (target, draft) row pair at position tau_b;
-//            the CTA streams both rows with 128-bit loads, forms r_v = max(0, p_v - q_v) using
-//            the row statistics left in the workspace by bs_softmax_verify, and writes the
-//            segment mass.  An arrival counter per sequence elects the last CTA.
-//   level 2  that CTA scans the segment masses in fp64, picks the segment in which the
-//            cumulative mass crosses u * R, re-reads that one segment (an L2 hit) with each
-//            thread owning a contiguous chunk, scans the chunk masses, and the single thread
-//            whose chunk contains the crossing walks it element by element.
+//   level 1  each sequence's (target, draft) row pair at position tau_b is split into 16 KB
+//            segments, shared out contiguously over a few CTAs; a CTA streams its segments with
+//            128-bit loads, forms r_v = max(0, p_v - q_v) using the row statistics left in the
+//            workspace by bs_softmax_verify, and writes one mass per segment (no CTA-wide
+//            synchronisation between segments).  An arrival counter per sequence elects the last CTA.
+//   level 2  that CTA scans the segment masses in fp64 (one per thread), picks the segment in
+//            which the cumulative mass crosses u * R, re-reads that one segment (an L2 hit) into
+//            registers in the same coalesced layout, scans the per-vector masses across the CTA
+//            in fp64, and the one thread whose vector contains the crossing walks its 4 or 8
+//            elements.  The same r_v values feed the scan and the walk.
 #include "bs_common.cuh"
+
+#include <limits.h>
 
 namespace bs {
 
@@ -33,8 +37,9 @@ struct ResidParams {
     float c;
 };
 
-constexpr int kMaxSeg = 128;          // V <= 2^20 and segments of >= 8192 elements
-constexpr int kRUnroll = 4;           // 128-bit loads in flight per thread and per row
+constexpr int kMaxSeg = BS_MAX_VOCAB / kSegElemsMin;       // 256 = kThreads: one segment mass per thread
+constexpr int kVecTrip = kSegBytes / 16 / kThreads;        // 128-bit vectors per thread and row in one segment
+static_assert(kMaxSeg <= kThreads, "level 2 scans one segment mass per thread");
 
 // Mass of one element.  kt / kd fold the row max and normaliser: p = 2^(x*c + kt).
 struct MassFn {
@@ -48,6 +53,52 @@ struct MassFn {
     }
 };
 
+// Masses of this thread's vectors of segment [e0, e0 + n): vector k covers elements
+// (k * kThreads + tid) * kVec .. + kVec of the segment; elements past n get mass 0.
+template <typename T>
+__device__ __forceinline__ void segment_masses(const T* tp, const T* dp, int e0, int n, const MassFn& f,
+                                               float (&r)[kVecTrip][Elem<T>::kVec]) {
+    constexpr int kVec = Elem<T>::kVec;
+    const int tid = threadIdx.x;
+    const T* ts = tp + e0;
+    const T* ds = f.bonus ? ts : dp + e0;
+    const bool aligned = ((reinterpret_cast<uintptr_t>(ts) | reinterpret_cast<uintptr_t>(ds)) & 15) == 0;
+    if (aligned) {
+        uint4 a[kVecTrip], d[kVecTrip];
+#pragma unroll
+        for (int k = 0; k < kVecTrip; ++k) {
+            const int e = (k * kThreads + tid) * kVec;
+            if (e + kVec <= n) {
+                a[k] = ld_stream(reinterpret_cast<const uint4*>(ts + e));
+                d[k] = f.bonus ? a[k] : ld_stream(reinterpret_cast<const uint4*>(ds + e));
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < kVecTrip; ++k) {
+            const int e = (k * kThreads + tid) * kVec;
+            if (e + kVec <= n) {
+                float ft[kVec], fd[kVec];
+                Elem<T>::unpack(a[k], ft);
+                Elem<T>::unpack(d[k], fd);
+#pragma unroll
+                for (int q = 0; q < kVec; ++q) r[k][q] = f(ft[q], fd[q]);
+            } else {
+#pragma unroll
+                for (int q = 0; q < kVec; ++q)
+                    r[k][q] = (e + q < n) ? f(Elem<T>::load(ts + e + q), f.bonus ? 0.f : Elem<T>::load(ds + e + q)) : 0.f;
+            }
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < kVecTrip; ++k) {
+            const int e = (k * kThreads + tid) * kVec;
+#pragma unroll
+            for (int q = 0; q < kVec; ++q)
+                r[k][q] = (e + q < n) ? f(Elem<T>::load(ts + e + q), f.bonus ? 0.f : Elem<T>::load(ds + e + q)) : 0.f;
+        }
+    }
+}
+
 __device__ __forceinline__ float block_sum(float v, float* s_red) {   // fixed order; result in all threads
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     v = warp_sum(v);
@@ -60,70 +111,71 @@ __device__ __forceinline__ float block_sum(float v, float* s_red) {   // fixed o
     return t;
 }
 
-// Sum of the masses of elements [e0, e0 + n) of the row pair, whole CTA.
+// Sum of this thread's masses of segment [e0, e0 + n).
 template <typename T>
-__device__ __forceinline__ float segment_mass(const T* tp, const T* dp, int e0, int n, const MassFn& f, float* s_red) {
+__device__ __forceinline__ float thread_mass(const T* tp, const T* dp, int e0, int n, const MassFn& f) {
     constexpr int kVec = Elem<T>::kVec;
-    const int tid = threadIdx.x;
-    const T* ts = tp + e0;
-    const T* ds = f.bonus ? ts : dp + e0;
-    const bool aligned = ((reinterpret_cast<uintptr_t>(ts) | reinterpret_cast<uintptr_t>(ds)) & 15) == 0;
+    float r[kVecTrip][kVec];
+    segment_masses<T>(tp, dp, e0, n, f, r);
     float acc = 0.f;
-    int done = 0;
-    if (aligned) {
-        const int nv = n / kVec;
-        const uint4* tv = reinterpret_cast<const uint4*>(ts);
-        const uint4* dv = reinterpret_cast<const uint4*>(ds);
-        for (int base = 0; base < nv; base += kThreads * kRUnroll) {
-            uint4 a[kRUnroll], d[kRUnroll];
 #pragma unroll
-            for (int k = 0; k < kRUnroll; ++k) {
-                int i = base + k * kThreads + tid;
-                if (i < nv) {
-                    a[k] = ld_stream(tv + i);
-                    d[k] = f.bonus ? a[k] : ld_stream(dv + i);
-                }
-            }
+    for (int k = 0; k < kVecTrip; ++k) {
+        float s = 0.f;
 #pragma unroll
-            for (int k = 0; k < kRUnroll; ++k) {
-                int i = base + k * kThreads + tid;
-                if (i < nv) {
-                    float ft[kVec], fd[kVec];
-                    Elem<T>::unpack(a[k], ft);
-                    Elem<T>::unpack(d[k], fd);
-                    float s = 0.f;
-#pragma unroll
-                    for (int q = 0; q < kVec; ++q) s += f(ft[q], fd[q]);
-                    acc += s;
-                }
-            }
-        }
-        done = nv * kVec;
+        for (int q = 0; q < kVec; ++q) s += r[k][q];
+        acc += s;
     }
-    for (int i = done + tid; i < n; i += kThreads)
-        acc += f(Elem<T>::load(ts + i), f.bonus ? 0.f : Elem<T>::load(ds + i));
-    return block_sum(acc, s_red);
+    return acc;
+}
+
+// Inclusive scan over the CTA in thread order, fp64.  Returns this thread's inclusive value; `excl`
+// gets the value of the thread before it (0 for thread 0) and `total` the sum over the CTA.
+__device__ __forceinline__ double block_scan(double v, double* s_w, double& excl, double& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    double incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    double prev = __shfl_up_sync(0xffffffffu, incl, 1);
+    if (lane == 0) prev = 0.0;
+    __syncthreads();
+    if (lane == 31) s_w[warp] = incl;
+    __syncthreads();
+    double woff = 0.0, tot = 0.0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+        if (w == warp) woff = tot;
+        tot += s_w[w];
+    }
+    total = tot;
+    excl = woff + prev;
+    return woff + incl;
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kThreads) residual_kernel(const ResidParams p) {
+__global__ void __launch_bounds__(kThreads, 2) residual_kernel(const ResidParams p, const int nsplit) {
+    constexpr int kVec = Elem<T>::kVec;
     __shared__ float s_red[kWarps];
-    __shared__ double s_scan[kWarps];
-    __shared__ double s_cum[kMaxSeg];
+    __shared__ double s_w[kWarps];
+    __shared__ float s_mass[kMaxSeg];
+    __shared__ float s_wm[kMaxSeg][kWarps];
     __shared__ int s_flag;
     __shared__ int s_pick;
+    __shared__ int s_lastseg;
     __shared__ int s_token;
     __shared__ int s_lastpos;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int total = p.B * p.nseg;
-
-    for (int item = blockIdx.x; item < total; item += gridDim.x) {
-        const int b = item / p.nseg, sg = item - b * p.nseg;
+    // CTA (b, part) owns a contiguous range of the segments of sequence b
+    {
+        const int b = blockIdx.x / nsplit, part = blockIdx.x - b * nsplit;
+        const int sg0 = (int)((long long)p.nseg * part / nsplit);
+        const int sg1 = (int)((long long)p.nseg * (part + 1) / nsplit);
         int g = p.gamma[b];
         if (g < 0 || g > p.Gmax) g = 0;
-        int tau = p.accept_len[b];
-        tau = max(0, min(tau, g));
+        const int tau = max(0, min(p.accept_len[b], g));
         MassFn f;
         f.c = p.c;
         f.bonus = tau >= g;
@@ -137,100 +189,99 @@ __global__ void __launch_bounds__(kThreads) residual_kernel(const ResidParams p)
             f.kd = -(ds.x * p.c + log2f(ds.y));
             dp = row_ptr(static_cast<const T*>(p.draft), b, p.Gmax, tau, p.V);
         }
-        const int e0 = sg * p.seg;
-        const int n = min(p.seg, p.V - e0);
-        const float mass = segment_mass<T>(tp, dp, e0, n, f, s_red);
+        // ---- level 1: segment masses, no CTA-wide synchronisation between segments ----
+        for (int sg = sg0; sg < sg1; ++sg) {
+            const int e0 = sg * p.seg;
+            const float w = warp_sum(thread_mass<T>(tp, dp, e0, min(p.seg, p.V - e0), f));
+            if (lane == 0) s_wm[sg - sg0][warp] = w;
+        }
+        __syncthreads();
+        if (tid < sg1 - sg0) {
+            float t = 0.f;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) t += s_wm[tid][w];         // fixed order
+            p.resid_partial[(size_t)b * p.S + sg0 + tid] = t;
+        }
+        __threadfence();
+        __syncthreads();
         if (tid == 0) {
-            p.resid_partial[(size_t)b * p.S + sg] = mass;
-            __threadfence();
-            unsigned old = atomicAdd(p.ticket + b, 1u);
-            s_flag = (old == (unsigned)(p.nseg - 1));
+            const unsigned old = atomicAdd(p.ticket + b, 1u);
+            s_flag = (old == (unsigned)(nsplit - 1));
         }
         __syncthreads();
         if (s_flag) {
-            // ---- last CTA of sequence b: inverse CDF ----
+            // ---- level 2, last CTA of sequence b: inverse CDF over the vocabulary ----
             __threadfence();
             int bits = 0;
-            const float* pp = p.resid_partial + (size_t)b * p.S;
-            if (tid == 0) {
-                double cum = 0.0;
-                for (int q = 0; q < p.nseg; ++q) { cum += (double)__ldcg(pp + q); s_cum[q] = cum; }
-            }
-            __syncthreads();
-            double Rtot = s_cum[p.nseg - 1];
+            s_mass[tid] = tid < p.nseg ? __ldcg(p.resid_partial + (size_t)b * p.S + tid) : 0.f;
+            double excl, Rtot;
+            double incl = block_scan((double)s_mass[tid], s_w, excl, Rtot);
             if (!(Rtot > 0.0) || !isfinite(Rtot)) {
                 // [P - Q]_+ has no mass (P == Q up to rounding) or the row is not finite:
                 // fall back to the target distribution of the same row
                 bits |= f.bonus ? BS_DEV_NONFINITE : BS_DEV_RESIDUAL_FALLBACK;
                 f.bonus = true;
-                __syncthreads();
                 for (int q = 0; q < p.nseg; ++q) {
                     const int qe0 = q * p.seg;
-                    float m2 = segment_mass<T>(tp, tp, qe0, min(p.seg, p.V - qe0), f, s_red);
-                    if (tid == 0) s_cum[q] = (q ? s_cum[q - 1] : 0.0) + (double)m2;
+                    const float m2 = block_sum(thread_mass<T>(tp, tp, qe0, min(p.seg, p.V - qe0), f), s_red);
+                    if (tid == q) s_mass[q] = m2;
                 }
                 __syncthreads();
-                Rtot = s_cum[p.nseg - 1];
+                incl = block_scan((double)s_mass[tid], s_w, excl, Rtot);
                 if (!(Rtot > 0.0) || !isfinite(Rtot)) bits |= BS_DEV_NONFINITE;
             }
             const double target = (double)p.u_resample[b] * Rtot;
-            if (tid == 0) {
-                int pick = -1, lastpos = 0;
-                for (int q = 0; q < p.nseg; ++q) {
-                    if ((q ? s_cum[q] - s_cum[q - 1] : s_cum[0]) > 0.0) lastpos = q;
-                    if (pick < 0 && s_cum[q] > target) pick = q;
-                }
-                s_pick = pick < 0 ? lastpos : pick;
-                s_token = -1;
-                s_lastpos = -1;
+            if (tid == 0) { s_pick = -1; s_lastseg = 0; s_token = INT_MAX; s_lastpos = -1; }
+            __syncthreads();
+            if (tid < p.nseg) {
+                if (s_mass[tid] > 0.f) atomicMax(&s_lastseg, tid);
+                if (incl > target && !(excl > target)) s_pick = tid;       // at most one thread
             }
             __syncthreads();
-            const int ps = s_pick;
-            const double t_in = target - (ps ? s_cum[ps - 1] : 0.0);
-            // chunk of this thread inside the picked segment, in vocabulary order
+            const int ps = s_pick >= 0 ? s_pick : s_lastseg;
+            // cumulative mass before the picked segment
+            const double before = __shfl_sync(0xffffffffu, excl, ps & 31);     // valid in warp ps / 32
+            if ((tid >> 5) == (ps >> 5) && (tid & 31) == 0) s_w[0] = before;
+            __syncthreads();
+            const double t_in = target - s_w[0];
+            __syncthreads();
+            // ---- inside the picked segment ----
             const int pe0 = ps * p.seg;
             const int pn = min(p.seg, p.V - pe0);
-            const int chunk = div_up(pn, kThreads);
-            const int c0 = min(pn, tid * chunk), c1 = min(pn, c0 + chunk);
-            const T* ts2 = tp + pe0;
-            const T* ds2 = dp + pe0;
-            float csum = 0.f;
-            int lastpos = -1;
-            for (int i = c0; i < c1; ++i) {
-                float r = f(Elem<T>::load(ts2 + i), f.bonus ? 0.f : Elem<T>::load(ds2 + i));
-                csum += r;
-                if (r > 0.f) lastpos = i;
-            }
-            // inclusive scan of the chunk masses over the CTA, fp64
-            double incl = (double)csum;
+            float r[kVecTrip][kVec];
+            segment_masses<T>(tp, dp, pe0, pn, f, r);
+            double base = 0.0;
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                double t = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += t;
-            }
-            if (lane == 31) s_scan[warp] = incl;
-            __syncthreads();
-            double woff = 0.0;
-            for (int w = 0; w < warp; ++w) woff += s_scan[w];
-            incl += woff;
-            const double excl = incl - (double)csum;
-            if (lastpos >= 0) atomicMax(&s_lastpos, lastpos);
-            if (incl > t_in && !(excl > t_in)) {
-                // the crossing lies in this chunk (exactly one thread satisfies both)
-                double run = excl;
-                int tok = -1;
-                for (int i = c0; i < c1; ++i) {
-                    float r = f(Elem<T>::load(ts2 + i), f.bonus ? 0.f : Elem<T>::load(ds2 + i));
-                    run += (double)r;
-                    if (run > t_in && r > 0.f) { tok = i; break; }
+            for (int k = 0; k < kVecTrip; ++k) {
+                float vs = 0.f;
+                int lastq = -1;
+#pragma unroll
+                for (int q = 0; q < kVec; ++q) { vs += r[k][q]; if (r[k][q] > 0.f) lastq = q; }
+                double vex, vtot;
+                const double vin = base + block_scan((double)vs, s_w, vex, vtot);
+                vex += base;
+                const int e = (k * kThreads + tid) * kVec;
+                if (lastq >= 0) atomicMax(&s_lastpos, e + lastq);
+                if (vin > t_in && !(vex > t_in)) {
+                    double run = vex;
+                    int tok = -1;
+#pragma unroll
+                    for (int q = 0; q < kVec; ++q) {
+                        run += (double)r[k][q];
+                        if (tok < 0 && run > t_in && r[k][q] > 0.f) tok = q;
+                    }
+                    if (tok < 0) tok = lastq;
+                    if (tok >= 0) atomicMin(&s_token, pe0 + e + tok);
                 }
-                if (tok < 0) tok = lastpos;          // rounding between the two passes
-                if (tok >= 0) s_token = pe0 + tok;
+                base += vtot;
             }
             __syncthreads();
             if (tid == 0) {
                 int tok = s_token;
-                if (tok < 0) tok = (s_lastpos >= 0) ? pe0 + s_lastpos : 0;   // u * R beyond the recomputed mass
+                if (tok == INT_MAX) {                    // u * R at or beyond the recomputed mass of the segment
+                    if (s_lastpos >= 0) tok = pe0 + s_lastpos;
+                    else { tok = 0; bits |= BS_DEV_NONFINITE; }
+                }
                 int32_t* ot = p.out_tokens + (size_t)b * (p.Gmax + 1);
                 for (int j = 0; j <= p.Gmax; ++j)
                     ot[j] = j < tau ? p.tokens[(size_t)b * p.Gmax + j] : (j == tau ? tok : -1);
@@ -239,7 +290,6 @@ __global__ void __launch_bounds__(kThreads) residual_kernel(const ResidParams p)
                 p.ticket[b] = 0u;
             }
         }
-        __syncthreads();
     }
 }
 
@@ -257,23 +307,13 @@ __global__ void greedy_emit_kernel(const ResidParams p) {
     p.out_len[b] = tau + 1;
 }
 
-static int g_rocc[2][64];
-
 template <typename T>
-static bs_status launch_residual(const ResidParams& p, int variant, cudaStream_t st) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (dev < 0 || dev >= 64) dev = 0;
-    if (!g_rocc[variant][dev]) {
-        int occ = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, residual_kernel<T>, kThreads, 0) != cudaSuccess || occ < 1)
-            occ = 1;
-        g_rocc[variant][dev] = occ;
-    }
-    long long grid = (long long)sm_count() * g_rocc[variant][dev];
-    const long long items = (long long)p.B * p.nseg;
-    if (grid > items) grid = items;
-    residual_kernel<T><<<(unsigned)grid, kThreads, 0, st>>>(p);
+static bs_status launch_residual(const ResidParams& p, cudaStream_t st) {
+    // about two CTAs per SM in total, each owning a contiguous share of one sequence's segments
+    int nsplit = div_up(2 * sm_count(), p.B);
+    if (nsplit > p.nseg) nsplit = p.nseg;
+    if (nsplit < 1) nsplit = 1;
+    residual_kernel<T><<<(unsigned)(p.B * nsplit), kThreads, 0, st>>>(p, nsplit);
     return cuda_status(cudaGetLastError());
 }
 
@@ -287,7 +327,7 @@ extern "C" bs_status bs_residual_sample(const void* target_logits, const void* d
                                         int32_t* out_tokens, int32_t* out_len,
                                         void* workspace, size_t workspace_bytes, void* stream) {
     if (B < 1 || Gmax < 0 || V < 1) return BS_ERR_INVALID_ARG;
-    if (B > BS_MAX_BATCH || Gmax > BS_MAX_GAMMA || V > (1 << 20)) return BS_ERR_UNSUPPORTED;
+    if (B > BS_MAX_BATCH || Gmax > BS_MAX_GAMMA || V > BS_MAX_VOCAB) return BS_ERR_UNSUPPORTED;
     if (dtype != BS_F32 && dtype != BS_BF16) return BS_ERR_INVALID_ARG;
     if (!(temperature >= 0.f) || !isfinite(temperature)) return BS_ERR_INVALID_ARG;
     const bool greedy = temperature == 0.f;
@@ -314,5 +354,5 @@ extern "C" bs_status bs_residual_sample(const void* target_logits, const void* d
         greedy_emit_kernel<<<div_up(B, 128), 128, 0, st>>>(p);
         return cuda_status(cudaGetLastError());
     }
-    return dtype == BS_F32 ? launch_residual<float>(p, 0, st) : launch_residual<__nv_bfloat16>(p, 1, st);
+    return dtype == BS_F32 ? launch_residual<float>(p, st) : launch_residual<__nv_bfloat16>(p, st);
 }

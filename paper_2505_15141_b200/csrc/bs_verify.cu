@@ -1,100 +1,19 @@
-// bs_softmax_verify: single-pass row softmax statistics over every valid target / draft row,
-// then (by the last CTA to finish a sequence) token-probability gather, accept test and
-// first-rejection scan.  Algorithm 6 of the paper, second line and for-loop; softmax with
-// temperature as in Section 2.
+// bs_softmax_verify: entry point, plus the generic row-statistics kernel used when rows do not
+// start on 16-byte boundaries (V * sizeof(element) not a multiple of 16).  Rows that do are
+// handled by the pipelined kernel in bs_verify_stream.cu.  Algorithm 6 of the paper, second
+// line and for-loop; softmax with temperature as in Section 2.
 //
-// Work decomposition: a work item is one 32 KB segment of one valid row.  Sequences have
-// ragged speculation lengths, so every CTA builds the prefix sum of items per sequence in
-// shared memory and the persistent grid strides over the flat item list; rows beyond
-// gamma_b cost nothing.  Each item is streamed with 128-bit read-once loads (8 in flight
-// per thread), reduced to (max, sum exp) with ONE exp per logit, and written as a partial.
-// An arrival counter per sequence (atomic ticket, nobody waits) elects the CTA that merges
-// the partials and runs the accept scan.
-#include "bs_common.cuh"
-
-#include <limits.h>
+// Generic kernel: a work item is one segment of one valid row.  Every CTA builds the prefix sum
+// of items per sequence in shared memory and the persistent grid strides over the flat item
+// list.  Each item is read with a scalar head up to the next 16-byte boundary, a 128-bit body
+// and a scalar tail, reduced to (max, sum exp) with one exp per logit, and written as a
+// partial.  An arrival counter per sequence elects the CTA that merges the partials and runs
+// the accept scan.
+#include "bs_verify_common.cuh"
 
 namespace bs {
 
-struct VerifyParams {
-    const void* target;
-    const void* draft;
-    const int32_t* tokens;
-    const int32_t* gamma;
-    const float* u_accept;
-    int32_t* accept_len;
-    float* p_tok;
-    float* q_tok;
-    uint32_t* ticket;
-    int32_t* status;
-    float2* row_stats;
-    float2* partial;
-    int B, Gmax, V, R, S;
-    int nseg, seg;     // segments per row and elements per segment for this dtype
-    float c;           // log2(e) / temperature
-};
-
-constexpr int kUnroll = 8;      // 128-bit loads in flight per thread
-
-struct ArgMax {
-    float m;
-    int idx;
-};
-__device__ __forceinline__ ArgMax better(ArgMax a, ArgMax b) {
-    return (b.m > a.m || (b.m == a.m && b.idx < a.idx)) ? b : a;
-}
-
-// Running (m, s) of one thread: s = sum over seen x of exp2((x - m) * c).
-struct Online {
-    float m, s;
-    __device__ __forceinline__ void raise_to(float mc, float c) {
-        if (mc > m) { s *= rescale(m, mc, c); m = mc; }
-    }
-};
-
-template <typename T>
-__device__ __forceinline__ float chunk_max(const uint4 (&v)[kUnroll]);
-
-template <>
-__device__ __forceinline__ float chunk_max<float>(const uint4 (&v)[kUnroll]) {
-    float m = -INFINITY;
-#pragma unroll
-    for (int k = 0; k < kUnroll; ++k) {
-        m = fmaxf(m, fmaxf(fmaxf(__uint_as_float(v[k].x), __uint_as_float(v[k].y)),
-                           fmaxf(__uint_as_float(v[k].z), __uint_as_float(v[k].w))));
-    }
-    return m;
-}
-
-template <>
-__device__ __forceinline__ float chunk_max<__nv_bfloat16>(const uint4 (&v)[kUnroll]) {
-    // packed max on the raw bf16 pairs: two elements per instruction
-    __nv_bfloat162 m2 = *reinterpret_cast<const __nv_bfloat162*>(&v[0].x);
-#pragma unroll
-    for (int k = 0; k < kUnroll; ++k) {
-        m2 = __hmax2(m2, *reinterpret_cast<const __nv_bfloat162*>(&v[k].x));
-        m2 = __hmax2(m2, *reinterpret_cast<const __nv_bfloat162*>(&v[k].y));
-        m2 = __hmax2(m2, *reinterpret_cast<const __nv_bfloat162*>(&v[k].z));
-        m2 = __hmax2(m2, *reinterpret_cast<const __nv_bfloat162*>(&v[k].w));
-    }
-    uint32_t w = *reinterpret_cast<uint32_t*>(&m2);
-    return fmaxf(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
-}
-
-template <typename T> __device__ __forceinline__ uint4 neg_inf_vec();
-template <> __device__ __forceinline__ uint4 neg_inf_vec<float>() {
-    return make_uint4(0xff800000u, 0xff800000u, 0xff800000u, 0xff800000u);
-}
-template <> __device__ __forceinline__ uint4 neg_inf_vec<__nv_bfloat16>() {
-    return make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
-}
-
-// Items of sequence b: rows * segments.  An out-of-range gamma is processed as gamma = 0.
-template <bool GREEDY>
-__device__ __forceinline__ int seq_rows(int g, int Gmax) {
-    if (g < 0 || g > Gmax) g = 0;
-    return GREEDY ? g + 1 : 2 * g + 1;
-}
+constexpr int kUnroll = 4;      // 128-bit loads in flight per thread: one segment per trip
 
 template <typename T, bool GREEDY>
 __global__ void __launch_bounds__(kThreads) verify_kernel(const VerifyParams p) {
@@ -108,7 +27,7 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const VerifyParams p) 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int kVec = Elem<T>::kVec;
 
-    // ---- prefix sum of work items over the batch (every CTA, redundantly; B <= 4096) ----
+    // ---- prefix sum of work items over the batch (every CTA, redundantly) ----
     {
         const int per = div_up(p.B, kThreads);
         const int b0 = tid * per;
@@ -150,11 +69,9 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const VerifyParams p) 
         const int b = lo;
         const int local = item - s_prefix[b];
         const int lr = local / p.nseg, sg = local - lr * p.nseg;
-        int g = p.gamma[b];
-        if (g < 0 || g > p.Gmax) g = 0;
-        // local rows 0..g are target rows; g+1..2g are draft rows 0..g-1
+        const int g = clamp_gamma(p.gamma[b], p.Gmax);
         const bool is_target = lr <= g;
-        const int r = is_target ? lr : p.Gmax + 1 + (lr - g - 1);
+        const int r = row_slot(lr, g, p.Gmax);
         const T* rowp = is_target
             ? row_ptr(static_cast<const T*>(p.target), b, p.Gmax + 1, lr, p.V)
             : row_ptr(static_cast<const T*>(p.draft), b, p.Gmax, lr - g - 1, p.V);
@@ -184,35 +101,8 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const VerifyParams p) 
                 int i = base + k * kThreads + tid;
                 v[k] = (i < nv) ? ld_stream(vp + i) : neg_inf_vec<T>();
             }
-            if (GREEDY) {
-#pragma unroll
-                for (int k = 0; k < kUnroll; ++k) {
-                    float f[kVec];
-                    Elem<T>::unpack(v[k], f);
-                    int ei = e0 + head + (base + k * kThreads + tid) * kVec;
-#pragma unroll
-                    for (int q = 0; q < kVec; ++q)
-                        if (f[q] > am.m) { am.m = f[q]; am.idx = ei + q; }
-                }
-            } else {
-                float mc = chunk_max<T>(v);
-                on.raise_to(mc, p.c);
-                if (on.m > -INFINITY) {
-                    const float nm = -on.m * p.c;
-                    float acc0 = 0.f, acc1 = 0.f;
-#pragma unroll
-                    for (int k = 0; k < kUnroll; ++k) {
-                        float f[kVec];
-                        Elem<T>::unpack(v[k], f);
-#pragma unroll
-                        for (int q = 0; q < kVec; q += 2) {
-                            acc0 += ex2(fmaf(f[q], p.c, nm));
-                            acc1 += ex2(fmaf(f[q + 1], p.c, nm));
-                        }
-                    }
-                    on.s += acc0 + acc1;
-                }
-            }
+            if (GREEDY) argmax_add<T, kUnroll>(am, v, e0 + head + (base + tid) * kVec, kThreads * kVec);
+            else online_add<T, kUnroll>(on, v, p.c);
         }
         if (tid < n - tail0) {
             float x = Elem<T>::load(sp + tail0 + tid);
@@ -222,34 +112,22 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const VerifyParams p) 
 
         // ---- block reduction (fixed order, deterministic) ----
         if (GREEDY) {
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                ArgMax t{__shfl_xor_sync(0xffffffffu, am.m, o), __shfl_xor_sync(0xffffffffu, am.idx, o)};
-                am = better(am, t);
-            }
+            am = warp_best(am);
             if (lane == 0) { s_m[warp] = am.m; s_i[warp] = am.idx; }
         } else {
-            float wm = warp_max(on.m);
-            float ws = warp_sum(on.s * rescale(on.m, wm, p.c));
-            if (lane == 0) { s_m[warp] = wm; s_s[warp] = ws; }
+            const float2 w = warp_merge(on, p.c);
+            if (lane == 0) { s_m[warp] = w.x; s_s[warp] = w.y; }
         }
         __syncthreads();
         if (warp == 0) {
             float2 out;
             if (GREEDY) {
                 ArgMax a{lane < kWarps ? s_m[lane] : -INFINITY, lane < kWarps ? s_i[lane] : INT_MAX};
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
-                    ArgMax t{__shfl_xor_sync(0xffffffffu, a.m, o), __shfl_xor_sync(0xffffffffu, a.idx, o)};
-                    a = better(a, t);
-                }
+                a = warp_best(a);
                 out = make_float2(a.m, __int_as_float(a.idx));
             } else {
-                float m = lane < kWarps ? s_m[lane] : -INFINITY;
-                float s = lane < kWarps ? s_s[lane] : 0.f;
-                float M = warp_max(m);
-                float Z = warp_sum(s * rescale(m, M, p.c));
-                out = make_float2(M, Z);
+                Online o{lane < kWarps ? s_m[lane] : -INFINITY, lane < kWarps ? s_s[lane] : 0.f};
+                out = warp_merge(o, p.c);
             }
             if (lane == 0) {
                 const int items_b = seq_rows<GREEDY>(g, p.Gmax) * p.nseg;
@@ -267,33 +145,8 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const VerifyParams p) 
             __threadfence();
             const int rows_b = seq_rows<GREEDY>(g, p.Gmax);
             for (int l2 = warp; l2 < rows_b; l2 += kWarps) {
-                const int r2 = (l2 <= g) ? l2 : p.Gmax + 1 + (l2 - g - 1);
-                const float2* pp = p.partial + ((size_t)b * p.R + r2) * p.S;
-                float2 st;
-                if (GREEDY) {
-                    ArgMax a{-INFINITY, INT_MAX};
-                    for (int q = lane; q < p.nseg; q += 32) {
-                        float2 v = __ldcg(pp + q);
-                        a = better(a, ArgMax{v.x, __float_as_int(v.y)});
-                    }
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) {
-                        ArgMax t{__shfl_xor_sync(0xffffffffu, a.m, o), __shfl_xor_sync(0xffffffffu, a.idx, o)};
-                        a = better(a, t);
-                    }
-                    if (a.idx == INT_MAX) a.idx = 0;          // row of -inf / NaN only
-                    st = make_float2(a.m, __int_as_float(a.idx));
-                } else {
-                    Online o2{-INFINITY, 0.f};
-                    for (int q = lane; q < p.nseg; q += 32) {
-                        float2 v = __ldcg(pp + q);
-                        o2.raise_to(v.x, p.c);
-                        o2.s += v.y * rescale(v.x, o2.m, p.c);
-                    }
-                    float M = warp_max(o2.m);
-                    float Z = warp_sum(o2.s * rescale(o2.m, M, p.c));
-                    st = make_float2(M, Z);
-                }
+                const int r2 = row_slot(l2, g, p.Gmax);
+                const float2 st = merge_row_partials<GREEDY>(p.partial + ((size_t)b * p.R + r2) * p.S, p.nseg, p.c);
                 if (lane == 0) {
                     s_stats[r2] = st;
                     p.row_stats[(size_t)b * p.R + r2] = st;
@@ -301,61 +154,15 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const VerifyParams p) 
             }
             __syncthreads();
             if (warp == 0) {
-                const int j = lane;
-                const bool valid = j < g;
-                int st_bits = (p.gamma[b] < 0 || p.gamma[b] > p.Gmax) ? BS_DEV_BAD_GAMMA : 0;
-                bool acc = false;
-                float pj = 0.f, qj = 0.f;
-                if (valid) {
-                    const int x = p.tokens[(size_t)b * p.Gmax + j];
-                    const bool bad = x < 0 || x >= p.V;
-                    if (bad) st_bits |= BS_DEV_BAD_TOKEN;
-                    const float2 ts = s_stats[j];
-                    if (GREEDY) {
-                        acc = !bad && x == __float_as_int(ts.y);
-                    } else {
-                        const float2 ds = s_stats[p.Gmax + 1 + j];
-                        if (!(ts.y > 0.f) || !(ds.y > 0.f) || !isfinite(ts.y) || !isfinite(ds.y) ||
-                            !isfinite(ts.x) || !isfinite(ds.x))
-                            st_bits |= BS_DEV_NONFINITE;
-                        if (!bad) {
-                            const float tl = Elem<T>::load(row_ptr(static_cast<const T*>(p.target), b, p.Gmax + 1, j, p.V) + x);
-                            const float dl = Elem<T>::load(row_ptr(static_cast<const T*>(p.draft), b, p.Gmax, j, p.V) + x);
-                            // log2 of the two probabilities; the ratio is formed in the log domain
-                            const float lp = (tl - ts.x) * p.c - log2f(ts.y);
-                            const float lq = (dl - ds.x) * p.c - log2f(ds.y);
-                            pj = exp2f(lp);
-                            qj = exp2f(lq);
-                            const float u = p.u_accept[(size_t)b * p.Gmax + j];
-                            // r <= min{1, P/Q}; Q(x) = 0 counts as an infinite ratio
-                            acc = (lq == -INFINITY) ? true : (u <= fminf(1.f, exp2f(lp - lq)));
-                        }
-                    }
-                }
-                if (!GREEDY && !valid && j == g) {   // the bonus row's normaliser is used by the resampler
-                    const float2 ts = s_stats[g];
-                    if (!(ts.y > 0.f) || !isfinite(ts.y) || !isfinite(ts.x)) st_bits |= BS_DEV_NONFINITE;
-                }
-                const unsigned accmask = __ballot_sync(0xffffffffu, valid && acc);
-                const unsigned validmask = (g >= 32) ? 0xffffffffu : ((1u << g) - 1u);
-                const unsigned rej = ~accmask & validmask;          // first zero among the valid bits
-                const int tau = rej ? (__ffs(rej) - 1) : g;
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) st_bits |= __shfl_xor_sync(0xffffffffu, st_bits, o);
-                if (j < p.Gmax) {
-                    if (p.p_tok) p.p_tok[(size_t)b * p.Gmax + j] = valid ? pj : 0.f;
-                    if (p.q_tok) p.q_tok[(size_t)b * p.Gmax + j] = valid ? qj : 0.f;
-                }
-                if (lane == 0) {
-                    p.accept_len[b] = tau;
-                    p.status[b] = st_bits;
-                    p.ticket[b] = 0u;                // leave the counter clear for the next call
-                }
+                accept_scan_warp<T, GREEDY>(p, b, [&](int rr) { return s_stats[rr]; });
+                if (lane == 0) p.ticket[b] = 0u;         // leave the counter clear for the next call
             }
         }
         __syncthreads();
     }
 }
+
+thread_local int g_last_cuda_error = 0;
 
 static int g_occ[4][64];     // resident CTAs per SM per kernel variant, per device (0 = not queried)
 static int g_sms[64];
@@ -406,8 +213,12 @@ extern "C" const char* bs_status_string(bs_status s) {
     return "unknown";
 }
 
+extern "C" const char* bs_last_cuda_error(void) {
+    return g_last_cuda_error ? cudaGetErrorString(static_cast<cudaError_t>(g_last_cuda_error)) : "no error";
+}
+
 static bool sizes_ok(int B, int Gmax, int V) {
-    return B >= 1 && B <= BS_MAX_BATCH && Gmax >= 0 && Gmax <= BS_MAX_GAMMA && V >= 1 && V <= (1 << 20);
+    return B >= 1 && B <= BS_MAX_BATCH && Gmax >= 0 && Gmax <= BS_MAX_GAMMA && V >= 1 && V <= BS_MAX_VOCAB;
 }
 
 extern "C" size_t bs_workspace_bytes(int B, int Gmax, int V) {
@@ -427,10 +238,15 @@ extern "C" bs_status bs_get_device_status(const void* workspace, size_t workspac
     const Workspace w = workspace_layout(B, Gmax, V);
     if (workspace_bytes < w.total) return BS_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t aborted = 0;
     cudaError_t e = cudaMemcpyAsync(host_status, static_cast<const char*>(workspace) + w.off_status,
                                     sizeof(int32_t) * B, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(&aborted, static_cast<const char*>(workspace) + w.off_abort, sizeof(int32_t),
+                            cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return BS_ERR_CUDA;
+    if (aborted) return BS_ERR_TIMEOUT;
     for (int b = 0; b < B; ++b)
         if (host_status[b]) return BS_ERR_DEVICE_DATA;
     return BS_OK;
@@ -459,7 +275,9 @@ extern "C" bs_status bs_softmax_verify(const void* target_logits, const void* dr
     p.target = target_logits; p.draft = draft_logits; p.tokens = draft_tokens; p.gamma = gamma;
     p.u_accept = u_accept; p.accept_len = accept_len; p.p_tok = p_tok; p.q_tok = q_tok;
     p.ticket = reinterpret_cast<uint32_t*>(ws + w.off_ticket_verify);
+    p.ticket_row = reinterpret_cast<uint32_t*>(ws + w.off_ticket_row);
     p.status = reinterpret_cast<int32_t*>(ws + w.off_status);
+    p.abort_flag = reinterpret_cast<int32_t*>(ws + w.off_abort);
     p.row_stats = reinterpret_cast<float2*>(ws + w.off_row_stats);
     p.partial = reinterpret_cast<float2*>(ws + w.off_partial);
     p.B = B; p.Gmax = Gmax; p.V = V; p.R = w.R; p.S = w.S;
@@ -467,6 +285,15 @@ extern "C" bs_status bs_softmax_verify(const void* target_logits, const void* dr
     p.nseg = div_up(V, p.seg);
     p.c = greedy ? 1.f : kLog2e / temperature;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // rows start on 16-byte boundaries: bulk-copy pipeline; otherwise the generic kernel
+    const bool aligned = ((size_t)V * es) % 16 == 0 && (reinterpret_cast<uintptr_t>(target_logits) & 15) == 0 &&
+                         (reinterpret_cast<uintptr_t>(draft_logits) & 15) == 0;
+    if (aligned) {
+        if (dtype == BS_F32)
+            return greedy ? launch_verify_stream<float, true>(p, st) : launch_verify_stream<float, false>(p, st);
+        return greedy ? launch_verify_stream<__nv_bfloat16, true>(p, st)
+                      : launch_verify_stream<__nv_bfloat16, false>(p, st);
+    }
     if (dtype == BS_F32)
         return greedy ? launch_verify<float, true>(p, 0, st) : launch_verify<float, false>(p, 1, st);
     return greedy ? launch_verify<__nv_bfloat16, true>(p, 2, st) : launch_verify<__nv_bfloat16, false>(p, 3, st);

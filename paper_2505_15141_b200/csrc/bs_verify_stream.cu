@@ -1,0 +1,344 @@
+// Pipelined row-statistics kernel of bs_softmax_verify for rows that start on 16-byte
+// boundaries (V * sizeof(element) a multiple of 16): softmax with temperature (Section 2 of the
+// paper) and the accept loop of Algorithm 6.
+//
+// The flat list of work items (one item = one 16 KB segment of one valid row; ragged gamma_b
+// handled through a prefix sum over the batch) is cut into gridDim.x contiguous ranges, one
+// per CTA, so every CTA streams the same number of bytes (+-1 segment) and mostly whole rows.
+//
+//   warp 8 (one lane)  producer: walks its range, and for each segment arms a "full" mbarrier
+//                      with the byte count and issues one bulk async copy (TMA, no multicast)
+//                      global -> shared into a ring of kStages 16 KB slots.
+//   warps 0..7         consumers: wait for the slot, read it with conflict-free 128-bit shared
+//                      loads, update a per-thread online softmax state (chunk max first, then
+//                      ONE exp per logit), release the slot through an "empty" mbarrier.
+//
+// The per-thread state lives across all segments of a row piece; it is reduced only when the
+// row (or the CTA's range) ends.  Row partials are merged by whichever warp completes the row
+// (atomic ticket per row), and the accept scan of a sequence is run by whichever warp completes
+// its last row (atomic ticket per sequence).  Nobody waits on another CTA.  All waits on
+// mbarriers are bounded; a wait that gives up sets the abort word and the thread leaves.
+#include "bs_verify_common.cuh"
+
+namespace bs {
+
+constexpr int kConsumerWarps = 8;
+constexpr int kStreamThreads = (kConsumerWarps + 1) * 32;
+constexpr int kVecPerStage = kSegBytes / 16;                     // 1024
+constexpr int kVecPerThread = kVecPerStage / (kConsumerWarps * 32);   // 4
+constexpr int kMaxStages = 6;
+constexpr int kRedSlots = 8;                                     // >= kMaxStages + 1 piece ends in flight
+constexpr long long kWaitCycles = 2000000000LL;                  // about one second
+
+struct StageMeta {
+    int nvec;        // 16-byte vectors in this stage
+    int b;           // sequence
+    int lr;          // local row index within the sequence
+    int sg;          // segment index within the row
+    int flags;       // bit 0: first stage of a row piece, bit 1: last stage of a row piece
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: false if the phase did not complete within about a second.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (clock64() - t0 > kWaitCycles) return false;
+    }
+    return true;
+}
+// The same for a whole warp: every lane polls, the outcome is made uniform by a vote.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity));
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+
+template <typename T, bool GREEDY>
+__global__ void __launch_bounds__(kStreamThreads) verify_stream_kernel(const VerifyParams p, const int nstages) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    // layout: [nstages * 16 KB ring][prefix (B+1) ints]
+    unsigned char* ring = smem;
+    int* s_prefix = reinterpret_cast<int*>(smem + (size_t)nstages * kSegBytes);
+    __shared__ __align__(8) unsigned long long s_full[kMaxStages];
+    __shared__ __align__(8) unsigned long long s_empty[kMaxStages];
+    // one reduction barrier per s_red slot: a warp may run several row pieces ahead of another,
+    // so arrivals of different pieces must never meet on one barrier
+    __shared__ __align__(8) unsigned long long s_redbar[kRedSlots];
+    __shared__ StageMeta s_meta[kMaxStages];
+    __shared__ float2 s_red[kRedSlots][kConsumerWarps];
+    __shared__ int s_scan[kConsumerWarps + 1];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int kVec = Elem<T>::kVec;
+
+    if (tid == 0) {
+        for (int s = 0; s < nstages; ++s) {
+            mbar_init(smem_u32(&s_full[s]), 1);
+            mbar_init(smem_u32(&s_empty[s]), kConsumerWarps);
+        }
+        for (int s = 0; s < kRedSlots; ++s) mbar_init(smem_u32(&s_redbar[s]), kConsumerWarps);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+
+    // ---- prefix sum of work items over the batch (all threads, redundantly per CTA) ----
+    {
+        const int per = div_up(p.B, kStreamThreads);
+        const int b0 = tid * per;
+        int local = 0;
+        for (int k = 0; k < per; ++k) {
+            const int b = b0 + k;
+            if (b < p.B) local += seq_rows<GREEDY>(p.gamma[b], p.Gmax) * p.nseg;
+        }
+        int incl = local;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (lane == 31) s_scan[warp] = incl;
+        __syncthreads();
+        int woff = 0;
+        for (int w = 0; w < warp; ++w) woff += s_scan[w];
+        int run = woff + incl - local;
+        for (int k = 0; k < per; ++k) {
+            const int b = b0 + k;
+            if (b < p.B) {
+                s_prefix[b] = run;
+                run += seq_rows<GREEDY>(p.gamma[b], p.Gmax) * p.nseg;
+            }
+        }
+        if (tid == kStreamThreads - 1) s_prefix[p.B] = run;
+        __syncthreads();                                      // also publishes the mbarrier inits
+    }
+    const int total = s_prefix[p.B];
+    const int lo = (int)((long long)total * blockIdx.x / gridDim.x);
+    const int hi = (int)((long long)total * (blockIdx.x + 1) / gridDim.x);
+    const int count = hi - lo;
+    if (count <= 0) return;
+
+    // first item of the range -> (sequence, local row, segment)
+    int b, lr, sg, g, rows_b;
+    {
+        int l = 0, h = p.B;                                   // largest b with prefix[b] <= lo
+        while (h - l > 1) {
+            const int mid = (l + h) >> 1;
+            if (s_prefix[mid] <= lo) l = mid; else h = mid;
+        }
+        b = l;
+        const int local = lo - s_prefix[b];
+        lr = local / p.nseg;
+        sg = local - lr * p.nseg;
+        g = clamp_gamma(p.gamma[b], p.Gmax);
+        rows_b = GREEDY ? g + 1 : 2 * g + 1;
+    }
+
+    if (warp == kConsumerWarps) {
+        // =============================== producer ===============================
+        if (lane != 0) return;
+        for (int k = 0; k < count; ++k) {
+            const int slot = k % nstages;
+            const uint32_t ph = (uint32_t)(k / nstages) & 1u;
+            if (!mbar_wait(smem_u32(&s_empty[slot]), ph ^ 1u)) { atomicExch(p.abort_flag, 1); return; }
+            const bool is_target = lr <= g;
+            const T* rowp = is_target
+                ? row_ptr(static_cast<const T*>(p.target), b, p.Gmax + 1, lr, p.V)
+                : row_ptr(static_cast<const T*>(p.draft), b, p.Gmax, lr - g - 1, p.V);
+            const int e0 = sg * p.seg;
+            const int n = min(p.seg, p.V - e0);
+            const uint32_t bytes = (uint32_t)n * (uint32_t)sizeof(T);
+            const bool row_end = sg == p.nseg - 1;
+            StageMeta m;
+            m.nvec = n / kVec; m.b = b; m.lr = lr; m.sg = sg;
+            m.flags = ((sg == 0 || k == 0) ? 1 : 0) | ((row_end || k == count - 1) ? 2 : 0);
+            s_meta[slot] = m;
+            const uint32_t bar = smem_u32(&s_full[slot]);
+            mbar_arrive_expect_tx(bar, bytes);                // releases the meta write to the waiters
+            bulk_load(smem_u32(ring + (size_t)slot * kSegBytes), rowp + e0, bytes, bar);
+            // advance to the next item
+            if (++sg == p.nseg) {
+                sg = 0;
+                if (++lr == rows_b) {
+                    lr = 0;
+                    ++b;
+                    if (b < p.B) {
+                        g = clamp_gamma(p.gamma[b], p.Gmax);
+                        rows_b = GREEDY ? g + 1 : 2 * g + 1;
+                    }
+                }
+            }
+        }
+        return;
+    }
+
+    // ================================= consumers =================================
+    Online on{-INFINITY, 0.f};
+    ArgMax am{-INFINITY, INT_MAX};
+    int piece_first_sg = 0;
+    int pc = 0;                                               // row pieces finished by this CTA
+    for (int k = 0; k < count; ++k) {
+        const int slot = k % nstages;
+        const uint32_t ph = (uint32_t)(k / nstages) & 1u;
+        if (!mbar_wait_warp(smem_u32(&s_full[slot]), ph)) { atomicExch(p.abort_flag, 1); return; }
+        const StageMeta m = s_meta[slot];
+        if (m.flags & 1) piece_first_sg = m.sg;
+        const uint32_t base = smem_u32(ring + (size_t)slot * kSegBytes);
+        uint4 v[kVecPerThread];
+#pragma unroll
+        for (int q = 0; q < kVecPerThread; ++q) {
+            const int i = q * (kConsumerWarps * 32) + tid;
+            v[q] = (i < m.nvec) ? lds128(base + (uint32_t)i * 16u) : neg_inf_vec<T>();
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&s_empty[slot]));  // the slot's data is in registers now
+        if (GREEDY) argmax_add<T, kVecPerThread>(am, v, m.sg * p.seg + tid * kVec, kConsumerWarps * 32 * kVec);
+        else online_add<T, kVecPerThread>(on, v, p.c);
+
+        if (m.flags & 2) {
+            // ---- end of a row piece: reduce over the 8 consumer warps ----
+            float2 wr;
+            if (GREEDY) { am = warp_best(am); wr = make_float2(am.m, __int_as_float(am.idx)); }
+            else wr = warp_merge(on, p.c);
+            const int rs = pc % kRedSlots;
+            if (lane == 0) {
+                s_red[rs][warp] = wr;
+                mbar_arrive(smem_u32(&s_redbar[rs]));         // release: the write above is visible to warp 0
+            }
+            if (warp == 0) {
+                if (!mbar_wait_warp(smem_u32(&s_redbar[rs]), (uint32_t)(pc / kRedSlots) & 1u)) {
+                    atomicExch(p.abort_flag, 1);
+                    return;
+                }
+                float2 out;
+                if (GREEDY) {
+                    ArgMax a{-INFINITY, INT_MAX};
+                    if (lane < kConsumerWarps) { const float2 t = s_red[rs][lane]; a = ArgMax{t.x, __float_as_int(t.y)}; }
+                    a = warp_best(a);
+                    out = make_float2(a.m, __int_as_float(a.idx));
+                } else {
+                    Online o{-INFINITY, 0.f};
+                    if (lane < kConsumerWarps) { const float2 t = s_red[rs][lane]; o.m = t.x; o.s = t.y; }
+                    out = warp_merge(o, p.c);
+                }
+                // ---- publish; the warp that completes a row / a sequence does the follow-up ----
+                const int gb = clamp_gamma(p.gamma[m.b], p.Gmax);
+                const int r = row_slot(m.lr, gb, p.Gmax);
+                const int piece_len = m.sg - piece_first_sg + 1;
+                bool row_done;
+                if (piece_len == p.nseg) {                    // the whole row was ours
+                    if (GREEDY && __float_as_int(out.y) == INT_MAX) out.y = __int_as_float(0);
+                    if (lane == 0) p.row_stats[(size_t)m.b * p.R + r] = out;
+                    row_done = true;
+                } else {
+                    float2* pp = p.partial + ((size_t)m.b * p.R + r) * p.S;
+                    // slot of the piece's first segment carries the result, the rest are neutral
+                    for (int q = piece_first_sg + lane; q <= m.sg; q += 32)
+                        pp[q] = (q == piece_first_sg) ? out
+                                                      : make_float2(-INFINITY, GREEDY ? __int_as_float(INT_MAX) : 0.f);
+                    __threadfence();
+                    __syncwarp();
+                    unsigned old = 0;
+                    if (lane == 0) old = atomicAdd(p.ticket_row + (size_t)m.b * p.R + r, (unsigned)piece_len);
+                    old = __shfl_sync(0xffffffffu, old, 0);
+                    row_done = (old + (unsigned)piece_len == (unsigned)p.nseg);
+                    if (row_done) {
+                        __threadfence();
+                        const float2 st = merge_row_partials<GREEDY>(pp, p.nseg, p.c);
+                        if (lane == 0) {
+                            p.row_stats[(size_t)m.b * p.R + r] = st;
+                            p.ticket_row[(size_t)m.b * p.R + r] = 0u;
+                        }
+                    }
+                }
+                if (row_done) {
+                    __threadfence();
+                    __syncwarp();
+                    const int rows_mb = GREEDY ? gb + 1 : 2 * gb + 1;
+                    unsigned old = 0;
+                    if (lane == 0) old = atomicAdd(p.ticket + m.b, 1u);
+                    old = __shfl_sync(0xffffffffu, old, 0);
+                    if (old + 1u == (unsigned)rows_mb) {
+                        __threadfence();
+                        const float2* rsb = p.row_stats + (size_t)m.b * p.R;
+                        accept_scan_warp<T, GREEDY>(p, m.b, [rsb](int rr) { return __ldcg(rsb + rr); });
+                        if (lane == 0) p.ticket[m.b] = 0u;
+                    }
+                }
+            }
+            on = Online{-INFINITY, 0.f};
+            am = ArgMax{-INFINITY, INT_MAX};
+            ++pc;
+        }
+    }
+}
+
+static int g_stream_smem[64];          // opt-in shared memory limit per device (0 = not queried)
+static bool g_attr_set[4][64];
+
+template <typename T, bool GREEDY>
+bs_status launch_verify_stream(const VerifyParams& p, cudaStream_t st) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64) dev = 0;
+    if (!g_stream_smem[dev]) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
+            return cuda_status(cudaGetLastError());
+        g_stream_smem[dev] = v;
+    }
+    // two CTAs per SM: each may use half of the SM's shared memory minus the static part
+    const size_t prefix_bytes = align_up(sizeof(int) * (size_t)(p.B + 1), 128);
+    const size_t budget = (size_t)(g_stream_smem[dev] + 1024) / 2 - 3072;        // per CTA
+    int nst = (int)((budget - prefix_bytes) / kSegBytes);
+    if (nst > kMaxStages) nst = kMaxStages;
+    if (nst < 2) return BS_ERR_UNSUPPORTED;
+    const size_t smem = (size_t)nst * kSegBytes + prefix_bytes;
+    const int variant = (Elem<T>::kDtype == BS_F32 ? 0 : 2) + (GREEDY ? 1 : 0);
+    if (!g_attr_set[variant][dev]) {
+        // the opt-in limit covers static + dynamic shared memory: leave room for the static part
+        if (cudaFuncSetAttribute(verify_stream_kernel<T, GREEDY>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 g_stream_smem[dev] - 4096) != cudaSuccess)
+            return cuda_status(cudaGetLastError());
+        g_attr_set[variant][dev] = true;
+    }
+    const long long upper = (long long)p.B * (GREEDY ? p.Gmax + 1 : p.R) * p.nseg;
+    long long grid = 2LL * sm_count();
+    if (grid > upper) grid = upper;
+    if (grid < 1) grid = 1;
+    verify_stream_kernel<T, GREEDY><<<(unsigned)grid, kStreamThreads, smem, st>>>(p, nst);
+    return cuda_status(cudaGetLastError());
+}
+
+template bs_status launch_verify_stream<float, false>(const VerifyParams&, cudaStream_t);
+template bs_status launch_verify_stream<float, true>(const VerifyParams&, cudaStream_t);
+template bs_status launch_verify_stream<__nv_bfloat16, false>(const VerifyParams&, cudaStream_t);
+template bs_status launch_verify_stream<__nv_bfloat16, true>(const VerifyParams&, cudaStream_t);
+
+}  // namespace bs
