@@ -12,11 +12,15 @@ namespace bs {
 
 constexpr int kThreads = 256;              // threads per CTA of the streaming kernels
 constexpr int kWarps = kThreads / 32;
-constexpr int kSegBytes = 16384;           // bytes of one row segment = one work item = one pipeline stage
+constexpr int kSegBytes = 32768;           // row-statistics kernels: bytes of one row segment = one work item
+                                           // = one pipeline stage
 constexpr int kSegElemsMin = kSegBytes / 4;  // segment length of the widest dtype (fp32)
+constexpr int kResSegBytes = 16384;        // resampling kernel: bytes of one row segment
+constexpr int kResSegElemsMin = kResSegBytes / 4;
 constexpr float kLog2e = 1.4426950408889634f;
 
 __host__ __device__ inline int seg_elems(int dtype) { return dtype == BS_F32 ? kSegBytes / 4 : kSegBytes / 2; }
+__host__ __device__ inline int res_seg_elems(int dtype) { return dtype == BS_F32 ? kResSegBytes / 4 : kResSegBytes / 2; }
 __host__ __device__ inline int div_up(int a, int b) { return (a + b - 1) / b; }
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -28,18 +32,19 @@ __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a -
 //   abort         [1] i32     set when a bounded pipeline wait gave up (reported as BS_ERR_TIMEOUT)
 //   row_stats     [B, R, 2] f32, R = 2*Gmax+1: (raw max logit, Z) per row; greedy: (max, arg-max bits)
 //                 rows 0..Gmax are target rows, rows Gmax+1..2*Gmax are draft rows
-//   partial       [B, R, S, 2] f32, S = ceil(V / 4096): per-segment (max, Z) / (max, arg-max)
-//   resid_partial [B, S] f32  per-segment residual mass
+//   partial       [B, R, S, 2] f32, S = ceil(V / 8192): per-segment (max, Z) / (max, arg-max)
+//   resid_partial [B, Sr] f32, Sr = ceil(V / 4096): per-segment residual mass
 struct Workspace {
     size_t off_ticket_verify, off_ticket_resid, off_ticket_row, off_status, off_abort, off_row_stats, off_partial,
         off_resid_partial, total;
-    int R, S;
+    int R, S, Sr;
 };
 
 __host__ __device__ inline Workspace workspace_layout(int B, int Gmax, int V) {
     Workspace w;
     w.R = 2 * Gmax + 1;
     w.S = div_up(V, kSegElemsMin);
+    w.Sr = div_up(V, kResSegElemsMin);
     size_t o = 0;
     w.off_ticket_verify = o; o = align_up(o + sizeof(uint32_t) * (size_t)B, 256);
     w.off_ticket_resid = o;  o = align_up(o + sizeof(uint32_t) * (size_t)B, 256);
@@ -48,7 +53,7 @@ __host__ __device__ inline Workspace workspace_layout(int B, int Gmax, int V) {
     w.off_abort = o;         o = align_up(o + sizeof(int32_t), 256);
     w.off_row_stats = o;     o = align_up(o + sizeof(float) * 2 * (size_t)B * w.R, 256);
     w.off_partial = o;       o = align_up(o + sizeof(float) * 2 * (size_t)B * w.R * w.S, 256);
-    w.off_resid_partial = o; o = align_up(o + sizeof(float) * (size_t)B * w.S, 256);
+    w.off_resid_partial = o; o = align_up(o + sizeof(float) * (size_t)B * w.Sr, 256);
     w.total = o;
     return w;
 }

@@ -37,8 +37,8 @@ struct ResidParams {
     float c;
 };
 
-constexpr int kMaxSeg = BS_MAX_VOCAB / kSegElemsMin;       // 256 = kThreads: one segment mass per thread
-constexpr int kVecTrip = kSegBytes / 16 / kThreads;        // 128-bit vectors per thread and row in one segment
+constexpr int kMaxSeg = BS_MAX_VOCAB / kResSegElemsMin;       // 256 = kThreads: one segment mass per thread
+constexpr int kVecTrip = kResSegBytes / 16 / kThreads;        // 128-bit vectors per thread and row in one segment
 static_assert(kMaxSeg <= kThreads, "level 2 scans one segment mass per thread");
 
 // Mass of one element.  kt / kd fold the row max and normaliser: p = 2^(x*c + kt).
@@ -345,8 +345,8 @@ extern "C" bs_status bs_residual_sample(const void* target_logits, const void* d
     p.status = reinterpret_cast<int32_t*>(ws + w.off_status);
     p.row_stats = reinterpret_cast<const float2*>(ws + w.off_row_stats);
     p.resid_partial = reinterpret_cast<float*>(ws + w.off_resid_partial);
-    p.B = B; p.Gmax = Gmax; p.V = V; p.R = w.R; p.S = w.S;
-    p.seg = seg_elems(dtype);
+    p.B = B; p.Gmax = Gmax; p.V = V; p.R = w.R; p.S = w.Sr;
+    p.seg = res_seg_elems(dtype);
     p.nseg = div_up(V, p.seg);
     p.c = greedy ? 1.f : kLog2e / temperature;
     cudaStream_t st = static_cast<cudaStream_t>(stream);

@@ -2,14 +2,14 @@
 // boundaries (V * sizeof(element) a multiple of 16): softmax with temperature (Section 2 of the
 // paper) and the accept loop of Algorithm 6.
 //
-// The flat list of work items (one item = one 16 KB segment of one valid row; ragged gamma_b
+// The flat list of work items (one item = one 32 KB segment of one valid row; ragged gamma_b
 // handled through a prefix sum over the batch) is cut into gridDim.x contiguous ranges, one
 // per CTA, so every CTA streams the same number of bytes (+-1 segment) and mostly whole rows.
 //
-//   warp 8 (one lane)  producer: walks its range, and for each segment arms a "full" mbarrier
+//   warp 16 (one lane) producer: walks its range, and for each segment arms a "full" mbarrier
 //                      with the byte count and issues one bulk async copy (TMA, no multicast)
-//                      global -> shared into a ring of kStages 16 KB slots.
-//   warps 0..7         consumers: wait for the slot, read it with conflict-free 128-bit shared
+//                      global -> shared into a ring of 32 KB slots.
+//   warps 0..15        consumers: wait for the slot, read it with conflict-free 128-bit shared
 //                      loads, update a per-thread online softmax state (chunk max first, then
 //                      ONE exp per logit), release the slot through an "empty" mbarrier.
 //
@@ -22,21 +22,23 @@
 
 namespace bs {
 
-constexpr int kConsumerWarps = 8;
-constexpr int kStreamThreads = (kConsumerWarps + 1) * 32;
-constexpr int kVecPerStage = kSegBytes / 16;                     // 1024
-constexpr int kVecPerThread = kVecPerStage / (kConsumerWarps * 32);   // 4
-constexpr int kMaxStages = 6;
-constexpr int kRedSlots = 8;                                     // >= kMaxStages + 1 piece ends in flight
+constexpr int kConsumerWarps = 16;
+constexpr int kConsumers = kConsumerWarps * 32;
+constexpr int kStreamThreads = kConsumers + 32;
+constexpr int kVecPerStage = kSegBytes / 16;                     // 2048
+constexpr int kVecPerThread = kVecPerStage / kConsumers;         // 4
+constexpr int kMaxStages = 3;
+constexpr int kRedSlots = 8;                                     // > kMaxStages + 1 row-piece ends in flight
 constexpr long long kWaitCycles = 2000000000LL;                  // about one second
+static_assert(kVecPerThread * kConsumers == kVecPerStage, "stage must divide evenly over the consumers");
 
+// Per-stage record written by the producer: w0 = nvec | flags << 16, w1 = b | lr << 13 | sg << 19
+// (b < 2^13, lr < 2^6, sg < 2^8).  flags bit 0: first stage of a row piece, bit 1: last stage.
 struct StageMeta {
-    int nvec;        // 16-byte vectors in this stage
-    int b;           // sequence
-    int lr;          // local row index within the sequence
-    int sg;          // segment index within the row
-    int flags;       // bit 0: first stage of a row piece, bit 1: last stage of a row piece
+    int w0, w1;
 };
+static_assert(BS_MAX_BATCH <= (1 << 13) && 2 * BS_MAX_GAMMA + 1 < (1 << 6) &&
+              BS_MAX_VOCAB / (kSegBytes / 4) <= (1 << 8), "StageMeta packing");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -84,7 +86,7 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
 template <typename T, bool GREEDY>
 __global__ void __launch_bounds__(kStreamThreads) verify_stream_kernel(const VerifyParams p, const int nstages) {
     extern __shared__ __align__(128) unsigned char smem[];
-    // layout: [nstages * 16 KB ring][prefix (B+1) ints]
+    // layout: [nstages * 32 KB ring][prefix (B+1) ints]
     unsigned char* ring = smem;
     int* s_prefix = reinterpret_cast<int*>(smem + (size_t)nstages * kSegBytes);
     __shared__ __align__(8) unsigned long long s_full[kMaxStages];
@@ -92,7 +94,7 @@ __global__ void __launch_bounds__(kStreamThreads) verify_stream_kernel(const Ver
     // one reduction barrier per s_red slot: a warp may run several row pieces ahead of another,
     // so arrivals of different pieces must never meet on one barrier
     __shared__ __align__(8) unsigned long long s_redbar[kRedSlots];
-    __shared__ StageMeta s_meta[kMaxStages];
+    __shared__ __align__(8) StageMeta s_meta[kMaxStages];
     __shared__ float2 s_red[kRedSlots][kConsumerWarps];
     __shared__ int s_scan[kConsumerWarps + 1];
 
@@ -144,28 +146,27 @@ __global__ void __launch_bounds__(kStreamThreads) verify_stream_kernel(const Ver
     const int count = hi - lo;
     if (count <= 0) return;
 
-    // first item of the range -> (sequence, local row, segment)
-    int b, lr, sg, g, rows_b;
-    {
-        int l = 0, h = p.B;                                   // largest b with prefix[b] <= lo
-        while (h - l > 1) {
-            const int mid = (l + h) >> 1;
-            if (s_prefix[mid] <= lo) l = mid; else h = mid;
-        }
-        b = l;
-        const int local = lo - s_prefix[b];
-        lr = local / p.nseg;
-        sg = local - lr * p.nseg;
-        g = clamp_gamma(p.gamma[b], p.Gmax);
-        rows_b = GREEDY ? g + 1 : 2 * g + 1;
-    }
-
     if (warp == kConsumerWarps) {
         // =============================== producer ===============================
         if (lane != 0) return;
+        // first item of the range -> (sequence, local row, segment)
+        int b, lr, sg, g, rows_b;
+        {
+            int l = 0, h = p.B;                               // largest b with prefix[b] <= lo
+            while (h - l > 1) {
+                const int mid = (l + h) >> 1;
+                if (s_prefix[mid] <= lo) l = mid; else h = mid;
+            }
+            b = l;
+            const int local = lo - s_prefix[b];
+            lr = local / p.nseg;
+            sg = local - lr * p.nseg;
+            g = clamp_gamma(p.gamma[b], p.Gmax);
+            rows_b = GREEDY ? g + 1 : 2 * g + 1;
+        }
+        int slot = 0;
+        uint32_t ph = 0;
         for (int k = 0; k < count; ++k) {
-            const int slot = k % nstages;
-            const uint32_t ph = (uint32_t)(k / nstages) & 1u;
             if (!mbar_wait(smem_u32(&s_empty[slot]), ph ^ 1u)) { atomicExch(p.abort_flag, 1); return; }
             const bool is_target = lr <= g;
             const T* rowp = is_target
@@ -174,10 +175,10 @@ __global__ void __launch_bounds__(kStreamThreads) verify_stream_kernel(const Ver
             const int e0 = sg * p.seg;
             const int n = min(p.seg, p.V - e0);
             const uint32_t bytes = (uint32_t)n * (uint32_t)sizeof(T);
-            const bool row_end = sg == p.nseg - 1;
+            const int flags = ((sg == 0 || k == 0) ? 1 : 0) | ((sg == p.nseg - 1 || k == count - 1) ? 2 : 0);
             StageMeta m;
-            m.nvec = n / kVec; m.b = b; m.lr = lr; m.sg = sg;
-            m.flags = ((sg == 0 || k == 0) ? 1 : 0) | ((row_end || k == count - 1) ? 2 : 0);
+            m.w0 = (n / kVec) | (flags << 16);
+            m.w1 = b | (lr << 13) | (sg << 19);
             s_meta[slot] = m;
             const uint32_t bar = smem_u32(&s_full[slot]);
             mbar_arrive_expect_tx(bar, bytes);                // releases the meta write to the waiters
@@ -194,6 +195,7 @@ __global__ void __launch_bounds__(kStreamThreads) verify_stream_kernel(const Ver
                     }
                 }
             }
+            if (++slot == nstages) { slot = 0; ph ^= 1u; }
         }
         return;
     }
@@ -203,26 +205,32 @@ __global__ void __launch_bounds__(kStreamThreads) verify_stream_kernel(const Ver
     ArgMax am{-INFINITY, INT_MAX};
     int piece_first_sg = 0;
     int pc = 0;                                               // row pieces finished by this CTA
+    int slot = 0;
+    uint32_t ph = 0;
     for (int k = 0; k < count; ++k) {
-        const int slot = k % nstages;
-        const uint32_t ph = (uint32_t)(k / nstages) & 1u;
         if (!mbar_wait_warp(smem_u32(&s_full[slot]), ph)) { atomicExch(p.abort_flag, 1); return; }
         const StageMeta m = s_meta[slot];
-        if (m.flags & 1) piece_first_sg = m.sg;
-        const uint32_t base = smem_u32(ring + (size_t)slot * kSegBytes);
+        const int nvec = m.w0 & 0xffff, flags = m.w0 >> 16;
+        const int m_sg = (m.w1 >> 19) & 0xff;
+        if (flags & 1) piece_first_sg = m_sg;
+        const uint32_t base = smem_u32(ring + (size_t)slot * kSegBytes) + (uint32_t)tid * 16u;
         uint4 v[kVecPerThread];
+        if (nvec == kVecPerStage) {
 #pragma unroll
-        for (int q = 0; q < kVecPerThread; ++q) {
-            const int i = q * (kConsumerWarps * 32) + tid;
-            v[q] = (i < m.nvec) ? lds128(base + (uint32_t)i * 16u) : neg_inf_vec<T>();
+            for (int q = 0; q < kVecPerThread; ++q) v[q] = lds128(base + (uint32_t)(q * kConsumers) * 16u);
+        } else {
+#pragma unroll
+            for (int q = 0; q < kVecPerThread; ++q)
+                v[q] = (q * kConsumers + tid < nvec) ? lds128(base + (uint32_t)(q * kConsumers) * 16u) : neg_inf_vec<T>();
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&s_empty[slot]));  // the slot's data is in registers now
-        if (GREEDY) argmax_add<T, kVecPerThread>(am, v, m.sg * p.seg + tid * kVec, kConsumerWarps * 32 * kVec);
+        if (GREEDY) argmax_add<T, kVecPerThread>(am, v, m_sg * p.seg + tid * kVec, kConsumers * kVec);
         else online_add<T, kVecPerThread>(on, v, p.c);
+        if (++slot == nstages) { slot = 0; ph ^= 1u; }
 
-        if (m.flags & 2) {
-            // ---- end of a row piece: reduce over the 8 consumer warps ----
+        if (flags & 2) {
+            // ---- end of a row piece: reduce over the consumer warps ----
             float2 wr;
             if (GREEDY) { am = warp_best(am); wr = make_float2(am.m, __int_as_float(am.idx)); }
             else wr = warp_merge(on, p.c);
@@ -248,32 +256,33 @@ __global__ void __launch_bounds__(kStreamThreads) verify_stream_kernel(const Ver
                     out = warp_merge(o, p.c);
                 }
                 // ---- publish; the warp that completes a row / a sequence does the follow-up ----
-                const int gb = clamp_gamma(p.gamma[m.b], p.Gmax);
-                const int r = row_slot(m.lr, gb, p.Gmax);
-                const int piece_len = m.sg - piece_first_sg + 1;
+                const int m_b = m.w1 & 0x1fff, m_lr = (m.w1 >> 13) & 0x3f;
+                const int gb = clamp_gamma(p.gamma[m_b], p.Gmax);
+                const int r = row_slot(m_lr, gb, p.Gmax);
+                const int piece_len = m_sg - piece_first_sg + 1;
                 bool row_done;
                 if (piece_len == p.nseg) {                    // the whole row was ours
                     if (GREEDY && __float_as_int(out.y) == INT_MAX) out.y = __int_as_float(0);
-                    if (lane == 0) p.row_stats[(size_t)m.b * p.R + r] = out;
+                    if (lane == 0) p.row_stats[(size_t)m_b * p.R + r] = out;
                     row_done = true;
                 } else {
-                    float2* pp = p.partial + ((size_t)m.b * p.R + r) * p.S;
+                    float2* pp = p.partial + ((size_t)m_b * p.R + r) * p.S;
                     // slot of the piece's first segment carries the result, the rest are neutral
-                    for (int q = piece_first_sg + lane; q <= m.sg; q += 32)
+                    for (int q = piece_first_sg + lane; q <= m_sg; q += 32)
                         pp[q] = (q == piece_first_sg) ? out
                                                       : make_float2(-INFINITY, GREEDY ? __int_as_float(INT_MAX) : 0.f);
                     __threadfence();
                     __syncwarp();
                     unsigned old = 0;
-                    if (lane == 0) old = atomicAdd(p.ticket_row + (size_t)m.b * p.R + r, (unsigned)piece_len);
+                    if (lane == 0) old = atomicAdd(p.ticket_row + (size_t)m_b * p.R + r, (unsigned)piece_len);
                     old = __shfl_sync(0xffffffffu, old, 0);
                     row_done = (old + (unsigned)piece_len == (unsigned)p.nseg);
                     if (row_done) {
                         __threadfence();
                         const float2 st = merge_row_partials<GREEDY>(pp, p.nseg, p.c);
                         if (lane == 0) {
-                            p.row_stats[(size_t)m.b * p.R + r] = st;
-                            p.ticket_row[(size_t)m.b * p.R + r] = 0u;
+                            p.row_stats[(size_t)m_b * p.R + r] = st;
+                            p.ticket_row[(size_t)m_b * p.R + r] = 0u;
                         }
                     }
                 }
@@ -282,13 +291,13 @@ __global__ void __launch_bounds__(kStreamThreads) verify_stream_kernel(const Ver
                     __syncwarp();
                     const int rows_mb = GREEDY ? gb + 1 : 2 * gb + 1;
                     unsigned old = 0;
-                    if (lane == 0) old = atomicAdd(p.ticket + m.b, 1u);
+                    if (lane == 0) old = atomicAdd(p.ticket + m_b, 1u);
                     old = __shfl_sync(0xffffffffu, old, 0);
                     if (old + 1u == (unsigned)rows_mb) {
                         __threadfence();
-                        const float2* rsb = p.row_stats + (size_t)m.b * p.R;
-                        accept_scan_warp<T, GREEDY>(p, m.b, [rsb](int rr) { return __ldcg(rsb + rr); });
-                        if (lane == 0) p.ticket[m.b] = 0u;
+                        const float2* rsb = p.row_stats + (size_t)m_b * p.R;
+                        accept_scan_warp<T, GREEDY>(p, m_b, [rsb](int rr) { return __ldcg(rsb + rr); });
+                        if (lane == 0) p.ticket[m_b] = 0u;
                     }
                 }
             }
