@@ -88,6 +88,30 @@ def oracle_sample(w, rnd_inputs, seconds: float, max_seqs=None):
     return done, time.perf_counter() - t0
 
 
+def rank_round_index(rank: int, i: int) -> int:
+    """Round number that seeds input set i of a rank: every rank verifies its own batches."""
+    return 1 + i + 1000 * rank
+
+
+def reduce_over_ranks(ms: float, nbytes: float, device):
+    """Whole-job timing: the slowest rank's time (MAX) and the bytes of all ranks (SUM).
+    Sequences are independent, so this is the only exchange between ranks."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms), float(nbytes)
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    b = torch.tensor([nbytes], dtype=torch.float64, device=device)
+    dist.all_reduce(b, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(b.item())
+
+
+def job_rounds_per_s(world: int, steps: int, ms: float) -> float:
+    """Each rank completes `steps` rounds of its own batch in the common time `ms`."""
+    return world * steps / (ms * 1e-3)
+
+
 def default_arms(w, step: int) -> np.ndarray:
     """Arms used to shape the pre-generated inputs (the device bandit picks its own gamma)."""
     return ((np.arange(w.B) + step) % w.K).astype(np.int32)
@@ -205,10 +229,9 @@ def run_cuda(args, w):
     # ---- ring of input sets, > 2 x L2 in total ----
     set_bytes = es * V * B * (2 * G + 1)
     ring = max(2, -(-2 * L2_BYTES // set_bytes) + 1)
-    seed_shift = 1000 * rank                                   # every rank verifies its own batch
     sets = []
     for i in range(ring):
-        rnd = wl.make_round(w, 1 + i + seed_shift, default_arms(w, i), device=dev)
+        rnd = wl.make_round(w, rank_round_index(rank, i), default_arms(w, i), device=dev)
         sets.append(dict(
             target=rnd.target, draft=rnd.draft, tokens=rnd.tokens.contiguous(),
             u_accept=torch.as_tensor(rnd.uniforms.u_accept, device=dev),
@@ -288,16 +311,8 @@ def run_cuda(args, w):
     assert dn.sum() == B * args.steps, "every sequence must have played every timed round"
     rows_timed = int((dn * (2 * arm_gamma + 1)[None, :]).sum())
     bytes_timed = rows_timed * V * es
-    if world > 1:
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-        bt = torch.tensor([bytes_timed], dtype=torch.float64, device=dev)
-        dist.all_reduce(bt, op=dist.ReduceOp.SUM)
-        bytes_all = float(bt.item())
-    else:
-        bytes_all = float(bytes_timed)
-    value = world * args.steps / (ms * 1e-3)
+    ms, bytes_all = reduce_over_ranks(ms, bytes_timed, dev)
+    value = job_rounds_per_s(world, args.steps, ms)
 
     # ---- kernel pass: CUDA events around bs_softmax_verify on its launching stream ----
     ksteps = min(args.steps, 50)
