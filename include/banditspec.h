@@ -131,6 +131,34 @@ bs_status bs_residual_sample(const void* target_logits, const void* draft_logits
                              int32_t* out_tokens, int32_t* out_len,
                              void* workspace, size_t workspace_bytes, void* stream);
 
+/* bs_softmax_verify without a caller-supplied workspace.  (No counterpart in the paper: this
+ * exists for integration, not for the method.)
+ *
+ * For callers that cannot allocate device memory where the call is made: a decoding loop that
+ * runs out of a pool sized at start-up, a plugin that only ever receives its input and output
+ * buffers, or a latency-critical path where cudaMalloc is off limits because it synchronises the
+ * device.  The scratch is a fixed array of BS_NOALLOC_SCRATCH_BYTES built into the library; every
+ * GPU that loads the library holds that much memory until the process exits.
+ *
+ *  - Same arguments, outputs and arithmetic as bs_softmax_verify, minus the workspace.  The
+ *    call allocates and frees nothing.
+ *  - Limit: bs_workspace_bytes(B, Gmax, V) must not exceed BS_NOALLOC_SCRATCH_BYTES, otherwise
+ *    BS_ERR_WORKSPACE is returned and nothing is launched (e.g. B=64, Gmax=8, V=128256 needs
+ *    about 160 KB; B=256, Gmax=8, V=152064 about 740 KB).
+ *  - The first call on each device looks up the device address of the array (with that device
+ *    current).  Make that first call outside any stream capture.
+ *  - All calls on a GPU share the one array.  It keeps what the previous call left; the counters
+ *    and status words the kernel reads before writing are cleared on the stream at the start of
+ *    every call.  Calls that overlap on the same GPU (different streams, different threads) race
+ *    on it and give wrong results: serialise them.
+ *  - The row statistics stay inside the library, so bs_residual_sample cannot follow this call;
+ *    it serves callers that need accept_len and the token probabilities only. */
+#define BS_NOALLOC_SCRATCH_BYTES (1 << 20)
+bs_status bs_softmax_verify_noalloc(const void* target_logits, const void* draft_logits, bs_dtype dtype,
+                                    const int32_t* draft_tokens, const int32_t* gamma, const float* u_accept,
+                                    float temperature, int B, int Gmax, int V,
+                                    int32_t* accept_len, float* p_tok, float* q_tok, void* stream);
+
 /* ---- arm selection (Algorithm 3, select and history lines) ---------------------------- */
 
 /* Bytes of the opaque device state of B independent bandits with K arms. 0 if out of limits. */

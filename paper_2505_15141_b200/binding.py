@@ -40,6 +40,7 @@ SIGNATURES = {
     "bs_get_device_status": (_i, [_vp, _sz, _i, _i, _i, _vp, _vp]),
     "bs_softmax_verify": (_i, [_vp, _vp, _i, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bs_residual_sample": (_i, [_vp, _vp, _i, _vp, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _sz, _vp]),
+    "bs_softmax_verify_noalloc": (_i, [_vp, _vp, _i, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _vp]),
     "bs_bandit_state_bytes": (_sz, [_i, _i, _i]),
     "bs_bandit_init": (_i, [_vp, _sz, _i, _i, _i, _vp, _d, _vp]),
     "bs_bandit_select": (_i, [_vp, _sz, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -132,6 +133,22 @@ def bs_residual_sample(target_logits, draft_logits, draft_tokens, gamma, accept_
                                    _ptr(draft_tokens), _ptr(gamma), _ptr(accept_len), _ptr(u_resample),
                                    float(temperature), B, G1 - 1, V, _ptr(out_tokens), _ptr(out_len),
                                    _ptr(workspace), workspace.numel(), _stream(stream)), "bs_residual_sample")
+
+
+BS_NOALLOC_SCRATCH_BYTES = 1 << 20
+
+
+def bs_softmax_verify_noalloc(target_logits, draft_logits, draft_tokens, gamma, u_accept, temperature: float,
+                              accept_len, p_tok, q_tok, stream=None) -> None:
+    """bs_softmax_verify on the scratch array built into the library: for callers that cannot
+    allocate device memory (fixed memory pools, buffer-only plugins, no-cudaMalloc paths).
+    Sizes whose workspace exceeds BS_NOALLOC_SCRATCH_BYTES raise BS_ERR_WORKSPACE; calls that
+    overlap on one GPU race on the shared array."""
+    B, G1, V = target_logits.shape
+    _check(_lib.bs_softmax_verify_noalloc(_ptr(target_logits), _ptr(draft_logits), _dtype_code(target_logits),
+                                          _ptr(draft_tokens), _ptr(gamma), _ptr(u_accept), float(temperature),
+                                          B, G1 - 1, V, _ptr(accept_len), _ptr(p_tok), _ptr(q_tok),
+                                          _stream(stream)), "bs_softmax_verify_noalloc")
 
 
 @dataclass
