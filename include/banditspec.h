@@ -159,6 +159,42 @@ bs_status bs_softmax_verify_noalloc(const void* target_logits, const void* draft
                                     float temperature, int B, int Gmax, int V,
                                     int32_t* accept_len, float* p_tok, float* q_tok, void* stream);
 
+/* ---- fused LM head (Algorithm 6, second line: the models are evaluated on all drafted positions
+ *      in parallel; the last step of that evaluation is logits = H W) -------------------------- */
+
+/* Bytes of device scratch bs_lmhead_verify needs.  The first bs_workspace_bytes(B, Gmax, V) bytes
+ * are an ordinary verification workspace (clear it with bs_workspace_init before the first call),
+ * so the same pointer and size are then handed to bs_residual_sample and bs_get_device_status.
+ * Returns 0 for arguments outside the limits. */
+size_t bs_lmhead_workspace_bytes(int B, int Gmax, int V);
+
+/* Computes the target and draft logits from the final hidden states on the tensor cores
+ * (bf16 x bf16 products, fp32 accumulation), the softmax statistics of every row while the
+ * logits are still on chip, and then the accept test and first-rejection scan of
+ * bs_softmax_verify.  The fp32 logits are written out so that
+ *   bs_residual_sample(logits_t_out, logits_d_out, BS_F32, ..., workspace, ...)
+ * can follow on the same stream.
+ *
+ *  H_t  [B * (Gmax+1), d_t] bf16, d_t contiguous: row b * (Gmax+1) + j is the target model's final
+ *       hidden state at drafted position j of sequence b (j = Gmax is the bonus position)
+ *  W_t  [d_t, V] bf16, V contiguous: the target model's output embedding
+ *  H_d  [B * Gmax, d_d] bf16, W_d [d_d, V] bf16: the same for the draft model; all four may be
+ *       NULL (and d_d 0) iff temperature == 0 or Gmax == 0
+ *  logits_t_out [B, Gmax+1, V] fp32 out;  logits_d_out [B, Gmax, V] fp32 out (NULL iff no draft product)
+ *  draft_tokens, gamma, u_accept, temperature, accept_len, p_tok, q_tok: as bs_softmax_verify
+ *  workspace    at least bs_lmhead_workspace_bytes(B, Gmax, V) bytes, 256-byte aligned
+ * Every row of H is multiplied, padded positions (j > gamma_b) included: they must be readable
+ * and their logits are written, but they take no part in the verification.
+ * Requirements: V, d_t and d_d multiples of 8; all matrix pointers 16-byte aligned; otherwise
+ * BS_ERR_UNSUPPORTED / BS_ERR_INVALID_ARG.  A pipeline wait inside the kernel that does not
+ * complete within about a second makes bs_get_device_status return BS_ERR_TIMEOUT. */
+bs_status bs_lmhead_verify(const void* H_t, const void* W_t, int d_t, const void* H_d, const void* W_d, int d_d,
+                           const int32_t* draft_tokens, const int32_t* gamma, const float* u_accept,
+                           float temperature, int B, int Gmax, int V,
+                           float* logits_t_out, float* logits_d_out,
+                           int32_t* accept_len, float* p_tok, float* q_tok,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
 /* ---- arm selection (Algorithm 3, select and history lines) ---------------------------- */
 
 /* Bytes of the opaque device state of B independent bandits with K arms. 0 if out of limits. */

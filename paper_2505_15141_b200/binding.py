@@ -41,6 +41,9 @@ SIGNATURES = {
     "bs_softmax_verify": (_i, [_vp, _vp, _i, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bs_residual_sample": (_i, [_vp, _vp, _i, _vp, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _sz, _vp]),
     "bs_softmax_verify_noalloc": (_i, [_vp, _vp, _i, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _vp]),
+    "bs_lmhead_workspace_bytes": (_sz, [_i, _i, _i]),
+    "bs_lmhead_verify": (_i, [_vp, _vp, _i, _vp, _vp, _i, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _vp, _vp,
+                              _vp, _sz, _vp]),
     "bs_bandit_state_bytes": (_sz, [_i, _i, _i]),
     "bs_bandit_init": (_i, [_vp, _sz, _i, _i, _i, _vp, _d, _vp]),
     "bs_bandit_select": (_i, [_vp, _sz, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -179,6 +182,38 @@ def verify_round(target_logits, draft_logits, draft_tokens, gamma, u_accept, u_r
     bs_residual_sample(target_logits, draft_logits, draft_tokens, gamma, accept_len, u_resample,
                        temperature, out_tokens, out_len, workspace)
     return RoundOutput(accept_len, p_tok, q_tok, out_tokens, out_len, workspace)
+
+
+# ---- fused LM head ----------------------------------------------------------------------
+
+def bs_lmhead_workspace_bytes(B: int, Gmax: int, V: int) -> int:
+    return int(_lib.bs_lmhead_workspace_bytes(B, Gmax, V))
+
+
+def new_lmhead_workspace(B: int, Gmax: int, V: int, device="cuda") -> torch.Tensor:
+    n = bs_lmhead_workspace_bytes(B, Gmax, V)
+    if n == 0:
+        raise BanditSpecError(BS_ERR_UNSUPPORTED, "bs_lmhead_workspace_bytes")
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    bs_workspace_init(ws)
+    return ws
+
+
+def bs_lmhead_verify(H_t, W_t, H_d, W_d, draft_tokens, gamma, u_accept, temperature: float, B: int, Gmax: int,
+                     logits_t_out, logits_d_out, accept_len, p_tok, q_tok, workspace, stream=None) -> None:
+    """H_t [B*(Gmax+1), d_t], W_t [d_t, V], H_d [B*Gmax, d_d], W_d [d_d, V] bf16; logits out fp32."""
+    d_t, V = W_t.shape
+    assert H_t.shape == (B * (Gmax + 1), d_t) and H_t.dtype == torch.bfloat16 and W_t.dtype == torch.bfloat16
+    d_d = 0
+    if W_d is not None:
+        d_d = W_d.shape[0]
+        assert W_d.shape[1] == V and H_d.shape == (B * Gmax, d_d)
+        assert H_d.dtype == torch.bfloat16 and W_d.dtype == torch.bfloat16
+    assert logits_t_out.dtype == torch.float32 and logits_t_out.numel() == B * (Gmax + 1) * V
+    _check(_lib.bs_lmhead_verify(_ptr(H_t), _ptr(W_t), d_t, _ptr(H_d), _ptr(W_d), d_d, _ptr(draft_tokens),
+                                 _ptr(gamma), _ptr(u_accept), float(temperature), B, Gmax, V,
+                                 _ptr(logits_t_out), _ptr(logits_d_out), _ptr(accept_len), _ptr(p_tok), _ptr(q_tok),
+                                 _ptr(workspace), workspace.numel(), _stream(stream)), "bs_lmhead_verify")
 
 
 # ---- bandits ---------------------------------------------------------------------------

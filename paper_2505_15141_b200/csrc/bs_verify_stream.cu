@@ -19,6 +19,7 @@
 // its last row (atomic ticket per sequence).  Nobody waits on another CTA.  All waits on
 // mbarriers are bounded; a wait that gives up sets the abort word and the thread leaves.
 #include "bs_verify_common.cuh"
+#include "bs_pipeline.cuh"
 
 namespace bs {
 
@@ -29,7 +30,6 @@ constexpr int kVecPerStage = kSegBytes / 16;                     // 2048
 constexpr int kVecPerThread = kVecPerStage / kConsumers;         // 4
 constexpr int kMaxStages = 3;
 constexpr int kRedSlots = 8;                                     // > kMaxStages + 1 row-piece ends in flight
-constexpr long long kWaitCycles = 2000000000LL;                  // about one second
 static_assert(kVecPerThread * kConsumers == kVecPerStage, "stage must divide evenly over the consumers");
 
 // Per-stage record written by the producer: w0 = nvec | flags << 16, w1 = b | lr << 13 | sg << 19
@@ -39,49 +39,6 @@ struct StageMeta {
 };
 static_assert(BS_MAX_BATCH <= (1 << 13) && 2 * BS_MAX_GAMMA + 1 < (1 << 6) &&
               BS_MAX_VOCAB / (kSegBytes / 4) <= (1 << 8), "StageMeta packing");
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait: false if the phase did not complete within about a second.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (!mbar_try_wait(bar, parity)) {
-        if (clock64() - t0 > kWaitCycles) return false;
-    }
-    return true;
-}
-// The same for a whole warp: every lane polls, the outcome is made uniform by a vote.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity) {
-    return __all_sync(0xffffffffu, mbar_wait(bar, parity));
-}
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-__device__ __forceinline__ uint4 lds128(uint32_t addr) {
-    uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-    return v;
-}
 
 template <typename T, bool GREEDY>
 __global__ void __launch_bounds__(kStreamThreads) verify_stream_kernel(const VerifyParams p, const int nstages) {

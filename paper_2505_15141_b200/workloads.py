@@ -257,3 +257,71 @@ def make_round(w: Workload, rnd: int, arm: Optional[np.ndarray] = None,
     gamma, sig = gamma[:nb], sig[:nb]
     tok = draw_draft_tokens(d, w.temperature, un.u_draft)
     return RoundInputs(target=t, draft=d, tokens=tok, gamma=gamma, uniforms=un, sigma=sig)
+
+
+# --------------------------------------------------------------------------
+# Inputs of the fused LM-head path
+# --------------------------------------------------------------------------
+
+@dataclass(frozen=True)
+class LmHeadWorkload:
+    name: str
+    B: int
+    gamma: int                      # fixed speculation length (= Gmax)
+    V: int
+    d_t: int                        # hidden size of the target model
+    d_d: int                        # hidden size of the draft model
+    temperature: float
+    seed: int
+
+
+LMHEAD_WORKLOADS = {
+    # 128256-entry vocabulary, 4096-wide target and 2048-wide draft model, 16 sequences
+    "lmhead_llama3": LmHeadWorkload("lmhead_llama3", B=16, gamma=4, V=128256, d_t=4096, d_d=2048,
+                                    temperature=1.0, seed=3),
+    # the same model pair at a batch where the products stop being bound by streaming W
+    "lmhead_llama3_b128": LmHeadWorkload("lmhead_llama3_b128", B=128, gamma=4, V=128256, d_t=4096, d_d=2048,
+                                         temperature=1.0, seed=3),
+}
+
+
+@dataclass
+class LmHeadInputs:
+    H_t: torch.Tensor          # [B*(G+1), d_t] bf16, N(0, 1)
+    W_t: torch.Tensor          # [d_t, V] bf16, N(0, 1/d_t)
+    H_d: torch.Tensor          # [B*G, d_d] bf16
+    W_d: torch.Tensor          # [d_d, V] bf16, N(0, 1/d_d)
+    tokens: torch.Tensor       # [B, G] int32 drafted tokens
+    gamma: np.ndarray          # [B] int32
+    uniforms: RoundUniforms
+
+
+def make_lmhead_inputs(w: LmHeadWorkload, rnd: int = 1, device="cpu", gamma: Optional[np.ndarray] = None,
+                       weights: Optional[Tuple[torch.Tensor, torch.Tensor]] = None) -> LmHeadInputs:
+    """Hidden states N(0,1) and output embeddings N(0, 1/d), rounded to bf16.  The drafted tokens
+    are drawn from softmax(H_d W_d / T) with torch's matmul (input generation only).
+    `weights` re-uses (W_t, W_d) from an earlier call: the embeddings are fixed across rounds."""
+    B, G, V = w.B, w.gamma, w.V
+    g = torch_generator(w.seed, rnd, device)
+    if weights is None:
+        gw = torch_generator(w.seed, 0, device)
+        W_t = torch.empty(w.d_t, V, dtype=torch.float32, device=device).normal_(0.0, w.d_t ** -0.5, generator=gw)
+        W_t = W_t.to(torch.bfloat16)
+        W_d = torch.empty(w.d_d, V, dtype=torch.float32, device=device).normal_(0.0, w.d_d ** -0.5, generator=gw)
+        W_d = W_d.to(torch.bfloat16)
+    else:
+        W_t, W_d = weights
+    H_t = torch.empty(B * (G + 1), w.d_t, dtype=torch.float32, device=device).normal_(generator=g).to(torch.bfloat16)
+    H_d = torch.empty(B * G, w.d_d, dtype=torch.float32, device=device).normal_(generator=g).to(torch.bfloat16)
+    un = round_uniforms(w.seed, rnd, B, G)
+    if G > 0:
+        if torch.device(device).type == "cpu":
+            d_logits = (H_d.float() @ W_d.float()).view(B, G, V)
+        else:
+            d_logits = (H_d @ W_d).float().view(B, G, V)
+        tok = draw_draft_tokens(d_logits, w.temperature, un.u_draft)
+        del d_logits
+    else:
+        tok = torch.zeros(B, 0, dtype=torch.int32, device=device)
+    gam = np.full(B, G, dtype=np.int32) if gamma is None else np.asarray(gamma, dtype=np.int32)
+    return LmHeadInputs(H_t=H_t, W_t=W_t, H_d=H_d, W_d=W_d, tokens=tok.contiguous(), gamma=gam, uniforms=un)
