@@ -144,7 +144,7 @@ bs_status bs_residual_sample(const void* target_logits, const void* draft_logits
  *    call allocates and frees nothing.
  *  - Limit: bs_workspace_bytes(B, Gmax, V) must not exceed BS_NOALLOC_SCRATCH_BYTES, otherwise
  *    BS_ERR_WORKSPACE is returned and nothing is launched (e.g. B=64, Gmax=8, V=128256 needs
- *    about 160 KB; B=256, Gmax=8, V=152064 about 740 KB).
+ *    about 0.3 MB; B=256, Gmax=8, V=152064 about 1.4 MB).
  *  - The first call on each device looks up the device address of the array (with that device
  *    current).  Make that first call outside any stream capture.
  *  - All calls on a GPU share the one array.  It keeps what the previous call left; the counters
@@ -153,7 +153,7 @@ bs_status bs_residual_sample(const void* target_logits, const void* draft_logits
  *    on it and give wrong results: serialise them.
  *  - The row statistics stay inside the library, so bs_residual_sample cannot follow this call;
  *    it serves callers that need accept_len and the token probabilities only. */
-#define BS_NOALLOC_SCRATCH_BYTES (1 << 20)
+#define BS_NOALLOC_SCRATCH_BYTES (2 << 20)
 bs_status bs_softmax_verify_noalloc(const void* target_logits, const void* draft_logits, bs_dtype dtype,
                                     const int32_t* draft_tokens, const int32_t* gamma, const float* u_accept,
                                     float temperature, int B, int Gmax, int V,

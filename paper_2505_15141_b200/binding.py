@@ -138,7 +138,7 @@ def bs_residual_sample(target_logits, draft_logits, draft_tokens, gamma, accept_
                                    _ptr(workspace), workspace.numel(), _stream(stream)), "bs_residual_sample")
 
 
-BS_NOALLOC_SCRATCH_BYTES = 1 << 20
+BS_NOALLOC_SCRATCH_BYTES = 2 << 20
 
 
 def bs_softmax_verify_noalloc(target_logits, draft_logits, draft_tokens, gamma, u_accept, temperature: float,

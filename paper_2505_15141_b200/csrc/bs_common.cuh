@@ -17,6 +17,7 @@ constexpr int kSegBytes = 32768;           // row-statistics kernels: bytes of o
 constexpr int kSegElemsMin = kSegBytes / 4;  // segment length of the widest dtype (fp32)
 constexpr int kResSegBytes = 16384;        // resampling kernel: bytes of one row segment
 constexpr int kResSegElemsMin = kResSegBytes / 4;
+constexpr int kResSubSegs = 16;            // pieces of a segment whose masses are kept separately (one per consumer warp)
 constexpr float kLog2e = 1.4426950408889634f;
 
 __host__ __device__ inline int seg_elems(int dtype) { return dtype == BS_F32 ? kSegBytes / 4 : kSegBytes / 2; }
@@ -33,7 +34,8 @@ __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a -
 //   row_stats     [B, R, 2] f32, R = 2*Gmax+1: (raw max logit, Z) per row; greedy: (max, arg-max bits)
 //                 rows 0..Gmax are target rows, rows Gmax+1..2*Gmax are draft rows
 //   partial       [B, R, S, 2] f32, S = ceil(V / 8192): per-segment (max, Z) / (max, arg-max)
-//   resid_partial [B, Sr] f32, Sr = ceil(V / 4096): per-segment residual mass
+//   resid_partial [B, Sr] f32, Sr = 16 * ceil(V / 4096): residual mass of every 1 KB piece of a row pair
+//                 (the generic kernel uses one entry per 16 KB segment)
 struct Workspace {
     size_t off_ticket_verify, off_ticket_resid, off_ticket_row, off_status, off_abort, off_row_stats, off_partial,
         off_resid_partial, total;
@@ -44,7 +46,7 @@ __host__ __device__ inline Workspace workspace_layout(int B, int Gmax, int V) {
     Workspace w;
     w.R = 2 * Gmax + 1;
     w.S = div_up(V, kSegElemsMin);
-    w.Sr = div_up(V, kResSegElemsMin);
+    w.Sr = kResSubSegs * div_up(V, kResSegElemsMin);
     size_t o = 0;
     w.off_ticket_verify = o; o = align_up(o + sizeof(uint32_t) * (size_t)B, 256);
     w.off_ticket_resid = o;  o = align_up(o + sizeof(uint32_t) * (size_t)B, 256);

@@ -13,45 +13,15 @@
 //            registers in the same coalesced layout, scans the per-vector masses across the CTA
 //            in fp64, and the one thread whose vector contains the crossing walks its 4 or 8
 //            elements.  The same r_v values feed the scan and the walk.
-#include "bs_common.cuh"
+#include "bs_residual_common.cuh"
 
 #include <limits.h>
 
 namespace bs {
 
-struct ResidParams {
-    const void* target;
-    const void* draft;
-    const int32_t* tokens;
-    const int32_t* gamma;
-    const int32_t* accept_len;
-    const float* u_resample;
-    int32_t* out_tokens;
-    int32_t* out_len;
-    uint32_t* ticket;
-    int32_t* status;
-    const float2* row_stats;
-    float* resid_partial;
-    int B, Gmax, V, R, S;
-    int nseg, seg;
-    float c;
-};
-
 constexpr int kMaxSeg = BS_MAX_VOCAB / kResSegElemsMin;       // 256 = kThreads: one segment mass per thread
 constexpr int kVecTrip = kResSegBytes / 16 / kThreads;        // 128-bit vectors per thread and row in one segment
 static_assert(kMaxSeg <= kThreads, "level 2 scans one segment mass per thread");
-
-// Mass of one element.  kt / kd fold the row max and normaliser: p = 2^(x*c + kt).
-struct MassFn {
-    float c, kt, kd;
-    bool bonus;
-    __device__ __forceinline__ float operator()(float xt, float xd) const {
-        float pv = ex2(fmaf(xt, c, kt));
-        if (bonus) return pv;
-        float qv = ex2(fmaf(xd, c, kd));
-        return fmaxf(0.f, pv - qv);
-    }
-};
 
 // Masses of this thread's vectors of segment [e0, e0 + n): vector k covers elements
 // (k * kThreads + tid) * kVec .. + kVec of the segment; elements past n get mass 0.
@@ -309,8 +279,8 @@ __global__ void greedy_emit_kernel(const ResidParams p) {
 
 template <typename T>
 static bs_status launch_residual(const ResidParams& p, cudaStream_t st) {
-    // about two CTAs per SM in total, each owning a contiguous share of one sequence's segments
-    int nsplit = div_up(2 * sm_count(), p.B);
+    // at most two CTAs per SM in total (one wave), each owning a contiguous share of one sequence's segments
+    int nsplit = 2 * sm_count() / p.B;
     if (nsplit > p.nseg) nsplit = p.nseg;
     if (nsplit < 1) nsplit = 1;
     residual_kernel<T><<<(unsigned)(p.B * nsplit), kThreads, 0, st>>>(p, nsplit);
@@ -345,6 +315,7 @@ extern "C" bs_status bs_residual_sample(const void* target_logits, const void* d
     p.status = reinterpret_cast<int32_t*>(ws + w.off_status);
     p.row_stats = reinterpret_cast<const float2*>(ws + w.off_row_stats);
     p.resid_partial = reinterpret_cast<float*>(ws + w.off_resid_partial);
+    p.abort_flag = reinterpret_cast<int32_t*>(ws + w.off_abort);
     p.B = B; p.Gmax = Gmax; p.V = V; p.R = w.R; p.S = w.Sr;
     p.seg = res_seg_elems(dtype);
     p.nseg = div_up(V, p.seg);
@@ -354,5 +325,11 @@ extern "C" bs_status bs_residual_sample(const void* target_logits, const void* d
         greedy_emit_kernel<<<div_up(B, 128), 128, 0, st>>>(p);
         return cuda_status(cudaGetLastError());
     }
+    // rows on 16-byte boundaries: bulk-copy pipeline; otherwise the generic kernel
+    const size_t es = dtype == BS_F32 ? 4 : 2;
+    const bool aligned = ((size_t)V * es) % 16 == 0 && (reinterpret_cast<uintptr_t>(target_logits) & 15) == 0 &&
+                         (reinterpret_cast<uintptr_t>(draft_logits) & 15) == 0;
+    if (aligned)
+        return dtype == BS_F32 ? launch_residual_stream<float>(p, st) : launch_residual_stream<__nv_bfloat16>(p, st);
     return dtype == BS_F32 ? launch_residual<float>(p, st) : launch_residual<__nv_bfloat16>(p, st);
 }

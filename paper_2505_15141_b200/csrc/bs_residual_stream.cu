@@ -1,0 +1,528 @@
+// Pipelined resampling kernel of bs_residual_sample for rows that start on 16-byte boundaries:
+// the else-branch of Algorithm 6 (one token from Norm([P - Q]_+) at the first rejected position)
+// and the line after its loop (the bonus token from P), by inverse CDF in vocabulary order.
+//
+// A work item is one 16 KB segment of the row pair (target row tau_b, draft row tau_b) of one
+// sequence; a fully accepted sequence has only the target row, so its items weigh half.  The
+// weighted item list is cut into gridDim.x contiguous ranges, one per CTA.
+//
+//   warp 16 (one lane)  producer: for each item of its range, one or two bulk async copies
+//                       (TMA, no multicast) global -> shared into a ring of 2 x 16 KB slots,
+//                       completion on "full" mbarriers; the per-sequence constants that fold
+//                       the row statistics into the exponent travel in a per-slot record.
+//   warps 0..15         consumers: warp w owns the w-th 1 KB piece of the segment, forms
+//                       r_v = max(0, p_v - q_v) (or p_v) with two exps per element pair, and
+//                       writes the mass of its piece; no warp ever waits for another.
+//   warp 17             finisher: when the CTA's share of a sequence is done it adds the share
+//                       to the sequence's arrival counter; the finisher that completes the count
+//                       runs level 2 alone, while the other warps keep streaming: an fp64 scan of
+//                       the piece masses picks the piece in which the cumulative mass crosses
+//                       u * R, the piece (2 x 1 KB, an L2 hit) is read again, scanned in fp64 and
+//                       the crossing element is the token.  The same r_v feed both levels.
+//
+// Every wait (mbarriers, the finisher's poll of the consumers' progress) is bounded; a wait that
+// gives up sets the abort word and the thread leaves.
+#include "bs_residual_common.cuh"
+#include "bs_pipeline.cuh"
+
+#include <limits.h>
+
+namespace bs {
+
+constexpr int kRsWarps = kResSubSegs;                          // 16 consumer warps, one piece each
+constexpr int kRsConsumers = kRsWarps * 32;
+constexpr int kRsThreads = kRsConsumers + 64;                  // + producer warp + finisher warp
+constexpr int kRsStageBytes = 2 * kResSegBytes;                // target half, draft half
+constexpr int kRsMaxStages = 3;
+constexpr int kRsPieceBytes = kResSegBytes / kRsWarps;         // 1 KB of each row per warp and item
+constexpr int kRsPieceVecs = kRsPieceBytes / 16;               // 64
+constexpr int kRsVecPerLane = kRsPieceVecs / 32;               // 2
+static_assert(kRsVecPerLane * 32 * 16 * kRsWarps == kResSegBytes, "pieces must tile the segment");
+
+struct RsMeta {
+    int b, sg;
+    int nvec;        // valid 16-byte vectors of this segment (per row)
+    int flags;       // bit 0: bonus (target row only), bit 1: last item of this sequence in the CTA's range
+    float kt, kd;    // p_v = 2^(x_t c + kt), q_v = 2^(x_d c + kd)
+};
+
+// Per-sequence facts every role derives the same way.
+struct RsSeq {
+    int tau, bonus, wgt;     // weight of one item: 2 (row pair) or 1 (target row only)
+};
+__device__ __forceinline__ RsSeq rs_seq(const ResidParams& p, int b) {
+    int g = p.gamma[b];
+    if (g < 0 || g > p.Gmax) g = 0;
+    RsSeq s;
+    s.tau = max(0, min(p.accept_len[b], g));
+    s.bonus = s.tau >= g;
+    s.wgt = s.bonus ? 1 : 2;
+    return s;
+}
+// Items [i0, i1) of sequence b whose first weight unit lies in [lo, hi); pre = first unit of b.
+__device__ __forceinline__ void rs_items(int pre, int wgt, int nseg, int lo, int hi, int& i0, int& i1) {
+    const int a = max(lo, pre) - pre, e = min(hi, pre + wgt * nseg) - pre;
+    i0 = (a + wgt - 1) / wgt;
+    i1 = e > 0 ? (e + wgt - 1) / wgt : 0;
+    if (i1 < i0) i1 = i0;
+}
+
+template <typename T>
+struct RsElems {
+    static constexpr int kVec = Elem<T>::kVec;
+    // masses of one 16-byte vector of the row pair
+    __device__ static __forceinline__ void masses(const uint4& a, const uint4& d, const MassFn& f, float (&r)[kVec]) {
+        float ft[kVec], fd[kVec];
+        Elem<T>::unpack(a, ft);
+        Elem<T>::unpack(d, fd);
+#pragma unroll
+        for (int q = 0; q < kVec; ++q) r[q] = f(ft[q], fd[q]);
+    }
+};
+
+__device__ __forceinline__ double warp_scan_incl(double v) {
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double t = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += t;
+    }
+    return v;
+}
+
+// Level 2 for sequence b by one warp.  `f` has the sequence's constants.
+template <typename T>
+__device__ void rs_level2(const ResidParams& p, int b, const RsSeq sq, MassFn f) {
+    constexpr int kVec = Elem<T>::kVec;
+    const int lane = threadIdx.x & 31;
+    const T* tp = row_ptr(static_cast<const T*>(p.target), b, p.Gmax + 1, sq.tau, p.V);
+    const T* dp = f.bonus ? tp : row_ptr(static_cast<const T*>(p.draft), b, p.Gmax, sq.tau, p.V);
+    const float* pm = p.resid_partial + (size_t)b * p.S;
+    const int nsub = p.nseg * kRsWarps;
+    const int per = div_up(nsub, 32);
+    const int s0 = min(nsub, lane * per), s1 = min(nsub, s0 + per);
+    int bits = 0;
+
+    // ---- piece masses: fp64 sum per lane in index order, then a scan over the lanes ----
+    double mine = 0.0;
+    int lastpos = -1;
+    for (int i = s0; i < s1; ++i) {
+        const float m = __ldcg(pm + i);
+        mine += (double)m;
+        if (m > 0.f) lastpos = i;
+    }
+    double incl = warp_scan_incl(mine);
+    double Rtot = __shfl_sync(0xffffffffu, incl, 31);
+    const float u = p.u_resample[b];
+    int tok = -1;
+
+    if (Rtot > 0.0 && isfinite(Rtot)) {
+        const double target = (double)u * Rtot;
+        double excl = __shfl_up_sync(0xffffffffu, incl, 1);
+        if (lane == 0) excl = 0.0;
+        int ps = -1;
+        double before = 0.0;
+        if (incl > target && !(excl > target)) {              // the lane in whose pieces the crossing falls
+            double run = excl;
+            for (int i = s0; i < s1; ++i) {
+                const double m = (double)__ldcg(pm + i);
+                if (m > 0.0) { ps = i; before = run; }        // so far: the last piece with mass
+                if (run + m > target && m > 0.0) break;       // the first piece whose end passes the target
+                run += m;
+            }
+        }
+        // the lane that found the piece tells the others
+        const unsigned found = __ballot_sync(0xffffffffu, ps >= 0);
+        bool take_last = false;
+        if (found) {
+            const int src = __ffs(found) - 1;
+            ps = __shfl_sync(0xffffffffu, ps, src);
+            before = __shfl_sync(0xffffffffu, before, src);
+        } else {                                              // rounding only: the last piece with mass, its last token
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) lastpos = max(lastpos, __shfl_xor_sync(0xffffffffu, lastpos, o));
+            ps = lastpos;
+            take_last = true;
+        }
+        if (ps >= 0) {
+            const double t_in = target - before;
+            const int sg = ps / kRsWarps, w = ps - sg * kRsWarps;
+            const int e0 = sg * p.seg;
+            const int nvec = min(p.seg, p.V - e0) / kVec;
+            double pbase = 0.0;
+            int lastel = -1;
+#pragma unroll
+            for (int q = 0; q < kRsVecPerLane; ++q) {
+                const int iv = w * kRsPieceVecs + q * 32 + lane;
+                float r[kVec];
+#pragma unroll
+                for (int k = 0; k < kVec; ++k) r[k] = 0.f;
+                if (iv < nvec) {
+                    const uint4 a = __ldcg(reinterpret_cast<const uint4*>(tp + e0) + iv);
+                    const uint4 d = f.bonus ? a : __ldcg(reinterpret_cast<const uint4*>(dp + e0) + iv);
+                    RsElems<T>::masses(a, d, f, r);
+                }
+                float vs = 0.f;
+#pragma unroll
+                for (int k = 0; k < kVec; ++k) {
+                    vs += r[k];
+                    if (r[k] > 0.f) lastel = e0 + iv * kVec + k;
+                }
+                const double sc = warp_scan_incl((double)vs);
+                double sx = __shfl_up_sync(0xffffffffu, sc, 1);
+                if (lane == 0) sx = 0.0;
+                const double vin = pbase + sc, vex = pbase + sx;
+                int cand = INT_MAX;
+                if (!take_last && vin > t_in && !(vex > t_in)) {
+                    double run = vex;
+#pragma unroll
+                    for (int k = 0; k < kVec; ++k) {
+                        run += (double)r[k];
+                        if (cand == INT_MAX && run > t_in && r[k] > 0.f) cand = e0 + iv * kVec + k;
+                    }
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) cand = min(cand, __shfl_xor_sync(0xffffffffu, cand, o));
+                if (tok < 0 && cand != INT_MAX) tok = cand;
+                pbase = __shfl_sync(0xffffffffu, vin, 31);
+            }
+            if (tok < 0) {                                    // u * R at or beyond the recomputed mass of the piece
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) lastel = max(lastel, __shfl_xor_sync(0xffffffffu, lastel, o));
+                tok = lastel;
+            }
+        }
+    }
+    if (tok < 0) {
+        // [P - Q]_+ has no mass (P == Q up to rounding) or a statistic is not finite: sample from
+        // the target distribution of the same row.  Rare; one warp walks the row twice.
+        bits |= f.bonus ? BS_DEV_NONFINITE : BS_DEV_RESIDUAL_FALLBACK;
+        MassFn fp = f;
+        fp.bonus = true;
+        const int nv = p.V / kVec;
+        double tot = 0.0;
+        for (int v0 = 0; v0 < nv; v0 += 32) {
+            float vs = 0.f;
+            if (v0 + lane < nv) {
+                const uint4 a = __ldcg(reinterpret_cast<const uint4*>(tp) + v0 + lane);
+                float r[kVec];
+                RsElems<T>::masses(a, a, fp, r);
+#pragma unroll
+                for (int k = 0; k < kVec; ++k) vs += r[k];
+            }
+            tot += __shfl_sync(0xffffffffu, warp_scan_incl((double)vs), 31);
+        }
+        if (tot > 0.0 && isfinite(tot)) {
+            const double target = (double)u * tot;
+            double base = 0.0;
+            int lastel = -1;
+            for (int v0 = 0; v0 < nv && tok < 0; v0 += 32) {
+                float r[kVec];
+#pragma unroll
+                for (int k = 0; k < kVec; ++k) r[k] = 0.f;
+                if (v0 + lane < nv) {
+                    const uint4 a = __ldcg(reinterpret_cast<const uint4*>(tp) + v0 + lane);
+                    RsElems<T>::masses(a, a, fp, r);
+                }
+                float vs = 0.f;
+#pragma unroll
+                for (int k = 0; k < kVec; ++k) {
+                    vs += r[k];
+                    if (r[k] > 0.f) lastel = (v0 + lane) * kVec + k;
+                }
+                const double sc = warp_scan_incl((double)vs);
+                double sx = __shfl_up_sync(0xffffffffu, sc, 1);
+                if (lane == 0) sx = 0.0;
+                const double vin = base + sc, vex = base + sx;
+                int cand = INT_MAX;
+                if (vin > target && !(vex > target)) {
+                    double run = vex;
+#pragma unroll
+                    for (int k = 0; k < kVec; ++k) {
+                        run += (double)r[k];
+                        if (cand == INT_MAX && run > target && r[k] > 0.f) cand = (v0 + lane) * kVec + k;
+                    }
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) cand = min(cand, __shfl_xor_sync(0xffffffffu, cand, o));
+                if (cand != INT_MAX) tok = cand;
+                base = __shfl_sync(0xffffffffu, vin, 31);
+            }
+            if (tok < 0) {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) lastel = max(lastel, __shfl_xor_sync(0xffffffffu, lastel, o));
+                tok = lastel;
+            }
+        }
+        if (tok < 0) { tok = 0; bits |= BS_DEV_NONFINITE; }
+    }
+    // ---- outputs: the tau accepted drafts, the sampled token, padding ----
+    int32_t* ot = p.out_tokens + (size_t)b * (p.Gmax + 1);
+    for (int j = lane; j <= p.Gmax; j += 32)
+        ot[j] = j < sq.tau ? p.tokens[(size_t)b * p.Gmax + j] : (j == sq.tau ? tok : -1);
+    if (lane == 0) {
+        p.out_len[b] = sq.tau + 1;
+        if (bits) p.status[b] |= bits;
+        p.ticket[b] = 0u;                                     // leave the counter clear for the next call
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const ResidParams p, const int nstages) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    // layout: [nstages * 32 KB ring][prefix (B+1) ints]
+    unsigned char* ring = smem;
+    int* s_prefix = reinterpret_cast<int*>(smem + (size_t)nstages * kRsStageBytes);
+    __shared__ __align__(8) unsigned long long s_full[kRsMaxStages];
+    __shared__ __align__(8) unsigned long long s_empty[kRsMaxStages];
+    __shared__ RsMeta s_meta[kRsMaxStages];
+    __shared__ int s_scan[kRsThreads / 32];
+    __shared__ int s_count;                                   // items of this CTA
+    __shared__ unsigned int s_done;                           // consumer warps that finished a sequence share
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int kVec = Elem<T>::kVec;
+
+    if (tid == 0) {
+        for (int s = 0; s < nstages; ++s) {
+            mbar_init(smem_u32(&s_full[s]), 1);
+            mbar_init(smem_u32(&s_empty[s]), kRsWarps);
+        }
+        s_count = 0;
+        s_done = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+
+    // ---- prefix sum of item weights over the batch (all threads, redundantly per CTA) ----
+    {
+        const int per = div_up(p.B, kRsThreads);
+        const int b0 = tid * per;
+        int local = 0;
+        for (int k = 0; k < per; ++k) {
+            const int b = b0 + k;
+            if (b < p.B) local += rs_seq(p, b).wgt * p.nseg;
+        }
+        int incl = local;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (lane == 31) s_scan[warp] = incl;
+        __syncthreads();
+        int woff = 0;
+        for (int w = 0; w < warp; ++w) woff += s_scan[w];
+        int run = woff + incl - local;
+        for (int k = 0; k < per; ++k) {
+            const int b = b0 + k;
+            if (b < p.B) {
+                s_prefix[b] = run;
+                run += rs_seq(p, b).wgt * p.nseg;
+            }
+        }
+        if (tid == kRsThreads - 1) s_prefix[p.B] = run;
+        __syncthreads();                                      // also publishes the mbarrier inits
+    }
+    const int total = s_prefix[p.B];
+    const int lo = (int)((long long)total * blockIdx.x / gridDim.x);
+    const int hi = (int)((long long)total * (blockIdx.x + 1) / gridDim.x);
+    // first and last sequence that overlap [lo, hi)
+    int bfirst, blast;
+    {
+        int l = 0, h = p.B;                                   // largest b with prefix[b] <= lo
+        while (h - l > 1) {
+            const int mid = (l + h) >> 1;
+            if (s_prefix[mid] <= lo) l = mid; else h = mid;
+        }
+        bfirst = l;
+        l = 0; h = p.B;                                       // largest b with prefix[b] < hi
+        while (h - l > 1) {
+            const int mid = (l + h) >> 1;
+            if (s_prefix[mid] < hi) l = mid; else h = mid;
+        }
+        blast = l;
+    }
+    // number of items of this CTA (every thread needs it to know when to stop)
+    {
+        int mine = 0;
+        for (int b = bfirst + tid; b <= blast; b += kRsThreads) {
+            int i0, i1;
+            rs_items(s_prefix[b], (s_prefix[b + 1] - s_prefix[b]) / p.nseg, p.nseg, lo, hi, i0, i1);
+            mine += i1 - i0;
+        }
+        if (mine) atomicAdd(&s_count, mine);
+        __syncthreads();
+    }
+    const int count = s_count;
+    if (count <= 0 || hi <= lo) return;
+
+    if (warp == kRsWarps) {
+        // =============================== producer ===============================
+        if (lane != 0) return;
+        int slot = 0;
+        uint32_t ph = 0;
+        for (int b = bfirst; b <= blast; ++b) {
+            const RsSeq sq = rs_seq(p, b);
+            int i0, i1;
+            rs_items(s_prefix[b], sq.wgt, p.nseg, lo, hi, i0, i1);
+            if (i1 <= i0) continue;
+            const float2 ts = p.row_stats[(size_t)b * p.R + sq.tau];
+            float kt = -(ts.x * p.c + log2f(ts.y)), kd = 0.f;
+            const T* tp = row_ptr(static_cast<const T*>(p.target), b, p.Gmax + 1, sq.tau, p.V);
+            const T* dp = tp;
+            if (!sq.bonus) {
+                const float2 ds = p.row_stats[(size_t)b * p.R + p.Gmax + 1 + sq.tau];
+                kd = -(ds.x * p.c + log2f(ds.y));
+                dp = row_ptr(static_cast<const T*>(p.draft), b, p.Gmax, sq.tau, p.V);
+            }
+            for (int sg = i0; sg < i1; ++sg) {
+                if (!mbar_wait(smem_u32(&s_empty[slot]), ph ^ 1u)) { atomicExch(p.abort_flag, 1); return; }
+                const int e0 = sg * p.seg;
+                const int n = min(p.seg, p.V - e0);
+                const uint32_t bytes = (uint32_t)n * (uint32_t)sizeof(T);
+                RsMeta m;
+                m.b = b; m.sg = sg; m.nvec = n / kVec;
+                m.flags = (sq.bonus ? 1 : 0) | (sg == i1 - 1 ? 2 : 0);
+                m.kt = kt; m.kd = kd;
+                s_meta[slot] = m;
+                const uint32_t bar = smem_u32(&s_full[slot]);
+                const uint32_t dst = smem_u32(ring + (size_t)slot * kRsStageBytes);
+                mbar_arrive_expect_tx(bar, sq.bonus ? bytes : 2u * bytes);   // releases the record to the waiters
+                bulk_load(dst, tp + e0, bytes, bar);
+                if (!sq.bonus) bulk_load(dst + kResSegBytes, dp + e0, bytes, bar);
+                if (++slot == nstages) { slot = 0; ph ^= 1u; }
+            }
+        }
+        return;
+    }
+
+    if (warp == kRsWarps + 1) {
+        // =============================== finisher ===============================
+        unsigned shares = 0;                                  // sequence shares of this CTA seen so far
+        for (int b = bfirst; b <= blast; ++b) {
+            const RsSeq sq = rs_seq(p, b);
+            int i0, i1;
+            rs_items(s_prefix[b], sq.wgt, p.nseg, lo, hi, i0, i1);
+            if (i1 <= i0) continue;
+            ++shares;
+            // wait until all consumer warps have written their masses of this share
+            {
+                const unsigned want = shares * (unsigned)kRsWarps;
+                const long long t0 = clock64();
+                bool ok = true;
+                while (*reinterpret_cast<volatile unsigned int*>(&s_done) < want) {
+                    if (clock64() - t0 > kWaitCycles) { ok = false; break; }
+                    __nanosleep(64);
+                }
+                if (!__all_sync(0xffffffffu, ok)) {
+                    if (lane == 0) atomicExch(p.abort_flag, 1);
+                    return;
+                }
+            }
+            __threadfence();
+            unsigned old = 0;
+            if (lane == 0) old = atomicAdd(p.ticket + b, (unsigned)(i1 - i0));
+            old = __shfl_sync(0xffffffffu, old, 0);
+            if (old + (unsigned)(i1 - i0) == (unsigned)p.nseg) {
+                __threadfence();
+                MassFn f;
+                f.c = p.c;
+                f.bonus = sq.bonus;
+                const float2 ts = p.row_stats[(size_t)b * p.R + sq.tau];
+                f.kt = -(ts.x * p.c + log2f(ts.y));
+                f.kd = 0.f;
+                if (!sq.bonus) {
+                    const float2 ds = p.row_stats[(size_t)b * p.R + p.Gmax + 1 + sq.tau];
+                    f.kd = -(ds.x * p.c + log2f(ds.y));
+                }
+                rs_level2<T>(p, b, sq, f);
+            }
+        }
+        return;
+    }
+
+    // ================================= consumers =================================
+    int slot = 0;
+    uint32_t ph = 0;
+    for (int k = 0; k < count; ++k) {
+        if (!mbar_wait_warp(smem_u32(&s_full[slot]), ph)) { atomicExch(p.abort_flag, 1); return; }
+        const RsMeta m = s_meta[slot];
+        MassFn f;
+        f.c = p.c; f.kt = m.kt; f.kd = m.kd; f.bonus = (m.flags & 1) != 0;
+        const uint32_t base = smem_u32(ring + (size_t)slot * kRsStageBytes) + (uint32_t)(warp * kRsPieceBytes + lane * 16);
+        uint4 a[kRsVecPerLane], d[kRsVecPerLane];
+        bool valid[kRsVecPerLane];
+#pragma unroll
+        for (int q = 0; q < kRsVecPerLane; ++q) {
+            valid[q] = warp * kRsPieceVecs + q * 32 + lane < m.nvec;
+            if (valid[q]) {
+                a[q] = lds128(base + (uint32_t)(q * 512));
+                d[q] = f.bonus ? a[q] : lds128(base + (uint32_t)(kResSegBytes + q * 512));
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&s_empty[slot]));  // the slot's data is in registers now
+        float acc = 0.f;
+#pragma unroll
+        for (int q = 0; q < kRsVecPerLane; ++q) {
+            if (valid[q]) {
+                float r[kVec];
+                RsElems<T>::masses(a[q], d[q], f, r);
+                float vs = 0.f;
+#pragma unroll
+                for (int i = 0; i < kVec; ++i) vs += r[i];
+                acc += vs;
+            }
+        }
+        acc = warp_sum(acc);
+        if (lane == 0) {
+            p.resid_partial[(size_t)m.b * p.S + m.sg * kRsWarps + warp] = acc;
+            if (m.flags & 2) {                                // this CTA's share of the sequence ends here
+                __threadfence();
+                atomicAdd(&s_done, 1u);
+            }
+        }
+        if (++slot == nstages) { slot = 0; ph ^= 1u; }
+    }
+}
+
+static int g_rs_smem[64];          // opt-in shared memory limit per device (0 = not queried)
+static bool g_rs_attr[2][64];
+
+template <typename T>
+bs_status launch_residual_stream(const ResidParams& p, cudaStream_t st) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64) dev = 0;
+    if (!g_rs_smem[dev]) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
+            return cuda_status(cudaGetLastError());
+        g_rs_smem[dev] = v;
+    }
+    // two CTAs per SM: each may use half of the SM's shared memory minus the static part
+    const size_t prefix_bytes = align_up(sizeof(int) * (size_t)(p.B + 1), 128);
+    const size_t budget = (size_t)(g_rs_smem[dev] + 1024) / 2 - 3072;
+    int nst = (int)((budget - prefix_bytes) / kRsStageBytes);
+    if (nst > kRsMaxStages) nst = kRsMaxStages;
+    if (nst < 2) return BS_ERR_UNSUPPORTED;
+    const size_t smem = (size_t)nst * kRsStageBytes + prefix_bytes;
+    const int variant = Elem<T>::kDtype == BS_F32 ? 0 : 1;
+    if (!g_rs_attr[variant][dev]) {
+        if (cudaFuncSetAttribute(residual_stream_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 g_rs_smem[dev] - 4096) != cudaSuccess)
+            return cuda_status(cudaGetLastError());
+        g_rs_attr[variant][dev] = true;
+    }
+    long long grid = 2LL * sm_count();
+    const long long items = (long long)p.B * p.nseg;
+    if (grid > items) grid = items;
+    if (grid < 1) grid = 1;
+    residual_stream_kernel<T><<<(unsigned)grid, kRsThreads, smem, st>>>(p, nst);
+    return cuda_status(cudaGetLastError());
+}
+
+template bs_status launch_residual_stream<float>(const ResidParams&, cudaStream_t);
+template bs_status launch_residual_stream<__nv_bfloat16>(const ResidParams&, cudaStream_t);
+
+}  // namespace bs
