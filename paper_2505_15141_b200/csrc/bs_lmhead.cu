@@ -6,7 +6,7 @@
 //   W  [d, V]  bf16, V contiguous   (the output embedding, streamed once from HBM)
 //   out[M, V]  fp32                 (kept for the resampling step)
 //
-// One persistent CTA per SM walks a static list of 128 x BN output tiles (target product first,
+// One persistent CTA per SM walks a static list of 128 x BN or 256 x BN output tiles (target product first,
 // then the draft product; tiles that share a slice of W are adjacent in the list so the slice
 // comes from L2 the second time).  Per CTA:
 //   warp 0 (one lane)   TMA producer: per 64-deep k-block one 128 x 64 box of H (K-major,
@@ -17,12 +17,11 @@
 //                       K = 16) on shared-memory descriptors, accumulating in tensor memory;
 //                       tcgen05.commit releases the stage ("empty") and, after the last
 //                       k-block, publishes the accumulator ("tmem_full").
-//   warps 2..5          epilogue: tcgen05.ld their 32 lanes of the accumulator, 32 columns at a
-//                       time; every thread owns one output row, so the running (max, sum exp)
-//                       or (max, arg-max) of that row over the tile needs no shuffle; the fp32
-//                       logits go to global memory, the per-(row, tile) statistics to a partial
-//                       buffer.  Two accumulators in tensor memory let the epilogue of a tile
-//                       overlap the k-loop of the next.
+//   warps 2..9          epilogue: tcgen05.ld their 32 lanes of the accumulator, 32 columns at a
+//                       time (four lane quarters x two column halves); every thread owns one
+//                       output row, so the running (max, sum exp) or (max, arg-max) of that row
+//                       over its half tile needs no shuffle; the fp32 logits go to global memory,
+//                       the per-(row, half tile) statistics to a partial buffer.
 // A second small kernel merges the partials of every row, stores the row statistics in the
 // workspace (where bs_residual_sample reads them) and runs the accept scan.
 //
@@ -38,7 +37,8 @@ namespace bs {
 constexpr int kLmBM = 128;                 // tile rows = UMMA M = tensor-memory lanes
 constexpr int kLmBK = 64;                  // k-extent of a stage: 64 bf16 = one 128-byte swizzle row
 constexpr int kLmUK = 16;                  // k-extent of one tcgen05.mma for 16-bit operands
-constexpr int kLmThreads = 192;            // producer warp, MMA warp, four epilogue warps
+constexpr int kLmEpiWarps = 8;             // epilogue warps: 4 lane quarters x 2 column halves
+constexpr int kLmThreads = 64 + 32 * kLmEpiWarps;   // producer warp, MMA warp, epilogue warps
 constexpr int kLmABytes = kLmBM * kLmBK * 2;                      // 16 KB of H per stage
 constexpr int kLmChunkBytes = kLmBK * 128;                        // 64 k-rows x 64 n (128 B) of W = 8 KB
 constexpr int kLmTmemCols = 512;           // two fp32 accumulators of up to 256 columns
@@ -47,7 +47,7 @@ struct LmProduct {
     float* out;            // [M, V] fp32 logits
     int M;                 // rows of H
     int KB;                // k-blocks: ceil(d / 64)
-    int MT;                // row tiles: ceil(M / 128)
+    int MT;                // row tiles of one CTA: ceil(M / (128 * MH))
     int rows_per_seq;      // Gmax + 1 (target) or Gmax (draft)
     int slot0;             // row slot of a sequence's first row in the statistics: 0 or Gmax + 1
 };
@@ -57,7 +57,7 @@ struct LmParams {
     int nprod;             // 2, or 1 when there are no draft rows (greedy mode, Gmax = 0)
     int V, NT, R;          // vocabulary, column tiles ceil(V / BN), row slots per sequence 2 Gmax + 1
     float c;               // log2(e) / temperature
-    float2* partial;       // [B * R, NT] per-tile statistics
+    float2* partial;       // [B * R, 2 NT] statistics per row and half column tile
     int32_t* abort_flag;
 };
 
@@ -73,6 +73,11 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm,
 __device__ __forceinline__ uint64_t policy_evict_first() {
     uint64_t p;
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t policy_evict_normal() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
     return p;
 }
 __device__ __forceinline__ uint64_t policy_evict_last() {
@@ -136,15 +141,23 @@ __device__ __forceinline__ LmTile lm_tile(const LmParams& p, int t) {
     return r;
 }
 
-template <int BN, int STAGES, bool GREEDY>
+// MH = row tiles of 128 that one CTA multiplies against the same 64 x BN block of W per stage.
+//   MH = 1  (M <= 128): two accumulators of BN columns alternate between tiles, so the epilogue
+//           of a tile runs under the k-loop of the next; 4 stages of 16 + 32 KB.
+//   MH = 2  (larger M): a 256 x BN tile, both accumulators belong to the current tile; every byte
+//           of W brought into shared memory feeds twice the MMAs (half the L2 -> SM traffic per
+//           flop, twice the time a stage lasts); 3 stages of 32 + 32 KB.
+template <int BN, int MH, int STAGES, bool GREEDY>
 __global__ void __launch_bounds__(kLmThreads, 1)
 lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tm_h0, const __grid_constant__ CUtensorMap tm_w0,
                    const __grid_constant__ CUtensorMap tm_h1, const __grid_constant__ CUtensorMap tm_w1,
                    const LmParams p) {
     constexpr int kChunks = BN / 64;
     constexpr int kBBytes = kChunks * kLmChunkBytes;
-    constexpr int kStageBytes = kLmABytes + kBBytes;
+    constexpr int kStageBytes = MH * kLmABytes + kBBytes;
+    constexpr int kHalfCols = BN / 2;                         // columns one epilogue warp covers
     static_assert(BN % 64 == 0 && BN >= 64 && 2 * BN <= kLmTmemCols, "tile width");
+    static_assert(MH == 1 || MH == 2, "row tiles per CTA");
     static_assert(kStageBytes % 1024 == 0, "stages must keep the 1024-byte swizzle alignment");
 
     extern __shared__ unsigned char lm_smem_raw[];
@@ -168,7 +181,7 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tm_h0, const __grid_const
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(smem_u32(&s_tmem_full[a]), 1);
-            mbar_init(smem_u32(&s_tmem_empty[a]), 4);         // one arrival per epilogue warp
+            mbar_init(smem_u32(&s_tmem_empty[a]), kLmEpiWarps);   // one arrival per epilogue warp
         }
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -183,11 +196,20 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tm_h0, const __grid_const
     tc_fence_after();
     const uint32_t tmem_base = s_tmem_base;
 
+    // Accumulator used by tile number `it` of this CTA for row half `h`.  The MMA issuer and the
+    // epilogue warps each count how often an accumulator has been used (`uses`): the parity of
+    // that count is the phase of its two barriers.
+    auto acc_of = [](int it, int h) { return MH == 1 ? (it & 1) : h; };
+
     if (warp == 0) {
         // ================================ TMA producer ================================
         if (lane == 0) {
-            const uint64_t pol_w = policy_evict_first();      // W is read once
-            const uint64_t pol_h = policy_evict_last();       // H is re-read by every column tile
+            // W is read by one CTA per column tile (evict first) or by several at about the same
+            // time (normal priority, so that the later ones find it in L2); H is re-read by every
+            // column tile.
+            const bool w_once = p.prod[0].MT == 1 && (p.nprod == 1 || p.prod[1].MT == 1);
+            const uint64_t pol_w = w_once ? policy_evict_first() : policy_evict_normal();
+            const uint64_t pol_h = policy_evict_last();
             int slot = 0;
             uint32_t ph = 0;
             bool ok = true;
@@ -197,16 +219,19 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tm_h0, const __grid_const
                 const CUtensorMap* tw = tl.prod ? &tm_w1 : &tm_w0;
                 const int KB = p.prod[tl.prod].KB;
                 const int n0 = tl.nt * BN;
+                const int m0 = tl.mt * (kLmBM * MH);
+                const int halves = (MH == 2 && m0 + kLmBM < p.prod[tl.prod].M) ? 2 : 1;
                 const int chunks = min(kChunks, (p.V - n0 + 63) / 64);      // chunks that hold any column < V
-                const uint32_t tx = (uint32_t)(kLmABytes + chunks * kLmChunkBytes);
+                const uint32_t tx = (uint32_t)(halves * kLmABytes + chunks * kLmChunkBytes);
                 for (int kb = 0; kb < KB; ++kb) {
                     if (!mbar_wait(smem_u32(&s_empty[slot]), ph ^ 1u) || s_abort) { ok = false; break; }
                     const uint32_t bar = smem_u32(&s_full[slot]);
                     const uint32_t sa = smem_u32(smem + (size_t)slot * kStageBytes);
                     mbar_arrive_expect_tx(bar, tx);
-                    tma_load_2d(sa, th, kb * kLmBK, tl.mt * kLmBM, bar, pol_h);
+                    for (int h = 0; h < halves; ++h)
+                        tma_load_2d(sa + h * kLmABytes, th, kb * kLmBK, m0 + h * kLmBM, bar, pol_h);
                     for (int j = 0; j < chunks; ++j)
-                        tma_load_2d(sa + kLmABytes + j * kLmChunkBytes, tw, n0 + j * 64, kb * kLmBK, bar, pol_w);
+                        tma_load_2d(sa + MH * kLmABytes + j * kLmChunkBytes, tw, n0 + j * 64, kb * kLmBK, bar, pol_w);
                     if (++slot == STAGES) { slot = 0; ph ^= 1u; }
                 }
             }
@@ -218,105 +243,127 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tm_h0, const __grid_const
             constexpr uint32_t idesc = lm_idesc(BN);
             int slot = 0;
             uint32_t ph = 0;
+            uint32_t uses[2] = {0u, 0u};
             int it = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
                 const LmTile tl = lm_tile(p, t);
                 const int KB = p.prod[tl.prod].KB;
-                const int acc = it & 1;
-                // the epilogue must have drained this accumulator (two tiles ago)
-                if (!mbar_wait(smem_u32(&s_tmem_empty[acc]), (((uint32_t)it >> 1) & 1u) ^ 1u) || s_abort) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-                for (int kb = 0; kb < KB; ++kb) {
+                const int m0 = tl.mt * (kLmBM * MH);
+                const int halves = (MH == 2 && m0 + kLmBM < p.prod[tl.prod].M) ? 2 : 1;
+                for (int kb = 0; kb < KB && ok; ++kb) {
                     if (!mbar_wait(smem_u32(&s_full[slot]), ph) || s_abort) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = smem_u32(smem + (size_t)slot * kStageBytes);
-                    const uint32_t sb = sa + kLmABytes;
+                    const uint32_t sb = sa + MH * kLmABytes;
+                    for (int h = 0; h < halves; ++h) {
+                        const int acc = acc_of(it, h);
+                        if (kb == 0) {
+                            // the epilogue must have drained this accumulator (its previous use)
+                            if (!mbar_wait(smem_u32(&s_tmem_empty[acc]), (uses[acc] & 1u) ^ 1u) || s_abort) { ok = false; break; }
+                            tc_fence_after();
+                        }
+                        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
 #pragma unroll
-                    for (int k = 0; k < kLmBK / kLmUK; ++k) {
-                        // A, K-major: rows of 128 B, 8-row groups 1024 B apart; a k-step is 32 B inside the row
-                        const uint64_t a_desc = smem_desc(sa + k * (kLmUK * 2), 16, 1024);
-                        // B, N-major: 64-column chunks kLmChunkBytes apart (leading), 8-k-row groups
-                        // 1024 B apart (stride); a k-step is 16 rows of 128 B
-                        const uint64_t b_desc = smem_desc(sb + k * (kLmUK * 128), kLmChunkBytes, 1024);
-                        tc_mma_bf16(d_tmem, a_desc, b_desc, idesc, (kb | k) ? 1u : 0u);
+                        for (int k = 0; k < kLmBK / kLmUK; ++k) {
+                            // A, K-major: rows of 128 B, 8-row groups 1024 B apart; a k-step is 32 B inside the row
+                            const uint64_t a_desc = smem_desc(sa + h * kLmABytes + k * (kLmUK * 2), 16, 1024);
+                            // B, N-major: 64-column chunks kLmChunkBytes apart (leading), 8-k-row groups
+                            // 1024 B apart (stride); a k-step is 16 rows of 128 B
+                            const uint64_t b_desc = smem_desc(sb + k * (kLmUK * 128), kLmChunkBytes, 1024);
+                            tc_mma_bf16(d_tmem, a_desc, b_desc, idesc, (kb | k) ? 1u : 0u);
+                        }
                     }
+                    if (!ok) break;
                     tc_commit(smem_u32(&s_empty[slot]));       // the stage may be refilled once these MMAs retire
                     if (++slot == STAGES) { slot = 0; ph ^= 1u; }
                 }
-                if (ok) tc_commit(smem_u32(&s_tmem_full[acc]));
+                if (ok)
+                    for (int h = 0; h < halves; ++h) {
+                        tc_commit(smem_u32(&s_tmem_full[acc_of(it, h)]));
+                        ++uses[acc_of(it, h)];
+                    }
             }
             if (!ok) { s_abort = 1; atomicExch(p.abort_flag, 1); }
         }
     } else {
         // ================================== epilogue ==================================
-        const int quarter = warp & 3;                         // the tensor-memory lanes this warp may read
+        // warps 2..9: lane quarter warp % 4 of the accumulator (the lanes a warp may read), column
+        // half (warp - 2) / 4 of the tile
+        const int quarter = warp & 3;
+        const int chalf = (warp - 2) >> 2;
+        uint32_t uses[2] = {0u, 0u};
         int it = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
             const LmTile tl = lm_tile(p, t);
             const LmProduct& pr = p.prod[tl.prod];
-            const int acc = it & 1;
-            // warp-uniform outcome: the tensor-memory loads below need the whole warp
-            const bool arrived = mbar_wait_warp(smem_u32(&s_tmem_full[acc]), ((uint32_t)it >> 1) & 1u);
-            const int aborted = __shfl_sync(0xffffffffu, (int)s_abort, 0);
-            if (!arrived || aborted) { ok = false; break; }
-            tc_fence_after();
-            const int row = tl.mt * kLmBM + quarter * 32 + lane;
-            const bool row_ok = row < pr.M;
-            const int n0 = tl.nt * BN;
-            const int ncols = min(BN, p.V - n0);
-            float* orow = pr.out + (size_t)(row_ok ? row : 0) * p.V + n0;
-            Online on{-INFINITY, 0.f};
-            ArgMax am{-INFINITY, INT_MAX};
-            if (quarter * 32 + tl.mt * kLmBM < pr.M) {        // some row of this warp exists
-                for (int c0 = 0; c0 < ncols; c0 += 32) {
-                    uint32_t v[32];
-                    tc_load_32cols(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + c0), v);
-                    const int nv = min(32, ncols - c0);       // valid columns of this group (a multiple of 4)
-                    if (row_ok) {
-                        if (GREEDY) {
+            const int m0 = tl.mt * (kLmBM * MH);
+            const int halves = (MH == 2 && m0 + kLmBM < pr.M) ? 2 : 1;
+            for (int h = 0; h < halves && ok; ++h) {
+                const int acc = acc_of(it, h);
+                // warp-uniform outcome: the tensor-memory loads below need the whole warp
+                const bool arrived = mbar_wait_warp(smem_u32(&s_tmem_full[acc]), uses[acc] & 1u);
+                ++uses[acc];
+                const int aborted = __shfl_sync(0xffffffffu, (int)s_abort, 0);
+                if (!arrived || aborted) { ok = false; break; }
+                tc_fence_after();
+                const int row = m0 + h * kLmBM + quarter * 32 + lane;
+                const bool row_ok = row < pr.M;
+                const int n0 = tl.nt * BN + chalf * kHalfCols;
+                const int ncols = max(0, min(kHalfCols, p.V - n0));
+                float* orow = pr.out + (size_t)(row_ok ? row : 0) * p.V + n0;
+                Online on{-INFINITY, 0.f};
+                ArgMax am{-INFINITY, INT_MAX};
+                if (m0 + h * kLmBM + quarter * 32 < pr.M) {   // some row of this warp exists
+                    for (int c0 = 0; c0 < ncols; c0 += 32) {
+                        uint32_t v[32];
+                        tc_load_32cols(tmem_base + ((uint32_t)(quarter * 32) << 16) +
+                                           (uint32_t)(acc * BN + chalf * kHalfCols + c0), v);
+                        const int nv = min(32, ncols - c0);   // valid columns of this group (a multiple of 4)
+                        if (row_ok) {
+                            if (GREEDY) {
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) {
-                                const float x = __uint_as_float(v[i]);
-                                if (i < nv && x > am.m) { am.m = x; am.idx = n0 + c0 + i; }
-                            }
-                        } else {
-                            float cm = -INFINITY;
-#pragma unroll
-                            for (int i = 0; i < 32; ++i)
-                                if (i < nv) cm = fmaxf(cm, __uint_as_float(v[i]));
-                            on.raise_to(cm, p.c);
-                            if (on.m > -INFINITY) {
-                                const float nm = -on.m * p.c;
-                                float a0 = 0.f, a1 = 0.f;
-#pragma unroll
-                                for (int i = 0; i < 32; i += 2) {
-                                    if (i < nv) {
-                                        a0 += ex2(fmaf(__uint_as_float(v[i]), p.c, nm));
-                                        a1 += ex2(fmaf(__uint_as_float(v[i + 1]), p.c, nm));
-                                    }
+                                for (int i = 0; i < 32; ++i) {
+                                    const float x = __uint_as_float(v[i]);
+                                    if (i < nv && x > am.m) { am.m = x; am.idx = n0 + c0 + i; }
                                 }
-                                on.s += a0 + a1;
-                            }
-                        }
+                            } else {
+                                float cm = -INFINITY;
 #pragma unroll
-                        for (int i = 0; i < 32; i += 4)
-                            if (i < nv)
-                                *reinterpret_cast<uint4*>(orow + c0 + i) = make_uint4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                                for (int i = 0; i < 32; ++i)
+                                    if (i < nv) cm = fmaxf(cm, __uint_as_float(v[i]));
+                                on.raise_to(cm, p.c);
+                                if (on.m > -INFINITY) {
+                                    const float nm = -on.m * p.c;
+                                    float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+                                    for (int i = 0; i < 32; i += 2) {
+                                        if (i < nv) {
+                                            a0 += ex2(fmaf(__uint_as_float(v[i]), p.c, nm));
+                                            a1 += ex2(fmaf(__uint_as_float(v[i + 1]), p.c, nm));
+                                        }
+                                    }
+                                    on.s += a0 + a1;
+                                }
+                            }
+#pragma unroll
+                            for (int i = 0; i < 32; i += 4)
+                                if (i < nv)
+                                    *reinterpret_cast<uint4*>(orow + c0 + i) = make_uint4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                        }
                     }
                 }
-            }
-            // accumulator drained: hand it back before the bookkeeping
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&s_tmem_empty[acc]));
-            if (row_ok) {
-                const int b = row / pr.rows_per_seq;
-                const int j = row - b * pr.rows_per_seq;
-                p.partial[((size_t)b * p.R + pr.slot0 + j) * p.NT + tl.nt] =
-                    GREEDY ? make_float2(am.m, __int_as_float(am.idx)) : make_float2(on.m, on.s);
+                // accumulator drained: hand it back before the bookkeeping
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&s_tmem_empty[acc]));
+                if (row_ok) {
+                    const int b = row / pr.rows_per_seq;
+                    const int j = row - b * pr.rows_per_seq;
+                    p.partial[((size_t)b * p.R + pr.slot0 + j) * (2 * p.NT) + 2 * tl.nt + chalf] =
+                        GREEDY ? make_float2(am.m, __int_as_float(am.idx)) : make_float2(on.m, on.s);
+                }
             }
         }
         if (!ok && lane == 0) { s_abort = 1; atomicExch(p.abort_flag, 1); }
@@ -332,25 +379,65 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tm_h0, const __grid_const
     }
 }
 
-// Merges the per-tile statistics of every valid row of sequence blockIdx.x, stores the row
-// statistics and runs the accept / first-rejection scan (Algorithm 6, for-loop).
+// One CTA per (sequence, row): merges the row's per-tile statistics and stores the row statistics;
+// the CTA that completes a sequence (arrival counter) runs the accept / first-rejection scan
+// (Algorithm 6, for-loop).
 template <bool GREEDY>
 __global__ void __launch_bounds__(kThreads) lmhead_finalize_kernel(const VerifyParams p, const float2* lm_partial,
                                                                    const int NT) {
-    __shared__ float2 s_stats[2 * BS_MAX_GAMMA + 1];
-    const int b = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    __shared__ float2 s_w[kWarps];
+    const int b = blockIdx.x / p.R, lr = blockIdx.x - b * p.R;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = clamp_gamma(p.gamma[b], p.Gmax);
     const int rows_b = GREEDY ? g + 1 : 2 * g + 1;
-    for (int lr = warp; lr < rows_b; lr += kWarps) {
-        const int r = row_slot(lr, g, p.Gmax);
-        const float2 st = merge_row_partials<GREEDY>(lm_partial + ((size_t)b * p.R + r) * NT, NT, p.c);
-        if (lane == 0) {
-            s_stats[r] = st;
-            p.row_stats[(size_t)b * p.R + r] = st;
+    if (lr >= rows_b) return;
+    const int r = row_slot(lr, g, p.Gmax);
+    const float2* pp = lm_partial + ((size_t)b * p.R + r) * NT;
+    float2 wr;
+    if (GREEDY) {
+        ArgMax a{-INFINITY, INT_MAX};
+        for (int q = tid; q < NT; q += kThreads) {
+            const float2 v = __ldcg(pp + q);
+            a = better(a, ArgMax{v.x, __float_as_int(v.y)});
         }
+        a = warp_best(a);
+        wr = make_float2(a.m, __int_as_float(a.idx));
+    } else {
+        Online o{-INFINITY, 0.f};
+        for (int q = tid; q < NT; q += kThreads) {
+            const float2 v = __ldcg(pp + q);
+            o.merge(v.x, v.y, p.c);
+        }
+        wr = warp_merge(o, p.c);
     }
+    if (lane == 0) s_w[warp] = wr;
     __syncthreads();
-    if (warp == 0) accept_scan_warp<float, GREEDY>(p, b, [&](int rr) { return s_stats[rr]; });
+    if (warp != 0) return;
+    float2 st;
+    if (GREEDY) {
+        ArgMax a{-INFINITY, INT_MAX};
+        if (lane < kWarps) a = ArgMax{s_w[lane].x, __float_as_int(s_w[lane].y)};
+        a = warp_best(a);
+        if (a.idx == INT_MAX) a.idx = 0;                      // row of -inf / NaN only
+        st = make_float2(a.m, __int_as_float(a.idx));
+    } else {
+        Online o{-INFINITY, 0.f};
+        if (lane < kWarps) { o.m = s_w[lane].x; o.s = s_w[lane].y; }
+        st = warp_merge(o, p.c);
+    }
+    unsigned old = 0;
+    if (lane == 0) {
+        p.row_stats[(size_t)b * p.R + r] = st;
+        __threadfence();
+        old = atomicAdd(p.ticket + b, 1u);
+    }
+    old = __shfl_sync(0xffffffffu, old, 0);
+    if (old + 1u == (unsigned)rows_b) {
+        __threadfence();
+        const float2* rsb = p.row_stats + (size_t)b * p.R;
+        accept_scan_warp<float, GREEDY>(p, b, [rsb](int rr) { return __ldcg(rsb + rr); });
+        if (lane == 0) p.ticket[b] = 0u;                      // leave the counter clear for the next call
+    }
 }
 
 // ---- host side ------------------------------------------------------------------------------
@@ -388,34 +475,37 @@ static bool make_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t 
 }
 
 constexpr int kLmBN = 256;
-constexpr int kLmStages = 4;
-constexpr size_t kLmSmem = (size_t)kLmStages * (kLmABytes + (kLmBN / 64) * kLmChunkBytes) + 1024;
-
-static size_t lm_partial_bytes(int B, int Gmax, int V) {
-    return align_up(sizeof(float2) * (size_t)B * (2 * Gmax + 1) * div_up(V, kLmBN), 256);
+constexpr size_t lm_smem_bytes(int mh, int stages) {
+    return (size_t)stages * (mh * kLmABytes + (kLmBN / 64) * kLmChunkBytes) + 1024;
 }
 
-static bool g_lm_attr[2][64];
+static size_t lm_partial_bytes(int B, int Gmax, int V) {
+    return align_up(sizeof(float2) * (size_t)B * (2 * Gmax + 1) * 2 * div_up(V, kLmBN), 256);
+}
 
-template <bool GREEDY>
+static bool g_lm_attr[4][64];
+
+template <int MH, int STAGES, bool GREEDY>
 static bs_status launch_lmhead(const CUtensorMap* tms, const LmParams& lp, const VerifyParams& vp,
                                const float2* partial, cudaStream_t st) {
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64) dev = 0;
-    auto kern = lmhead_gemm_kernel<kLmBN, kLmStages, GREEDY>;
-    if (!g_lm_attr[GREEDY ? 1 : 0][dev]) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLmSmem) != cudaSuccess)
+    auto kern = lmhead_gemm_kernel<kLmBN, MH, STAGES, GREEDY>;
+    constexpr size_t smem = lm_smem_bytes(MH, STAGES);
+    const int variant = (MH - 1) * 2 + (GREEDY ? 1 : 0);
+    if (!g_lm_attr[variant][dev]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
             return cuda_status(cudaGetLastError());
-        g_lm_attr[GREEDY ? 1 : 0][dev] = true;
+        g_lm_attr[variant][dev] = true;
     }
     const int tiles = lp.prod[0].MT * lp.NT + (lp.nprod > 1 ? lp.prod[1].MT * lp.NT : 0);
     int grid = sm_count();
     if (grid > tiles) grid = tiles;
-    kern<<<grid, kLmThreads, kLmSmem, st>>>(tms[0], tms[1], tms[2], tms[3], lp);
+    kern<<<grid, kLmThreads, smem, st>>>(tms[0], tms[1], tms[2], tms[3], lp);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_status(e);
-    lmhead_finalize_kernel<GREEDY><<<vp.B, kThreads, 0, st>>>(vp, partial, lp.NT);
+    lmhead_finalize_kernel<GREEDY><<<vp.B * vp.R, kThreads, 0, st>>>(vp, partial, 2 * lp.NT);
     return cuda_status(cudaGetLastError());
 }
 
@@ -464,9 +554,10 @@ extern "C" bs_status bs_lmhead_verify(const void* H_t, const void* W_t, int d_t,
     lp.partial = partial;
     lp.abort_flag = reinterpret_cast<int32_t*>(ws + w.off_abort);
     const int Mt = B * (Gmax + 1), Md = B * Gmax;
-    lp.prod[0] = LmProduct{logits_t_out, Mt, div_up(d_t, kLmBK), div_up(Mt, kLmBM), Gmax + 1, 0};
+    const int mh = Mt > kLmBM ? 2 : 1;                 // 256-row tiles once there is more than one row tile
+    lp.prod[0] = LmProduct{logits_t_out, Mt, div_up(d_t, kLmBK), div_up(Mt, kLmBM * mh), Gmax + 1, 0};
     lp.prod[1] = LmProduct{logits_d_out, need_draft ? Md : 0, need_draft ? div_up(d_d, kLmBK) : 0,
-                           need_draft ? div_up(Md, kLmBM) : 0, Gmax > 0 ? Gmax : 1, Gmax + 1};
+                           need_draft ? div_up(Md, kLmBM * mh) : 0, Gmax > 0 ? Gmax : 1, Gmax + 1};
 
     CUtensorMap tms[4];
     if (!make_map(&tms[0], H_t, (uint64_t)Mt, (uint64_t)d_t, kLmBM) || !make_map(&tms[1], W_t, (uint64_t)d_t, (uint64_t)V, kLmBK))
@@ -492,5 +583,8 @@ extern "C" bs_status bs_lmhead_verify(const void* H_t, const void* W_t, int d_t,
     vp.seg = seg_elems(BS_F32); vp.nseg = div_up(V, vp.seg);
     vp.c = lp.c;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    return greedy ? launch_lmhead<true>(tms, lp, vp, partial, st) : launch_lmhead<false>(tms, lp, vp, partial, st);
+    if (mh == 1)
+        return greedy ? launch_lmhead<1, 4, true>(tms, lp, vp, partial, st)
+                      : launch_lmhead<1, 4, false>(tms, lp, vp, partial, st);
+    return greedy ? launch_lmhead<2, 3, true>(tms, lp, vp, partial, st) : launch_lmhead<2, 3, false>(tms, lp, vp, partial, st);
 }
