@@ -13,11 +13,15 @@
 //                      loads, update a per-thread online softmax state (chunk max first, then
 //                      ONE exp per logit), release the slot through an "empty" mbarrier.
 //
+//   warp 17            finisher: takes the row pieces the consumers finish (a small ring of
+//                      per-warp results in shared memory), merges them, publishes the piece and
+//                      does what the piece completes, so the consumers never leave the stream.
+//
 // The per-thread state lives across all segments of a row piece; it is reduced only when the
-// row (or the CTA's range) ends.  Row partials are merged by whichever warp completes the row
-// (atomic ticket per row), and the accept scan of a sequence is run by whichever warp completes
-// its last row (atomic ticket per sequence).  Nobody waits on another CTA.  All waits on
-// mbarriers are bounded; a wait that gives up sets the abort word and the thread leaves.
+// row (or the CTA's range) ends.  Row partials are merged by whichever finisher completes the row
+// (atomic ticket per row), and the accept scan of a sequence is run by whichever finisher
+// completes its last row (atomic ticket per sequence).  Nobody waits on another CTA.  All waits
+// on mbarriers are bounded; a wait that gives up sets the abort word and the thread leaves.
 #include "bs_verify_common.cuh"
 #include "bs_pipeline.cuh"
 
@@ -25,11 +29,11 @@ namespace bs {
 
 constexpr int kConsumerWarps = 16;
 constexpr int kConsumers = kConsumerWarps * 32;
-constexpr int kStreamThreads = kConsumers + 32;
+constexpr int kStreamThreads = kConsumers + 64;                   // + producer warp + finisher warp
 constexpr int kVecPerStage = kSegBytes / 16;                     // 2048
 constexpr int kVecPerThread = kVecPerStage / kConsumers;         // 4
 constexpr int kMaxStages = 3;
-constexpr int kRedSlots = 8;                                     // > kMaxStages + 1 row-piece ends in flight
+constexpr int kRedSlots = 8;                                     // row-piece results the consumers may run ahead of the finisher
 static_assert(kVecPerThread * kConsumers == kVecPerStage, "stage must divide evenly over the consumers");
 
 // Per-stage record written by the producer: w0 = nvec | flags << 16, w1 = b | lr << 13 | sg << 19
@@ -37,11 +41,16 @@ static_assert(kVecPerThread * kConsumers == kVecPerStage, "stage must divide eve
 struct StageMeta {
     int w0, w1;
 };
+// Per finished row piece, written by consumer warp 0: w1 of the piece's last stage; first segment
+// of the piece in the low half, bit 16 set on the CTA's last piece.
+struct PieceMeta {
+    int w1, first_sg;
+};
 static_assert(BS_MAX_BATCH <= (1 << 13) && 2 * BS_MAX_GAMMA + 1 < (1 << 6) &&
               BS_MAX_VOCAB / (kSegBytes / 4) <= (1 << 8), "StageMeta packing");
 
 template <typename T, bool GREEDY>
-__global__ void __launch_bounds__(kStreamThreads) verify_stream_kernel(const VerifyParams p, const int nstages) {
+__global__ void __launch_bounds__(kStreamThreads, 2) verify_stream_kernel(const VerifyParams p, const int nstages) {
     extern __shared__ __align__(128) unsigned char smem[];
     // layout: [nstages * 32 KB ring][prefix (B+1) ints]
     unsigned char* ring = smem;
@@ -51,9 +60,11 @@ __global__ void __launch_bounds__(kStreamThreads) verify_stream_kernel(const Ver
     // one reduction barrier per s_red slot: a warp may run several row pieces ahead of another,
     // so arrivals of different pieces must never meet on one barrier
     __shared__ __align__(8) unsigned long long s_redbar[kRedSlots];
+    __shared__ __align__(8) unsigned long long s_redfree[kRedSlots];
+    __shared__ PieceMeta s_piece[kRedSlots];
     __shared__ __align__(8) StageMeta s_meta[kMaxStages];
     __shared__ float2 s_red[kRedSlots][kConsumerWarps];
-    __shared__ int s_scan[kConsumerWarps + 1];
+    __shared__ int s_scan[kStreamThreads / 32];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int kVec = Elem<T>::kVec;
@@ -63,7 +74,10 @@ __global__ void __launch_bounds__(kStreamThreads) verify_stream_kernel(const Ver
             mbar_init(smem_u32(&s_full[s]), 1);
             mbar_init(smem_u32(&s_empty[s]), kConsumerWarps);
         }
-        for (int s = 0; s < kRedSlots; ++s) mbar_init(smem_u32(&s_redbar[s]), kConsumerWarps);
+        for (int s = 0; s < kRedSlots; ++s) {
+            mbar_init(smem_u32(&s_redbar[s]), kConsumerWarps);
+            mbar_init(smem_u32(&s_redfree[s]), 1);
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
 
@@ -157,6 +171,79 @@ __global__ void __launch_bounds__(kStreamThreads) verify_stream_kernel(const Ver
         return;
     }
 
+    if (warp == kConsumerWarps + 1) {
+        // =============================== finisher ===============================
+        // Takes the row pieces the consumers finish, in order: merges the 16 warp results,
+        // publishes the piece, and does whatever the piece completes (row merge, accept scan).
+        // The consumers never wait for any of this.
+        for (int pc = 0;; ++pc) {
+            const int rs = pc % kRedSlots;
+            if (!mbar_wait_warp(smem_u32(&s_redbar[rs]), (uint32_t)(pc / kRedSlots) & 1u)) {
+                if (lane == 0) atomicExch(p.abort_flag, 1);
+                return;
+            }
+            const PieceMeta pm = s_piece[rs];
+            float2 mine = make_float2(-INFINITY, GREEDY ? __int_as_float(INT_MAX) : 0.f);
+            if (lane < kConsumerWarps) mine = s_red[rs][lane];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&s_redfree[rs]));   // the slot may be reused
+            float2 out;
+            if (GREEDY) {
+                ArgMax a = warp_best(ArgMax{mine.x, __float_as_int(mine.y)});
+                out = make_float2(a.m, __int_as_float(a.idx));
+            } else {
+                out = warp_merge(Online{mine.x, mine.y}, p.c);
+            }
+            // ---- publish; whoever completes a row / a sequence does the follow-up ----
+            const int m_b = pm.w1 & 0x1fff, m_lr = (pm.w1 >> 13) & 0x3f, m_sg = (pm.w1 >> 19) & 0xff;
+            const int first_sg = pm.first_sg & 0xffff;
+            const int gb = clamp_gamma(p.gamma[m_b], p.Gmax);
+            const int r = row_slot(m_lr, gb, p.Gmax);
+            const int piece_len = m_sg - first_sg + 1;
+            bool row_done;
+            if (piece_len == p.nseg) {                        // the whole row was ours
+                if (GREEDY && __float_as_int(out.y) == INT_MAX) out.y = __int_as_float(0);
+                if (lane == 0) p.row_stats[(size_t)m_b * p.R + r] = out;
+                row_done = true;
+            } else {
+                float2* pp = p.partial + ((size_t)m_b * p.R + r) * p.S;
+                // slot of the piece's first segment carries the result, the rest are neutral
+                for (int q = first_sg + lane; q <= m_sg; q += 32)
+                    pp[q] = (q == first_sg) ? out : make_float2(-INFINITY, GREEDY ? __int_as_float(INT_MAX) : 0.f);
+                __threadfence();
+                __syncwarp();
+                unsigned old = 0;
+                if (lane == 0) old = atomicAdd(p.ticket_row + (size_t)m_b * p.R + r, (unsigned)piece_len);
+                old = __shfl_sync(0xffffffffu, old, 0);
+                row_done = (old + (unsigned)piece_len == (unsigned)p.nseg);
+                if (row_done) {
+                    __threadfence();
+                    const float2 st = merge_row_partials<GREEDY>(pp, p.nseg, p.c);
+                    if (lane == 0) {
+                        p.row_stats[(size_t)m_b * p.R + r] = st;
+                        p.ticket_row[(size_t)m_b * p.R + r] = 0u;
+                    }
+                }
+            }
+            if (row_done) {
+                __threadfence();
+                __syncwarp();
+                const int rows_mb = GREEDY ? gb + 1 : 2 * gb + 1;
+                unsigned old = 0;
+                if (lane == 0) old = atomicAdd(p.ticket + m_b, 1u);
+                old = __shfl_sync(0xffffffffu, old, 0);
+                if (old + 1u == (unsigned)rows_mb) {
+                    __threadfence();
+                    const float2* rsb = p.row_stats + (size_t)m_b * p.R;
+                    accept_scan_warp<T, GREEDY>(p, m_b, [rsb](int rr) { return __ldcg(rsb + rr); });
+                    if (lane == 0) p.ticket[m_b] = 0u;
+                }
+            }
+            if (pm.first_sg >> 16) break;                     // that was the CTA's last piece
+        }
+        return;
+    }
+
     // ================================= consumers =================================
     Online on{-INFINITY, 0.f};
     ArgMax am{-INFINITY, INT_MAX};
@@ -187,76 +274,21 @@ __global__ void __launch_bounds__(kStreamThreads) verify_stream_kernel(const Ver
         if (++slot == nstages) { slot = 0; ph ^= 1u; }
 
         if (flags & 2) {
-            // ---- end of a row piece: reduce over the consumer warps ----
+            // ---- end of a row piece: hand the warp's result to the finisher ----
             float2 wr;
             if (GREEDY) { am = warp_best(am); wr = make_float2(am.m, __int_as_float(am.idx)); }
             else wr = warp_merge(on, p.c);
             const int rs = pc % kRedSlots;
+            // the finisher must have taken the piece that used this slot kRedSlots pieces ago
+            if (pc >= kRedSlots &&
+                !mbar_wait_warp(smem_u32(&s_redfree[rs]), (uint32_t)(pc / kRedSlots - 1) & 1u)) {
+                atomicExch(p.abort_flag, 1);
+                return;
+            }
             if (lane == 0) {
                 s_red[rs][warp] = wr;
-                mbar_arrive(smem_u32(&s_redbar[rs]));         // release: the write above is visible to warp 0
-            }
-            if (warp == 0) {
-                if (!mbar_wait_warp(smem_u32(&s_redbar[rs]), (uint32_t)(pc / kRedSlots) & 1u)) {
-                    atomicExch(p.abort_flag, 1);
-                    return;
-                }
-                float2 out;
-                if (GREEDY) {
-                    ArgMax a{-INFINITY, INT_MAX};
-                    if (lane < kConsumerWarps) { const float2 t = s_red[rs][lane]; a = ArgMax{t.x, __float_as_int(t.y)}; }
-                    a = warp_best(a);
-                    out = make_float2(a.m, __int_as_float(a.idx));
-                } else {
-                    Online o{-INFINITY, 0.f};
-                    if (lane < kConsumerWarps) { const float2 t = s_red[rs][lane]; o.m = t.x; o.s = t.y; }
-                    out = warp_merge(o, p.c);
-                }
-                // ---- publish; the warp that completes a row / a sequence does the follow-up ----
-                const int m_b = m.w1 & 0x1fff, m_lr = (m.w1 >> 13) & 0x3f;
-                const int gb = clamp_gamma(p.gamma[m_b], p.Gmax);
-                const int r = row_slot(m_lr, gb, p.Gmax);
-                const int piece_len = m_sg - piece_first_sg + 1;
-                bool row_done;
-                if (piece_len == p.nseg) {                    // the whole row was ours
-                    if (GREEDY && __float_as_int(out.y) == INT_MAX) out.y = __int_as_float(0);
-                    if (lane == 0) p.row_stats[(size_t)m_b * p.R + r] = out;
-                    row_done = true;
-                } else {
-                    float2* pp = p.partial + ((size_t)m_b * p.R + r) * p.S;
-                    // slot of the piece's first segment carries the result, the rest are neutral
-                    for (int q = piece_first_sg + lane; q <= m_sg; q += 32)
-                        pp[q] = (q == piece_first_sg) ? out
-                                                      : make_float2(-INFINITY, GREEDY ? __int_as_float(INT_MAX) : 0.f);
-                    __threadfence();
-                    __syncwarp();
-                    unsigned old = 0;
-                    if (lane == 0) old = atomicAdd(p.ticket_row + (size_t)m_b * p.R + r, (unsigned)piece_len);
-                    old = __shfl_sync(0xffffffffu, old, 0);
-                    row_done = (old + (unsigned)piece_len == (unsigned)p.nseg);
-                    if (row_done) {
-                        __threadfence();
-                        const float2 st = merge_row_partials<GREEDY>(pp, p.nseg, p.c);
-                        if (lane == 0) {
-                            p.row_stats[(size_t)m_b * p.R + r] = st;
-                            p.ticket_row[(size_t)m_b * p.R + r] = 0u;
-                        }
-                    }
-                }
-                if (row_done) {
-                    __threadfence();
-                    __syncwarp();
-                    const int rows_mb = GREEDY ? gb + 1 : 2 * gb + 1;
-                    unsigned old = 0;
-                    if (lane == 0) old = atomicAdd(p.ticket + m_b, 1u);
-                    old = __shfl_sync(0xffffffffu, old, 0);
-                    if (old + 1u == (unsigned)rows_mb) {
-                        __threadfence();
-                        const float2* rsb = p.row_stats + (size_t)m_b * p.R;
-                        accept_scan_warp<T, GREEDY>(p, m_b, [rsb](int rr) { return __ldcg(rsb + rr); });
-                        if (lane == 0) p.ticket[m_b] = 0u;
-                    }
-                }
+                if (warp == 0) s_piece[rs] = PieceMeta{m.w1, piece_first_sg | ((k == count - 1) ? (1 << 16) : 0)};
+                mbar_arrive(smem_u32(&s_redbar[rs]));         // release: the writes above are visible to the finisher
             }
             on = Online{-INFINITY, 0.f};
             am = ArgMax{-INFINITY, INT_MAX};
