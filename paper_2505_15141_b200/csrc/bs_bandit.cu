@@ -62,6 +62,7 @@ __device__ inline double confidence_radius(int L, int K, long long t, long long 
 __global__ void __launch_bounds__(128) bandit_select_kernel(void* state, int alg, int B, int K,
                                                            const float* u_arm, const uint8_t* active,
                                                            int32_t* arm_out, int32_t* gamma_out, double* index_out) {
+    pdl_enter();
     const int b = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (b >= B) return;
@@ -127,6 +128,7 @@ __global__ void __launch_bounds__(128) bandit_select_kernel(void* state, int alg
 
 __global__ void bandit_update_kernel(void* state, int alg, int B, int K, const int32_t* arm,
                                      const int32_t* reward_y, const uint8_t* active) {
+    pdl_enter();
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= B) return;
     if (active && !active[b]) return;
@@ -187,18 +189,17 @@ extern "C" bs_status bs_bandit_select(void* state, size_t state_bytes, bs_alg al
     if (!bandit_args_ok(state, state_bytes, alg, B, K) || !arm || !gamma) return BS_ERR_INVALID_ARG;
     if (alg == BS_EXP3 && !u_arm) return BS_ERR_INVALID_ARG;
     const int warps_per_cta = 4;
-    bandit_select_kernel<<<div_up(B, warps_per_cta), warps_per_cta * 32, 0, static_cast<cudaStream_t>(stream)>>>(
-        state, alg, B, K, u_arm, active, arm, gamma, index_out);
-    return cuda_status(cudaGetLastError());
+    return cuda_status(launch_pdl(bandit_select_kernel, div_up(B, warps_per_cta), warps_per_cta * 32, 0,
+                                  static_cast<cudaStream_t>(stream), state, (int)alg, B, K, u_arm, active, arm, gamma,
+                                  index_out));
 }
 
 extern "C" bs_status bs_bandit_update(void* state, size_t state_bytes, bs_alg alg, int B, int K,
                                       const int32_t* arm, const int32_t* reward_y, const uint8_t* active,
                                       void* stream) {
     if (!bandit_args_ok(state, state_bytes, alg, B, K) || !arm || !reward_y) return BS_ERR_INVALID_ARG;
-    bandit_update_kernel<<<div_up(B, 128), 128, 0, static_cast<cudaStream_t>(stream)>>>(state, alg, B, K, arm,
-                                                                                        reward_y, active);
-    return cuda_status(cudaGetLastError());
+    return cuda_status(launch_pdl(bandit_update_kernel, div_up(B, 128), 128, 0, static_cast<cudaStream_t>(stream),
+                                  state, (int)alg, B, K, arm, reward_y, active));
 }
 
 extern "C" bs_status bs_bandit_read(const void* state, size_t state_bytes, bs_alg alg, int B, int K,

@@ -137,4 +137,33 @@ inline bs_status cuda_status(cudaError_t e) {
 
 int sm_count();            // SMs of the current device (cached per device)
 
+// Programmatic dependent launch.  Every kernel of the library is launched with the attribute that
+// lets it start while the kernel before it on the stream is still draining: its CTAs take SMs as
+// they free up and run whatever does not touch global memory (barrier set-up, tensor-memory
+// allocation); pdl_wait() then holds them until the earlier grid has completed and its writes are
+// visible, and only after that pdl_release() lets the kernel behind this one do the same, so at
+// most two grids overlap.  Without the attribute both calls do nothing.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_enter() { pdl_wait(); pdl_release(); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+#ifdef BS_NO_PDL                                   // build-time switch for A/B timing: plain stream order
+    cfg.numAttrs = 0;
+#endif
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 }  // namespace bs

@@ -195,6 +195,7 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tm_h0, const __grid_const
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = s_tmem_base;
+    pdl_wait();                                               // H may come from the kernel before this one
 
     // Accumulator used by tile number `it` of this CTA for row half `h`.  The MMA issuer and the
     // epilogue warps each count how often an accumulator has been used (`uses`): the parity of
@@ -370,6 +371,7 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tm_h0, const __grid_const
     }
 
     // ---- all roles meet; tensor memory goes back ----
+    pdl_release();                                            // the merge kernel may start taking SMs now
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -386,6 +388,7 @@ template <bool GREEDY>
 __global__ void __launch_bounds__(kThreads) lmhead_finalize_kernel(const VerifyParams p, const float2* lm_partial,
                                                                    const int NT) {
     __shared__ float2 s_w[kWarps];
+    pdl_enter();
     const int b = blockIdx.x / p.R, lr = blockIdx.x - b * p.R;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = clamp_gamma(p.gamma[b], p.Gmax);
@@ -502,11 +505,9 @@ static bs_status launch_lmhead(const CUtensorMap* tms, const LmParams& lp, const
     const int tiles = lp.prod[0].MT * lp.NT + (lp.nprod > 1 ? lp.prod[1].MT * lp.NT : 0);
     int grid = sm_count();
     if (grid > tiles) grid = tiles;
-    kern<<<grid, kLmThreads, smem, st>>>(tms[0], tms[1], tms[2], tms[3], lp);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_pdl(kern, grid, kLmThreads, smem, st, tms[0], tms[1], tms[2], tms[3], lp);
     if (e != cudaSuccess) return cuda_status(e);
-    lmhead_finalize_kernel<GREEDY><<<vp.B * vp.R, kThreads, 0, st>>>(vp, partial, 2 * lp.NT);
-    return cuda_status(cudaGetLastError());
+    return cuda_status(launch_pdl(lmhead_finalize_kernel<GREEDY>, vp.B * vp.R, kThreads, 0, st, vp, partial, 2 * lp.NT));
 }
 
 }  // namespace bs

@@ -138,6 +138,7 @@ __global__ void __launch_bounds__(kThreads, 2) residual_kernel(const ResidParams
     __shared__ int s_lastpos;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    pdl_enter();
     // CTA (b, part) owns a contiguous range of the segments of sequence b
     {
         const int b = blockIdx.x / nsplit, part = blockIdx.x - b * nsplit;
@@ -265,6 +266,7 @@ __global__ void __launch_bounds__(kThreads, 2) residual_kernel(const ResidParams
 
 // Greedy mode: the emitted token is the arg-max of target row tau, already in the row statistics.
 __global__ void greedy_emit_kernel(const ResidParams p) {
+    pdl_enter();
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= p.B) return;
     int g = p.gamma[b];
@@ -283,8 +285,7 @@ static bs_status launch_residual(const ResidParams& p, cudaStream_t st) {
     int nsplit = 2 * sm_count() / p.B;
     if (nsplit > p.nseg) nsplit = p.nseg;
     if (nsplit < 1) nsplit = 1;
-    residual_kernel<T><<<(unsigned)(p.B * nsplit), kThreads, 0, st>>>(p, nsplit);
-    return cuda_status(cudaGetLastError());
+    return cuda_status(launch_pdl(residual_kernel<T>, (unsigned)(p.B * nsplit), kThreads, 0, st, p, nsplit));
 }
 
 }  // namespace bs
@@ -322,8 +323,7 @@ extern "C" bs_status bs_residual_sample(const void* target_logits, const void* d
     p.c = greedy ? 1.f : kLog2e / temperature;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (greedy) {
-        greedy_emit_kernel<<<div_up(B, 128), 128, 0, st>>>(p);
-        return cuda_status(cudaGetLastError());
+        return cuda_status(launch_pdl(greedy_emit_kernel, div_up(B, 128), 128, 0, st, p));
     }
     // rows on 16-byte boundaries: bulk-copy pipeline; otherwise the generic kernel
     const size_t es = dtype == BS_F32 ? 4 : 2;

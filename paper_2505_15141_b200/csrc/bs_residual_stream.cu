@@ -293,6 +293,8 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
 
+    pdl_enter();                                              // accept_len and the row statistics come from the kernel before
+
     // ---- prefix sum of item weights over the batch (all threads, redundantly per CTA) ----
     {
         const int per = div_up(p.B, kRsThreads);
@@ -518,8 +520,7 @@ bs_status launch_residual_stream(const ResidParams& p, cudaStream_t st) {
     const long long items = (long long)p.B * p.nseg;
     if (grid > items) grid = items;
     if (grid < 1) grid = 1;
-    residual_stream_kernel<T><<<(unsigned)grid, kRsThreads, smem, st>>>(p, nst);
-    return cuda_status(cudaGetLastError());
+    return cuda_status(launch_pdl(residual_stream_kernel<T>, (unsigned)grid, kRsThreads, smem, st, p, nst));
 }
 
 template bs_status launch_residual_stream<float>(const ResidParams&, cudaStream_t);

@@ -26,6 +26,7 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const VerifyParams p) 
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int kVec = Elem<T>::kVec;
+    pdl_enter();
 
     // ---- prefix sum of work items over the batch (every CTA, redundantly) ----
     {
@@ -192,8 +193,7 @@ static bs_status launch_verify(const VerifyParams& p, int variant, cudaStream_t 
     long long grid = (long long)sm_count() * g_occ[variant][dev];
     if (grid > upper) grid = upper;
     if (grid < 1) grid = 1;
-    verify_kernel<T, GREEDY><<<(unsigned)grid, kThreads, smem, st>>>(p);
-    return cuda_status(cudaGetLastError());
+    return cuda_status(launch_pdl(verify_kernel<T, GREEDY>, (unsigned)grid, kThreads, smem, st, p));
 }
 
 }  // namespace bs

@@ -81,6 +81,8 @@ __global__ void __launch_bounds__(kStreamThreads, 2) verify_stream_kernel(const 
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
 
+    pdl_enter();                                              // gamma comes from the kernel before this one
+
     // ---- prefix sum of work items over the batch (all threads, redundantly per CTA) ----
     {
         const int per = div_up(p.B, kStreamThreads);
@@ -330,8 +332,7 @@ bs_status launch_verify_stream(const VerifyParams& p, cudaStream_t st) {
     long long grid = 2LL * sm_count();
     if (grid > upper) grid = upper;
     if (grid < 1) grid = 1;
-    verify_stream_kernel<T, GREEDY><<<(unsigned)grid, kStreamThreads, smem, st>>>(p, nst);
-    return cuda_status(cudaGetLastError());
+    return cuda_status(launch_pdl(verify_stream_kernel<T, GREEDY>, (unsigned)grid, kStreamThreads, smem, st, p, nst));
 }
 
 template bs_status launch_verify_stream<float, false>(const VerifyParams&, cudaStream_t);
