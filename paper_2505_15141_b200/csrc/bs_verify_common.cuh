@@ -171,42 +171,62 @@ __device__ __forceinline__ float2 merge_row_partials(const float2* pp, int nseg,
     return warp_merge(o, c);
 }
 
-// Accept test and first-rejection scan for sequence b by one full warp (lane j = drafted position j).
-// stats(r) returns the (max, Z) / (max, arg-max) pair of row slot r.  Writes accept_len, p_tok, q_tok
-// and the status word.
+// Accept test and first-rejection scan for sequence b by one full warp (lane j = drafted position j),
+// in two steps so that a caller can start the loads before it knows whether it will need them.
+//
+// accept_prefetch: everything that does not depend on the row statistics -- the drafted token, the
+// two logits at that token, the uniform.
+struct AcceptLoads {
+    int x;              // drafted token of this lane's position (undefined if the position is not valid)
+    float tl, dl, u;    // target / draft logit at x, uniform
+    int bits;           // BS_DEV_BAD_TOKEN if x is out of range
+};
+template <typename T, bool GREEDY>
+__device__ __forceinline__ AcceptLoads accept_prefetch(const VerifyParams& p, int b, int g) {
+    const int j = threadIdx.x & 31;
+    AcceptLoads a{0, 0.f, 0.f, 2.f, 0};
+    if (j < g) {
+        a.x = p.tokens[(size_t)b * p.Gmax + j];
+        const bool bad = a.x < 0 || a.x >= p.V;
+        if (bad) a.bits = BS_DEV_BAD_TOKEN;
+        if (!GREEDY && !bad) {
+            a.tl = Elem<T>::load(row_ptr(static_cast<const T*>(p.target), b, p.Gmax + 1, j, p.V) + a.x);
+            a.dl = Elem<T>::load(row_ptr(static_cast<const T*>(p.draft), b, p.Gmax, j, p.V) + a.x);
+            a.u = p.u_accept[(size_t)b * p.Gmax + j];
+        }
+    }
+    return a;
+}
+
+// accept_finish: stats(r) returns the (max, Z) / (max, arg-max) pair of row slot r.  Writes
+// accept_len, p_tok, q_tok and the status word.  graw = gamma[b] as read, g = clamp_gamma(graw).
 template <typename T, bool GREEDY, typename StatsFn>
-__device__ __forceinline__ void accept_scan_warp(const VerifyParams& p, int b, StatsFn stats) {
+__device__ __forceinline__ void accept_finish(const VerifyParams& p, int b, int graw, int g, const AcceptLoads& a,
+                                              StatsFn stats) {
     const int lane = threadIdx.x & 31;
-    const int graw = p.gamma[b];
-    const int g = clamp_gamma(graw, p.Gmax);
     const int j = lane;
     const bool valid = j < g;
-    int st_bits = (graw != g) ? BS_DEV_BAD_GAMMA : 0;
+    int st_bits = ((graw != g) ? BS_DEV_BAD_GAMMA : 0) | a.bits;
     bool acc = false;
     float pj = 0.f, qj = 0.f;
     if (valid) {
-        const int x = p.tokens[(size_t)b * p.Gmax + j];
-        const bool bad = x < 0 || x >= p.V;
-        if (bad) st_bits |= BS_DEV_BAD_TOKEN;
+        const bool bad = a.bits != 0;
         const float2 ts = stats(j);
         if (GREEDY) {
-            acc = !bad && x == __float_as_int(ts.y);
+            acc = !bad && a.x == __float_as_int(ts.y);
         } else {
             const float2 ds = stats(p.Gmax + 1 + j);
             if (!(ts.y > 0.f) || !(ds.y > 0.f) || !isfinite(ts.y) || !isfinite(ds.y) || !isfinite(ts.x) ||
                 !isfinite(ds.x))
                 st_bits |= BS_DEV_NONFINITE;
             if (!bad) {
-                const float tl = Elem<T>::load(row_ptr(static_cast<const T*>(p.target), b, p.Gmax + 1, j, p.V) + x);
-                const float dl = Elem<T>::load(row_ptr(static_cast<const T*>(p.draft), b, p.Gmax, j, p.V) + x);
                 // log2 of the two probabilities; the ratio is formed in the log domain
-                const float lp = (tl - ts.x) * p.c - log2f(ts.y);
-                const float lq = (dl - ds.x) * p.c - log2f(ds.y);
+                const float lp = (a.tl - ts.x) * p.c - log2f(ts.y);
+                const float lq = (a.dl - ds.x) * p.c - log2f(ds.y);
                 pj = exp2f(lp);
                 qj = exp2f(lq);
-                const float u = p.u_accept[(size_t)b * p.Gmax + j];
                 // r <= min{1, P/Q}; Q(x) = 0 counts as an infinite ratio
-                acc = (lq == -INFINITY) ? true : (u <= fminf(1.f, exp2f(lp - lq)));
+                acc = (lq == -INFINITY) ? true : (a.u <= fminf(1.f, exp2f(lp - lq)));
             }
         }
     }
@@ -228,6 +248,14 @@ __device__ __forceinline__ void accept_scan_warp(const VerifyParams& p, int b, S
         p.accept_len[b] = tau;
         p.status[b] = st_bits;
     }
+}
+
+template <typename T, bool GREEDY, typename StatsFn>
+__device__ __forceinline__ void accept_scan_warp(const VerifyParams& p, int b, StatsFn stats) {
+    const int graw = p.gamma[b];
+    const int g = clamp_gamma(graw, p.Gmax);
+    const AcceptLoads a = accept_prefetch<T, GREEDY>(p, b, g);
+    accept_finish<T, GREEDY>(p, b, graw, g, a, stats);
 }
 
 template <typename T, bool GREEDY>

@@ -18,9 +18,9 @@
 //                      does what the piece completes, so the consumers never leave the stream.
 //
 // The per-thread state lives across all segments of a row piece; it is reduced only when the
-// row (or the CTA's range) ends.  Row partials are merged by whichever finisher completes the row
-// (atomic ticket per row), and the accept scan of a sequence is run by whichever finisher
-// completes its last row (atomic ticket per sequence).  Nobody waits on another CTA.  All waits
+// row (or the CTA's range) ends.  Every piece is published as a partial and counted on one atomic
+// ticket per sequence; the finisher whose piece completes the count merges all rows of the
+// sequence (one lane per row) and runs the accept scan.  Nobody waits on another CTA.  All waits
 // on mbarriers are bounded; a wait that gives up sets the abort word and the thread leaves.
 #include "bs_verify_common.cuh"
 #include "bs_pipeline.cuh"
@@ -62,6 +62,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) verify_stream_kernel(const 
     __shared__ __align__(8) unsigned long long s_redbar[kRedSlots];
     __shared__ __align__(8) unsigned long long s_redfree[kRedSlots];
     __shared__ PieceMeta s_piece[kRedSlots];
+    __shared__ float2 s_fin[2 * BS_MAX_GAMMA + 1];            // merged row statistics of the sequence being finished
     __shared__ __align__(8) StageMeta s_meta[kMaxStages];
     __shared__ float2 s_red[kRedSlots][kConsumerWarps];
     __shared__ int s_scan[kStreamThreads / 32];
@@ -196,50 +197,62 @@ __global__ void __launch_bounds__(kStreamThreads, 2) verify_stream_kernel(const 
             } else {
                 out = warp_merge(Online{mine.x, mine.y}, p.c);
             }
-            // ---- publish; whoever completes a row / a sequence does the follow-up ----
+            // ---- publish the piece; the finisher that completes the sequence does the rest ----
             const int m_b = pm.w1 & 0x1fff, m_lr = (pm.w1 >> 13) & 0x3f, m_sg = (pm.w1 >> 19) & 0xff;
             const int first_sg = pm.first_sg & 0xffff;
-            const int gb = clamp_gamma(p.gamma[m_b], p.Gmax);
+            const int graw = p.gamma[m_b];
+            const int gb = clamp_gamma(graw, p.Gmax);
             const int r = row_slot(m_lr, gb, p.Gmax);
             const int piece_len = m_sg - first_sg + 1;
-            bool row_done;
-            if (piece_len == p.nseg) {                        // the whole row was ours
-                if (GREEDY && __float_as_int(out.y) == INT_MAX) out.y = __int_as_float(0);
-                if (lane == 0) p.row_stats[(size_t)m_b * p.R + r] = out;
-                row_done = true;
-            } else {
+            const int rows_mb = GREEDY ? gb + 1 : 2 * gb + 1;
+            {
                 float2* pp = p.partial + ((size_t)m_b * p.R + r) * p.S;
                 // slot of the piece's first segment carries the result, the rest are neutral
                 for (int q = first_sg + lane; q <= m_sg; q += 32)
                     pp[q] = (q == first_sg) ? out : make_float2(-INFINITY, GREEDY ? __int_as_float(INT_MAX) : 0.f);
+            }
+            // the loads of the accept test do not depend on the statistics: start them now, so
+            // that they travel while the arrival counter does
+            const AcceptLoads al = accept_prefetch<T, GREEDY>(p, m_b, gb);
+            __threadfence();
+            __syncwarp();
+            unsigned old = 0;
+            if (lane == 0) old = atomicAdd(p.ticket + m_b, (unsigned)piece_len);
+            old = __shfl_sync(0xffffffffu, old, 0);
+            if (old + (unsigned)piece_len == (unsigned)(rows_mb * p.nseg)) {
+                // ---- last piece of the sequence: merge every row (one lane per row), accept scan ----
                 __threadfence();
-                __syncwarp();
-                unsigned old = 0;
-                if (lane == 0) old = atomicAdd(p.ticket_row + (size_t)m_b * p.R + r, (unsigned)piece_len);
-                old = __shfl_sync(0xffffffffu, old, 0);
-                row_done = (old + (unsigned)piece_len == (unsigned)p.nseg);
-                if (row_done) {
-                    __threadfence();
-                    const float2 st = merge_row_partials<GREEDY>(pp, p.nseg, p.c);
-                    if (lane == 0) {
-                        p.row_stats[(size_t)m_b * p.R + r] = st;
-                        p.ticket_row[(size_t)m_b * p.R + r] = 0u;
+                for (int lr0 = 0; lr0 < rows_mb; lr0 += 32) {
+                    const int lr = lr0 + lane;
+                    if (lr < rows_mb) {
+                        const int rr = row_slot(lr, gb, p.Gmax);
+                        const float2* pp = p.partial + ((size_t)m_b * p.R + rr) * p.S;
+                        float2 st;
+                        if (GREEDY) {
+                            ArgMax a{-INFINITY, INT_MAX};
+#pragma unroll 4
+                            for (int q = 0; q < p.nseg; ++q) {
+                                const float2 v = __ldcg(pp + q);
+                                a = better(a, ArgMax{v.x, __float_as_int(v.y)});
+                            }
+                            if (a.idx == INT_MAX) a.idx = 0;      // row of -inf / NaN only
+                            st = make_float2(a.m, __int_as_float(a.idx));
+                        } else {
+                            Online o{-INFINITY, 0.f};
+#pragma unroll 4
+                            for (int q = 0; q < p.nseg; ++q) {
+                                const float2 v = __ldcg(pp + q);
+                                o.merge(v.x, v.y, p.c);
+                            }
+                            st = make_float2(o.m, o.s);
+                        }
+                        s_fin[rr] = st;
+                        p.row_stats[(size_t)m_b * p.R + rr] = st;
                     }
                 }
-            }
-            if (row_done) {
-                __threadfence();
                 __syncwarp();
-                const int rows_mb = GREEDY ? gb + 1 : 2 * gb + 1;
-                unsigned old = 0;
-                if (lane == 0) old = atomicAdd(p.ticket + m_b, 1u);
-                old = __shfl_sync(0xffffffffu, old, 0);
-                if (old + 1u == (unsigned)rows_mb) {
-                    __threadfence();
-                    const float2* rsb = p.row_stats + (size_t)m_b * p.R;
-                    accept_scan_warp<T, GREEDY>(p, m_b, [rsb](int rr) { return __ldcg(rsb + rr); });
-                    if (lane == 0) p.ticket[m_b] = 0u;
-                }
+                accept_finish<T, GREEDY>(p, m_b, graw, gb, al, [&](int rr) { return s_fin[rr]; });
+                if (lane == 0) p.ticket[m_b] = 0u;                // leave the counter clear for the next call
             }
             if (pm.first_sg >> 16) break;                     // that was the CTA's last piece
         }
