@@ -23,6 +23,13 @@ from oracle import verify as ov
 from paper_2505_15141_b200 import workloads as wl
 
 P_TOL = 1e-5
+# EXP3Spec's cumulative loss estimates, fp64 on both sides.  The two exp() routines differ in the
+# last bit, and a difference d in S_i moves p_i by about eta * d * p_i, hence the next estimate
+# (L+1-y)/(L p_i) by eta * d relative: every pull multiplies the difference by about
+# 1 + eta * Z (measured: 1e-16 grows to 9e-7 over 1000 rounds of the 4-armed workload).  So the
+# states are compared over stretches of at most a few hundred rounds, within S_RTOL, and a
+# trajectory that is carried into another stretch restarts the oracle from the CUDA state.
+S_RTOL = 1e-10
 
 
 @dataclass
@@ -33,6 +40,7 @@ class Tally:
     flagged_token: int = 0
     flagged_arm: int = 0
     max_p_err: float = 0.0
+    max_S_rel: float = 0.0
     sum_y: int = 0
 
     def merge(self, o: "Tally") -> None:
@@ -122,7 +130,7 @@ def gpu_round(bs, rnd: wl.RoundInputs, temperature: float, workspace=None):
 
 
 def closed_loop(bs, w: wl.Workload, rounds: int, device, sample: Optional[Sequence[int]] = None,
-                first_round: int = 1, state=None, oracle_bandit=None) -> Tally:
+                first_round: int = 1, state=None, oracle_bandit=None, carry: Optional[dict] = None) -> Tally:
     """select -> make inputs for the chosen arms -> verify -> resample -> update, on the GPU and in
     the oracle side by side.  `sample`: sequences whose verification the oracle replays (default
     all); the oracle bandit of the others is fed the CUDA reward (teacher forcing)."""
@@ -130,9 +138,13 @@ def closed_loop(bs, w: wl.Workload, rounds: int, device, sample: Optional[Sequen
     alg = {None: None, "ucb": bs.BS_UCB, "exp3": bs.BS_EXP3}[w.alg]
     tally = Tally()
     ws = bs.new_workspace(B, G, V, device)
+    if carry is not None and "state" in carry:           # continue a trajectory started by an earlier call
+        state, oracle_bandit = carry["state"], carry["oracle_bandit"]
     if alg is not None and state is None:
         state = bs.new_bandit(alg, B, w.arm_gamma, w.delta, device)
         oracle_bandit = ob.UCBSpec(B, w.arm_gamma, w.delta) if w.alg == "ucb" else ob.EXP3Spec(B, w.arm_gamma)
+    if carry is not None:
+        carry["state"], carry["oracle_bandit"] = state, oracle_bandit
     arm_d = torch.zeros(B, dtype=torch.int32, device=device)
     gamma_d = torch.full((B,), w.arm_gamma[0], dtype=torch.int32, device=device)
     for rnd_i in range(first_round, first_round + rounds):
@@ -175,5 +187,9 @@ def closed_loop(bs, w: wl.Workload, rounds: int, device, sample: Optional[Sequen
         if w.alg == "ucb":
             assert (st["n"] == oracle_bandit.n).all() and (st["sumY"] == oracle_bandit.sumY).all()
         else:
-            assert np.allclose(st["S"], oracle_bandit.S, rtol=1e-9, atol=1e-12)
+            rel = np.abs(st["S"] - oracle_bandit.S) / np.maximum(np.abs(oracle_bandit.S), 1e-12)
+            tally.max_S_rel = max(tally.max_S_rel, float(rel.max()))
+            assert rel.max() <= S_RTOL, f"cumulative losses off by {rel.max()} (relative) after round {oracle_bandit.t.max()}"
+            if carry is not None:
+                oracle_bandit.S[...] = st["S"]
     return tally

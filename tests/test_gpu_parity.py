@@ -250,20 +250,45 @@ def test_closed_loop_llama2_fixed(lib):
     t = parity.closed_loop(lib, w, 40, DEV)
     assert t.sequences == 32 * 40
     assert t.flagged_accept + t.flagged_token <= 0.01 * t.sequences + 2
+    t2 = parity.closed_loop(lib, w, w.rounds - 40, DEV, sample=[0, 9, 18, 31], first_round=41)
+    assert t2.sequences == 4 * (w.rounds - 40) and t2.flagged_accept + t2.flagged_token <= 0.01 * t2.sequences + 2
 
 
 def test_closed_loop_llama3_ucb_full_size(lib):
     """Full-size ragged batch in the launch configuration the benchmark times; the oracle replays
     a sample of sequences each round, the bandits of all sequences are compared every round."""
     w = wl.WORKLOADS["llama3_ucb"]
-    t = parity.closed_loop(lib, w, 24, DEV, sample=[0, 1, 17, 40, 63])
-    assert t.sequences == 5 * 24 and t.flagged_accept + t.flagged_token <= 3
+    carry = {}
+    t = parity.closed_loop(lib, w, 64, DEV, sample=[0, 1, 17, 40, 63], carry=carry)
+    assert t.sequences == 5 * 64 and t.flagged_accept + t.flagged_token <= 5
+    # the remaining rounds of the 500: every sequence's arm against the oracle bandit every round
+    t2 = parity.closed_loop(lib, w, w.rounds - 64, DEV, sample=[], first_round=65, carry=carry)
+    assert t2.flagged_arm <= 2
 
 
 def test_closed_loop_qwen_exp3_full_size(lib):
+    """The first 64 rounds with the oracle replaying three sequences per round, then the bandits alone
+    (every sequence's arm compared every round, the oracle bandit fed the CUDA reward) up to the first
+    change of the arms' draft quality at round 201, and rounds 190-260 across it with the oracle
+    replaying again."""
     w = wl.WORKLOADS["qwen_exp3"]
-    t = parity.closed_loop(lib, w, 12, DEV, sample=[0, 100, 255])
-    assert t.sequences == 3 * 12 and t.flagged_accept + t.flagged_token <= 3
+    carry = {}
+    t = parity.closed_loop(lib, w, 64, DEV, sample=[0, 100, 255], carry=carry)
+    assert t.sequences == 3 * 64 and t.flagged_accept + t.flagged_token <= 5
+    t2 = parity.closed_loop(lib, w, 125, DEV, sample=[], first_round=65, carry=carry)
+    assert t2.sequences == 0 and t2.flagged_arm <= 2
+    t3 = parity.closed_loop(lib, w, 71, DEV, sample=[7, 200], first_round=190, carry=carry)
+    assert t3.sequences == 2 * 71 and t3.flagged_accept + t3.flagged_token <= 4
+    # the rest of the 1000 rounds, bandits only: four more rotations of the arms' draft qualities
+    flagged, worst = t2.flagged_arm, max(t.max_S_rel, t2.max_S_rel, t3.max_S_rel)
+    for first in range(261, w.rounds + 1, 148):
+        t4 = parity.closed_loop(lib, w, min(148, w.rounds + 1 - first), DEV, sample=[], first_round=first, carry=carry)
+        flagged += t4.flagged_arm
+        worst = max(worst, t4.max_S_rel)
+    assert flagged <= 3
+    print("largest relative difference of the cumulative loss estimates over a stretch:", worst)
+    n = lib.bs_bandit_read(carry["state"], lib.BS_EXP3, w.B, w.K)["n"]
+    assert (n.sum(axis=1) == w.rounds).all() and (n.sum(axis=0) > 0).all()
 
 
 def test_full_size_invariants_all_sequences(lib):
