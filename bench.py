@@ -37,9 +37,21 @@ UNIT = "rounds/s"
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_HBM_GBS = 6650.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one verify launch from the ncu captures
-# summarised under profiles/ (bytes per launch; None = not captured for that workload)
-NCU_TRAFFIC = {}
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel,
+# from the ncu captures summarised under profiles/: (read traffic per algorithmic byte, bytes
+# written per launch).  Captured on smaller cases of the same kernels; read traffic grows with the
+# bytes, the writes (workspace partials, write-backs) do not.  None = not captured.
+NCU_TRAFFIC = {
+    "qwen_exp3": (1.0002, 4.1e6),          # profiles/verify_stream_kernel.md, fp32 column
+    "llama3_ucb": (1.0005, 4.1e6),         # profiles/verify_stream_kernel.md, bf16 column
+    "lmhead_llama3": (1.0000, 29.0e6),     # profiles/lmhead_gemm_kernel.md, B=16 (logits still dirty in L2 not counted)
+    "lmhead_llama3_b128": (1.0232, 567.6e6),
+}
+
+
+def ncu_traffic(name: str, algorithmic_read_bytes: float):
+    t = NCU_TRAFFIC.get(name)
+    return None if t is None else t[0] * algorithmic_read_bytes + t[1]
 
 
 def parse_args():
@@ -52,6 +64,9 @@ def parse_args():
                              "lmhead_llama3_b128"])
     ap.add_argument("--batch", type=int, default=0,
                     help="override the workload's batch size (smaller cases for profiler captures)")
+    ap.add_argument("--fixed-gamma", type=int, default=0,
+                    help="replace the workload's arms by one arm of this speculation length, so that the bytes "
+                         "of every launch are known exactly (profiler captures)")
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="budget of the CPU-oracle sample")
@@ -417,7 +432,7 @@ def run_cuda(args, w):
             "algorithmic_gbs": bytes_all / (ms * 1e-3) / 1e9,
             "roofline": {"bound": "hbm", "kernel": "verify_kernel (bs_softmax_verify)", "achieved": achieved,
                          "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": NCU_TRAFFIC.get(w.name), "bytes_per_launch": verify_bytes,
+                         "traffic": ncu_traffic(w.name, verify_bytes), "bytes_per_launch": verify_bytes,
                          "ms_per_launch": verify_ms, "residual_ms_per_launch": resid_ms},
             "e2e": e2e, "cpu_baseline": cpu, "clocks": clocks,
             "gpu_launches": 4 * args.steps,
@@ -585,7 +600,8 @@ def run_lmhead(args, w):
             if hbm_bound else
             {"bound": "tensor", "achieved": tfs, "peak": tc_peak, "unit": "TFLOP/s", "frac": tfs / tc_peak})
     roof.update({"kernel": "lmhead_gemm_kernel (bs_lmhead_verify)", "peak_source": src,
-                 "traffic": NCU_TRAFFIC.get(w.name), "bytes_per_launch": nbytes, "flops_per_launch": flops,
+                 "traffic": ncu_traffic(w.name, 2.0 * w.V * (w.d_t + w.d_d) + 2.0 * w.B * ((w.gamma + 1) * w.d_t + w.gamma * w.d_d)),
+                 "bytes_per_launch": nbytes, "flops_per_launch": flops,
                  "ms_per_launch": lm_ms, "residual_ms_per_launch": res_ms,
                  "hbm_gbs": gbs, "hbm_frac": gbs / hbm_peak, "tensor_tflops": tfs, "tensor_frac": tfs / tc_peak})
 
@@ -665,6 +681,8 @@ def main():
     w = wl.WORKLOADS[args.workload]
     if args.batch:
         w = dataclasses.replace(w, B=args.batch)
+    if args.fixed_gamma:
+        w = dataclasses.replace(w, arm_gamma=(args.fixed_gamma,), alg=None)
     if args.impl == "reference":
         if int(os.environ.get("RANK", "0")) == 0:
             run_reference(args, w)
