@@ -9,6 +9,7 @@ nothing from the product.  Every function follows one passage of the paper:
 * residual Norm([P - Q]_+) and its definitions  -- Algorithm 6 (else-branch) and
                                                    the notation paragraph above it
 * bonus token from P when all drafts pass       -- Algorithm 6, the line after the loop
+* drafted token x~ ~ Q                          -- Algorithm 6, the first line
 * greedy decoding as temperature -> 0           -- Section 2
 * accepted length counts the bonus token, y = tau + 1 in [1, L+1]  -- Section 3
 
@@ -72,6 +73,15 @@ def inverse_cdf(mass: np.ndarray, u: float):
     lo = (c[v - 1] if v > 0 else 0.0) / total
     hi = c[v] / total
     return v, lo, hi
+
+
+def draft_token(draft_row: np.ndarray, u: float, temperature: float):
+    """Drafting step, Algorithm 6, first line: x~ ~ Q(. | pt, x~_{1:j}) with Q = softmax(draft row / T),
+    drawn from ONE uniform by the inverse-CDF reading above; at temperature 0 the arg-max
+    (Section 2).  Returns (token, lo, hi) with the token's CDF interval (0, 1 in greedy mode)."""
+    if temperature == 0.0:
+        return argmax_lowest(draft_row), 0.0, 1.0
+    return inverse_cdf(softmax_row(draft_row, temperature), u)
 
 
 @dataclass

@@ -234,3 +234,25 @@ def test_greedy_is_the_small_temperature_limit():
         s = ov.verify_sequence(tl, dl, toks, gamma, rng.random(gamma), rng.random(), 1e-3)
         agree += (g.out_tokens == s.out_tokens)
     assert agree >= 97
+
+
+def test_draft_token_partitions_the_unit_interval_like_q():
+    """x~ ~ Q by inverse CDF: the set of uniforms that map to token v is an interval of length Q(v),
+    so on an equally spaced grid of N uniforms every token's count is within 1 of N * Q(v); tokens
+    of zero mass never appear; temperature 0 gives the lowest arg-max."""
+    rng = np.random.default_rng(5)
+    row = rng.normal(0, 2, size=13)
+    row[4] = -np.inf                                   # a token of zero mass
+    for T in (1.0, 0.5):
+        q = np.exp(row / T - np.max(row / T)); q /= q.sum()
+        N = 200000
+        us = (np.arange(N) + 0.5) / N
+        toks = np.array([ov.draft_token(row, u, T)[0] for u in us[::40]])        # spot check of the call itself
+        c = np.cumsum(q)
+        assert (toks == np.searchsorted(c, us[::40], side="right")).all()
+        counts = np.bincount(np.searchsorted(c, us, side="right"), minlength=13)
+        assert np.abs(counts - N * q).max() <= 1.0 + 1e-9 and counts[4] == 0
+        v, lo, hi = ov.draft_token(row, 0.37, T)
+        assert lo <= 0.37 < hi and abs((hi - lo) - q[v]) < 1e-12
+    tie = np.array([1.0, 3.0, 3.0, -2.0])
+    assert ov.draft_token(tie, 0.9, 0.0)[0] == 1
