@@ -60,6 +60,8 @@ typedef enum { BS_UCB = 0, BS_EXP3 = 1 } bs_alg;
 #define BS_DEV_BAD_TOKEN   2   /* a drafted token outside [0, V); that position counts as rejected */
 #define BS_DEV_NONFINITE   4   /* a softmax normaliser or residual mass was NaN / Inf / 0 */
 #define BS_DEV_RESIDUAL_FALLBACK 8 /* [P-Q]_+ had zero mass at the rejected position; sampled from P instead */
+#define BS_DEV_DRAFT_MISSING 16    /* bs_softmax_verify_drafted: a draft row below gamma_b was not produced by
+                                      bs_draft_sample on this workspace; every draft of the sequence was rejected */
 
 /* Limits of this implementation. */
 #define BS_MAX_GAMMA   31      /* Gmax <= 31 (one warp scans the accept flags) */
@@ -158,6 +160,43 @@ bs_status bs_softmax_verify_noalloc(const void* target_logits, const void* draft
                                     const int32_t* draft_tokens, const int32_t* gamma, const float* u_accept,
                                     float temperature, int B, int Gmax, int V,
                                     int32_t* accept_len, float* p_tok, float* q_tok, void* stream);
+
+/* ---- drafting on the device (Algorithm 6, first line: x~_{j+1} ~ Q(. | pt, x~_{1:j})) ------------ */
+
+/* Draws the drafted token of ONE position for every sequence that drafts it (position < gamma_b):
+ * a categorical sample from softmax(draft row `position` / temperature) by inverse CDF in
+ * vocabulary order with the uniform u_draft[b, position] (the smallest v whose cumulative mass
+ * strictly exceeds u * total); at temperature 0 the arg-max of the row (lowest index among
+ * equal maxima).  A draft model produces its rows one position at a time, so this is called once
+ * per position, after the row has been written.
+ *
+ *  draft_logits [B, Gmax, V] dtype: only row `position` of each drafting sequence is read
+ *  position     0 <= position < Gmax
+ *  gamma        [B] int32: this round's speculation lengths
+ *  u_draft      [B, Gmax] fp32 uniforms in (0,1); may be NULL iff temperature == 0
+ *  draft_tokens [B, Gmax] int32: entry [b, position] is written for drafting sequences, others kept
+ *  workspace    the round's verification workspace (bs_workspace_bytes / bs_workspace_init)
+ * Besides the token, the call leaves the row's softmax statistics in the workspace and marks the
+ * position as drafted, which is what bs_softmax_verify_drafted relies on.
+ * Requirement: rows on 16-byte boundaries (V * element size a multiple of 16, base pointer
+ * 16-byte aligned), else BS_ERR_UNSUPPORTED. */
+bs_status bs_draft_sample(const void* draft_logits, bs_dtype dtype, int position, const int32_t* gamma,
+                          const float* u_draft, float temperature, int B, int Gmax, int V,
+                          int32_t* draft_tokens, void* workspace, size_t workspace_bytes, void* stream);
+
+/* bs_softmax_verify for a round whose draft rows 0..gamma_b-1 all went through bs_draft_sample on
+ * the same workspace: same arguments, outputs and arithmetic, but the draft rows are not streamed
+ * again -- their statistics are taken from the workspace and only the logit of each drafted token
+ * is read, so the call reads gamma_b + 1 rows per sequence instead of 2 gamma_b + 1.  A sequence
+ * with an undrafted position below gamma_b gets accept_len = 0 and the status bit
+ * BS_DEV_DRAFT_MISSING.  The drafted marks are consumed: the next round drafts again.
+ * bs_residual_sample follows as after bs_softmax_verify.  Same alignment requirement as
+ * bs_draft_sample. */
+bs_status bs_softmax_verify_drafted(const void* target_logits, const void* draft_logits, bs_dtype dtype,
+                                    const int32_t* draft_tokens, const int32_t* gamma, const float* u_accept,
+                                    float temperature, int B, int Gmax, int V,
+                                    int32_t* accept_len, float* p_tok, float* q_tok,
+                                    void* workspace, size_t workspace_bytes, void* stream);
 
 /* ---- fused LM head (Algorithm 6, second line: the models are evaluated on all drafted positions
  *      in parallel; the last step of that evaluation is logits = H W) -------------------------- */

@@ -26,7 +26,7 @@ BS_OK = 0
 BS_ERR_INVALID_ARG, BS_ERR_CUDA, BS_ERR_UNSUPPORTED, BS_ERR_WORKSPACE, BS_ERR_TIMEOUT, BS_ERR_DEVICE_DATA = 1, 2, 3, 4, 5, 6
 BS_F32, BS_BF16 = 0, 1
 BS_UCB, BS_EXP3 = 0, 1
-BS_DEV_BAD_GAMMA, BS_DEV_BAD_TOKEN, BS_DEV_NONFINITE, BS_DEV_RESIDUAL_FALLBACK = 1, 2, 4, 8
+BS_DEV_BAD_GAMMA, BS_DEV_BAD_TOKEN, BS_DEV_NONFINITE, BS_DEV_RESIDUAL_FALLBACK, BS_DEV_DRAFT_MISSING = 1, 2, 4, 8, 16
 BS_MAX_GAMMA, BS_MAX_ARMS, BS_MAX_BATCH = 31, 32, 4096
 
 _vp, _i, _f, _d, _sz = C.c_void_p, C.c_int, C.c_float, C.c_double, C.c_size_t
@@ -41,6 +41,8 @@ SIGNATURES = {
     "bs_softmax_verify": (_i, [_vp, _vp, _i, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bs_residual_sample": (_i, [_vp, _vp, _i, _vp, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _sz, _vp]),
     "bs_softmax_verify_noalloc": (_i, [_vp, _vp, _i, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _vp]),
+    "bs_draft_sample": (_i, [_vp, _i, _i, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _sz, _vp]),
+    "bs_softmax_verify_drafted": (_i, [_vp, _vp, _i, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bs_lmhead_workspace_bytes": (_sz, [_i, _i, _i]),
     "bs_lmhead_verify": (_i, [_vp, _vp, _i, _vp, _vp, _i, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _vp, _vp,
                               _vp, _sz, _vp]),
@@ -182,6 +184,28 @@ def verify_round(target_logits, draft_logits, draft_tokens, gamma, u_accept, u_r
     bs_residual_sample(target_logits, draft_logits, draft_tokens, gamma, accept_len, u_resample,
                        temperature, out_tokens, out_len, workspace)
     return RoundOutput(accept_len, p_tok, q_tok, out_tokens, out_len, workspace)
+
+
+# ---- drafting on the device ------------------------------------------------------------
+
+def bs_draft_sample(draft_logits, position: int, gamma, u_draft, temperature: float, draft_tokens, workspace,
+                    stream=None) -> None:
+    """Drafted token of `position` for every sequence with position < gamma_b, into draft_tokens[b, position]."""
+    B, G, V = draft_logits.shape
+    assert draft_tokens.shape == (B, G) and draft_tokens.dtype == torch.int32
+    _check(_lib.bs_draft_sample(_ptr(draft_logits), _dtype_code(draft_logits), int(position), _ptr(gamma),
+                                _ptr(u_draft), float(temperature), B, G, V, _ptr(draft_tokens),
+                                _ptr(workspace), workspace.numel(), _stream(stream)), "bs_draft_sample")
+
+
+def bs_softmax_verify_drafted(target_logits, draft_logits, draft_tokens, gamma, u_accept, temperature: float,
+                              accept_len, p_tok, q_tok, workspace, stream=None) -> None:
+    B, G1, V = target_logits.shape
+    _check(_lib.bs_softmax_verify_drafted(_ptr(target_logits), _ptr(draft_logits), _dtype_code(target_logits),
+                                          _ptr(draft_tokens), _ptr(gamma), _ptr(u_accept), float(temperature),
+                                          B, G1 - 1, V, _ptr(accept_len), _ptr(p_tok), _ptr(q_tok),
+                                          _ptr(workspace), workspace.numel(), _stream(stream)),
+           "bs_softmax_verify_drafted")
 
 
 # ---- fused LM head ----------------------------------------------------------------------

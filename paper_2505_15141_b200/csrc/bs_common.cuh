@@ -28,7 +28,8 @@ __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a -
 // Workspace regions (all offsets multiples of 256 bytes).
 //   ticket_verify [B] u32     per-sequence arrival counters of the statistics kernel (zero between calls)
 //   ticket_resid  [B] u32     per-sequence arrival counters of the resampling kernel (zero between calls)
-//   ticket_row    [B, R] u32  per-row arrival counters of the statistics kernel (zero between calls)
+//   ticket_row    [B, R] u32  first B words: bit j set = the statistics of draft row j were left by a
+//                             drafting call (bs_draft_sample) and not yet consumed; rest unused
 //   status        [B] i32     device-data status bits of the last call pair
 //   abort         [1] i32     set when a bounded pipeline wait gave up (reported as BS_ERR_TIMEOUT)
 //   row_stats     [B, R, 2] f32, R = 2*Gmax+1: (raw max logit, Z) per row; greedy: (max, arg-max bits)

@@ -583,6 +583,7 @@ extern "C" bs_status bs_lmhead_verify(const void* H_t, const void* W_t, int d_t,
     vp.B = B; vp.Gmax = Gmax; vp.V = V; vp.R = w.R; vp.S = w.S;
     vp.seg = seg_elems(BS_F32); vp.nseg = div_up(V, vp.seg);
     vp.c = lp.c;
+    vp.mode = kModeVerify; vp.position = 0; vp.draft_ready = vp.ticket_row; vp.draft_out = nullptr;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (mh == 1)
         return greedy ? launch_lmhead<1, 4, true>(tms, lp, vp, partial, st)

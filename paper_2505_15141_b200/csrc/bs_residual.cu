@@ -321,6 +321,7 @@ extern "C" bs_status bs_residual_sample(const void* target_logits, const void* d
     p.seg = res_seg_elems(dtype);
     p.nseg = div_up(V, p.seg);
     p.c = greedy ? 1.f : kLog2e / temperature;
+    p.mode = kResidVerify; p.position = 0; p.draft_out = nullptr;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (greedy) {
         return cuda_status(launch_pdl(greedy_emit_kernel, div_up(B, 128), 128, 0, st, p));
@@ -332,4 +333,29 @@ extern "C" bs_status bs_residual_sample(const void* target_logits, const void* d
     if (aligned)
         return dtype == BS_F32 ? launch_residual_stream<float>(p, st) : launch_residual_stream<__nv_bfloat16>(p, st);
     return dtype == BS_F32 ? launch_residual<float>(p, st) : launch_residual<__nv_bfloat16>(p, st);
+}
+
+// Sampling pass of bs_draft_sample: the resampling kernel in its drafting mode, on the draft row
+// `position` whose statistics the statistics pass has just left in the workspace.
+bs_status bs::run_draft_resample(const void* draft_logits, bs_dtype dtype, int position, const int32_t* gamma,
+                                 const float* u_draft, float temperature, int B, int Gmax, int V,
+                                 int32_t* draft_tokens, void* workspace, size_t workspace_bytes, void* stream) {
+    const Workspace w = workspace_layout(B, Gmax, V);
+    if (workspace_bytes < w.total || (reinterpret_cast<uintptr_t>(workspace) & 255)) return BS_ERR_WORKSPACE;
+    char* ws = static_cast<char*>(workspace);
+    ResidParams p;
+    p.target = nullptr; p.draft = draft_logits; p.tokens = nullptr; p.gamma = gamma;
+    p.accept_len = nullptr; p.u_resample = u_draft; p.out_tokens = nullptr; p.out_len = nullptr;
+    p.ticket = reinterpret_cast<uint32_t*>(ws + w.off_ticket_resid);
+    p.status = reinterpret_cast<int32_t*>(ws + w.off_status);
+    p.abort_flag = reinterpret_cast<int32_t*>(ws + w.off_abort);
+    p.row_stats = reinterpret_cast<const float2*>(ws + w.off_row_stats);
+    p.resid_partial = reinterpret_cast<float*>(ws + w.off_resid_partial);
+    p.B = B; p.Gmax = Gmax; p.V = V; p.R = w.R; p.S = w.Sr;
+    p.seg = res_seg_elems(dtype);
+    p.nseg = div_up(V, p.seg);
+    p.c = kLog2e / temperature;
+    p.mode = kResidDraft; p.position = position; p.draft_out = draft_tokens;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return dtype == BS_F32 ? launch_residual_stream<float>(p, st) : launch_residual_stream<__nv_bfloat16>(p, st);
 }

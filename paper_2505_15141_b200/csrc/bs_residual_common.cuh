@@ -24,7 +24,14 @@ struct ResidParams {
     int B, Gmax, V, R, S;
     int nseg, seg;
     float c;
+    // kResidVerify: Algorithm 6's resampling / bonus step.  kResidDraft: the drafting step -- for
+    // every sequence with position < gamma_b one token from softmax(draft row `position`), uniform
+    // u_resample[b, position] (a [B, Gmax] array in this mode), written to draft_out[b, position];
+    // the row's statistics are read from its draft slot.
+    int mode, position;
+    int32_t* draft_out;
 };
+constexpr int kResidVerify = 0, kResidDraft = 1;
 
 // Mass of one element.  kt / kd fold the row max and normaliser: p = 2^(x*c + kt).
 struct MassFn {
@@ -40,5 +47,9 @@ struct MassFn {
 
 template <typename T>
 bs_status launch_residual_stream(const ResidParams& p, cudaStream_t st);      // pipelined kernel, aligned rows
+
+bs_status run_draft_resample(const void* draft_logits, bs_dtype dtype, int position, const int32_t* gamma,
+                             const float* u_draft, float temperature, int B, int Gmax, int V, int32_t* draft_tokens,
+                             void* workspace, size_t workspace_bytes, void* stream);
 
 }  // namespace bs

@@ -54,6 +54,12 @@ __device__ __forceinline__ RsSeq rs_seq(const ResidParams& p, int b) {
     int g = p.gamma[b];
     if (g < 0 || g > p.Gmax) g = 0;
     RsSeq s;
+    if (p.mode == kResidDraft) {          // drafting: sample from the draft row `position` alone, if the sequence drafts it
+        s.tau = p.position;
+        s.bonus = 1;
+        s.wgt = p.position < g ? 1 : 0;
+        return s;
+    }
     s.tau = max(0, min(p.accept_len[b], g));
     s.bonus = s.tau >= g;
     s.wgt = s.bonus ? 1 : 2;
@@ -61,10 +67,21 @@ __device__ __forceinline__ RsSeq rs_seq(const ResidParams& p, int b) {
 }
 // Items [i0, i1) of sequence b whose first weight unit lies in [lo, hi); pre = first unit of b.
 __device__ __forceinline__ void rs_items(int pre, int wgt, int nseg, int lo, int hi, int& i0, int& i1) {
+    if (wgt <= 0) { i0 = i1 = 0; return; }
     const int a = max(lo, pre) - pre, e = min(hi, pre + wgt * nseg) - pre;
     i0 = (a + wgt - 1) / wgt;
     i1 = e > 0 ? (e + wgt - 1) / wgt : 0;
     if (i1 < i0) i1 = i0;
+}
+
+// The row that is sampled alone (or minus the draft row) and the slot of its statistics.
+template <typename T>
+__device__ __forceinline__ const T* rs_trow(const ResidParams& p, int b, const RsSeq& sq) {
+    return p.mode == kResidDraft ? row_ptr(static_cast<const T*>(p.draft), b, p.Gmax, p.position, p.V)
+                                 : row_ptr(static_cast<const T*>(p.target), b, p.Gmax + 1, sq.tau, p.V);
+}
+__device__ __forceinline__ int rs_tslot(const ResidParams& p, const RsSeq& sq) {
+    return p.mode == kResidDraft ? p.Gmax + 1 + p.position : sq.tau;
 }
 
 template <typename T>
@@ -95,7 +112,7 @@ template <typename T>
 __device__ void rs_level2(const ResidParams& p, int b, const RsSeq sq, MassFn f) {
     constexpr int kVec = Elem<T>::kVec;
     const int lane = threadIdx.x & 31;
-    const T* tp = row_ptr(static_cast<const T*>(p.target), b, p.Gmax + 1, sq.tau, p.V);
+    const T* tp = rs_trow<T>(p, b, sq);
     const T* dp = f.bonus ? tp : row_ptr(static_cast<const T*>(p.draft), b, p.Gmax, sq.tau, p.V);
     const float* pm = p.resid_partial + (size_t)b * p.S;
     const int nsub = p.nseg * kRsWarps;
@@ -113,7 +130,7 @@ __device__ void rs_level2(const ResidParams& p, int b, const RsSeq sq, MassFn f)
     }
     double incl = warp_scan_incl(mine);
     double Rtot = __shfl_sync(0xffffffffu, incl, 31);
-    const float u = p.u_resample[b];
+    const float u = p.mode == kResidDraft ? p.u_resample[(size_t)b * p.Gmax + p.position] : p.u_resample[b];
     int tok = -1;
 
     if (Rtot > 0.0 && isfinite(Rtot)) {
@@ -256,6 +273,14 @@ __device__ void rs_level2(const ResidParams& p, int b, const RsSeq sq, MassFn f)
         }
         if (tok < 0) { tok = 0; bits |= BS_DEV_NONFINITE; }
     }
+    if (p.mode == kResidDraft) {                              // drafting: the token is the whole output
+        if (lane == 0) {
+            p.draft_out[(size_t)b * p.Gmax + p.position] = tok;
+            if (bits) atomicOr(p.status + b, bits);
+            p.ticket[b] = 0u;
+        }
+        return;
+    }
     // ---- outputs: the tau accepted drafts, the sampled token, padding ----
     int32_t* ot = p.out_tokens + (size_t)b * (p.Gmax + 1);
     for (int j = lane; j <= p.Gmax; j += 32)
@@ -368,9 +393,9 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
             int i0, i1;
             rs_items(s_prefix[b], sq.wgt, p.nseg, lo, hi, i0, i1);
             if (i1 <= i0) continue;
-            const float2 ts = p.row_stats[(size_t)b * p.R + sq.tau];
+            const float2 ts = p.row_stats[(size_t)b * p.R + rs_tslot(p, sq)];
             float kt = -(ts.x * p.c + log2f(ts.y)), kd = 0.f;
-            const T* tp = row_ptr(static_cast<const T*>(p.target), b, p.Gmax + 1, sq.tau, p.V);
+            const T* tp = rs_trow<T>(p, b, sq);
             const T* dp = tp;
             if (!sq.bonus) {
                 const float2 ds = p.row_stats[(size_t)b * p.R + p.Gmax + 1 + sq.tau];
@@ -430,7 +455,7 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
                 MassFn f;
                 f.c = p.c;
                 f.bonus = sq.bonus;
-                const float2 ts = p.row_stats[(size_t)b * p.R + sq.tau];
+                const float2 ts = p.row_stats[(size_t)b * p.R + rs_tslot(p, sq)];
                 f.kt = -(ts.x * p.c + log2f(ts.y));
                 f.kd = 0.f;
                 if (!sq.bonus) {

@@ -252,18 +252,26 @@ extern "C" bs_status bs_get_device_status(const void* workspace, size_t workspac
     return BS_OK;
 }
 
-extern "C" bs_status bs_softmax_verify(const void* target_logits, const void* draft_logits, bs_dtype dtype,
-                                       const int32_t* draft_tokens, const int32_t* gamma, const float* u_accept,
-                                       float temperature, int B, int Gmax, int V,
-                                       int32_t* accept_len, float* p_tok, float* q_tok,
-                                       void* workspace, size_t workspace_bytes, void* stream) {
+// Host side shared by bs_softmax_verify (kModeVerify), bs_softmax_verify_drafted (kModeDrafted) and
+// the statistics pass of bs_draft_sample (kModeDraft: target_logits and accept_len unused,
+// draft_out = the token array for greedy drafting).
+bs_status bs::run_verify(const void* target_logits, const void* draft_logits, bs_dtype dtype,
+                         const int32_t* draft_tokens, const int32_t* gamma, const float* u_accept,
+                         float temperature, int B, int Gmax, int V, int32_t* accept_len, float* p_tok, float* q_tok,
+                         void* workspace, size_t workspace_bytes, void* stream, int mode, int position,
+                         int32_t* draft_out) {
     if (!sizes_ok(B, Gmax, V)) return (B < 1 || Gmax < 0 || V < 1) ? BS_ERR_INVALID_ARG : BS_ERR_UNSUPPORTED;
     if (dtype != BS_F32 && dtype != BS_BF16) return BS_ERR_INVALID_ARG;
     if (!(temperature >= 0.f) || !isfinite(temperature)) return BS_ERR_INVALID_ARG;
     const bool greedy = temperature == 0.f;
-    if (!target_logits || !gamma || !accept_len || !workspace) return BS_ERR_INVALID_ARG;
-    if (Gmax > 0 && !draft_tokens) return BS_ERR_INVALID_ARG;
-    if (!greedy && Gmax > 0 && (!draft_logits || !u_accept)) return BS_ERR_INVALID_ARG;
+    if (!gamma || !workspace) return BS_ERR_INVALID_ARG;
+    if (mode == kModeDraft) {
+        if (!draft_logits || position < 0 || position >= Gmax || (greedy && !draft_out)) return BS_ERR_INVALID_ARG;
+    } else {
+        if (!target_logits || !accept_len) return BS_ERR_INVALID_ARG;
+        if (Gmax > 0 && !draft_tokens) return BS_ERR_INVALID_ARG;
+        if (!greedy && Gmax > 0 && (!draft_logits || !u_accept)) return BS_ERR_INVALID_ARG;
+    }
     const size_t es = dtype == BS_F32 ? 4 : 2;
     if ((reinterpret_cast<uintptr_t>(target_logits) % es) || (reinterpret_cast<uintptr_t>(draft_logits) % es))
         return BS_ERR_INVALID_ARG;
@@ -284,10 +292,13 @@ extern "C" bs_status bs_softmax_verify(const void* target_logits, const void* dr
     p.seg = seg_elems(dtype);
     p.nseg = div_up(V, p.seg);
     p.c = greedy ? 1.f : kLog2e / temperature;
+    p.mode = mode; p.position = position; p.draft_out = draft_out;
+    p.draft_ready = p.ticket_row;          // the per-row counters' slot: the pipelined kernel counts per sequence
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // rows start on 16-byte boundaries: bulk-copy pipeline; otherwise the generic kernel
     const bool aligned = ((size_t)V * es) % 16 == 0 && (reinterpret_cast<uintptr_t>(target_logits) & 15) == 0 &&
                          (reinterpret_cast<uintptr_t>(draft_logits) & 15) == 0;
+    if (!aligned && mode != kModeVerify) return BS_ERR_UNSUPPORTED;   // the drafting path needs aligned rows
     if (aligned) {
         if (dtype == BS_F32)
             return greedy ? launch_verify_stream<float, true>(p, st) : launch_verify_stream<float, false>(p, st);
@@ -297,4 +308,13 @@ extern "C" bs_status bs_softmax_verify(const void* target_logits, const void* dr
     if (dtype == BS_F32)
         return greedy ? launch_verify<float, true>(p, 0, st) : launch_verify<float, false>(p, 1, st);
     return greedy ? launch_verify<__nv_bfloat16, true>(p, 2, st) : launch_verify<__nv_bfloat16, false>(p, 3, st);
+}
+
+extern "C" bs_status bs_softmax_verify(const void* target_logits, const void* draft_logits, bs_dtype dtype,
+                                       const int32_t* draft_tokens, const int32_t* gamma, const float* u_accept,
+                                       float temperature, int B, int Gmax, int V,
+                                       int32_t* accept_len, float* p_tok, float* q_tok,
+                                       void* workspace, size_t workspace_bytes, void* stream) {
+    return run_verify(target_logits, draft_logits, dtype, draft_tokens, gamma, u_accept, temperature, B, Gmax, V,
+                      accept_len, p_tok, q_tok, workspace, workspace_bytes, stream, kModeVerify, 0, nullptr);
 }

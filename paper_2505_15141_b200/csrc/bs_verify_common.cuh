@@ -27,7 +27,16 @@ struct VerifyParams {
     int B, Gmax, V, R, S;
     int nseg, seg;           // segments per row and elements per segment for this dtype
     float c;                 // log2(e) / temperature
+    // Which rows a sequence contributes (pipelined kernel only):
+    //   kModeVerify   target rows 0..g and draft rows 0..g-1 (target rows only in greedy mode)
+    //   kModeDraft    the one draft row `position` (if position < g): its statistics go to the
+    //                 draft slot of that position, no accept test; greedy: the arg-max is the token
+    //   kModeDrafted  target rows 0..g only; the draft statistics are those kModeDraft left
+    int mode, position;
+    uint32_t* draft_ready;   // [B] bit j set: the statistics of draft row j are in row_stats
+    int32_t* draft_out;      // kModeDraft, greedy: [B, Gmax] drafted tokens (entry [b, position] written)
 };
+constexpr int kModeVerify = 0, kModeDraft = 1, kModeDrafted = 2;
 
 struct ArgMax {
     float m;
@@ -149,6 +158,24 @@ __device__ __forceinline__ int seq_rows(int g, int Gmax) {
 // local row index (0..rows_b-1) -> row slot in [0, R): target rows first, then draft rows
 __device__ __forceinline__ int row_slot(int lr, int g, int Gmax) { return lr <= g ? lr : Gmax + 1 + (lr - g - 1); }
 
+// The same three questions for any mode of the pipelined kernel (g already clamped).
+template <bool GREEDY>
+__device__ __forceinline__ int mode_rows(const VerifyParams& p, int g) {
+    if (p.mode == kModeDraft) return p.position < g ? 1 : 0;
+    if (p.mode == kModeDrafted) return g + 1;
+    return GREEDY ? g + 1 : 2 * g + 1;
+}
+__device__ __forceinline__ int mode_slot(const VerifyParams& p, int lr, int g) {
+    if (p.mode == kModeDraft) return p.Gmax + 1 + p.position;
+    return row_slot(lr, g, p.Gmax);                      // kModeDrafted: lr <= g, so the slot is lr
+}
+template <typename T>
+__device__ __forceinline__ const T* mode_row(const VerifyParams& p, int b, int lr, int g) {
+    if (p.mode == kModeDraft) return row_ptr(static_cast<const T*>(p.draft), b, p.Gmax, p.position, p.V);
+    return lr <= g ? row_ptr(static_cast<const T*>(p.target), b, p.Gmax + 1, lr, p.V)
+                   : row_ptr(static_cast<const T*>(p.draft), b, p.Gmax, lr - g - 1, p.V);
+}
+
 // One warp merges the nseg partial slots of a row (all lanes return the result).
 template <bool GREEDY>
 __device__ __forceinline__ float2 merge_row_partials(const float2* pp, int nseg, float c) {
@@ -202,11 +229,11 @@ __device__ __forceinline__ AcceptLoads accept_prefetch(const VerifyParams& p, in
 // accept_len, p_tok, q_tok and the status word.  graw = gamma[b] as read, g = clamp_gamma(graw).
 template <typename T, bool GREEDY, typename StatsFn>
 __device__ __forceinline__ void accept_finish(const VerifyParams& p, int b, int graw, int g, const AcceptLoads& a,
-                                              StatsFn stats) {
+                                              StatsFn stats, int extra_bits = 0) {
     const int lane = threadIdx.x & 31;
     const int j = lane;
     const bool valid = j < g;
-    int st_bits = ((graw != g) ? BS_DEV_BAD_GAMMA : 0) | a.bits;
+    int st_bits = ((graw != g) ? BS_DEV_BAD_GAMMA : 0) | a.bits | extra_bits;
     bool acc = false;
     float pj = 0.f, qj = 0.f;
     if (valid) {
@@ -229,6 +256,7 @@ __device__ __forceinline__ void accept_finish(const VerifyParams& p, int b, int 
                 acc = (lq == -INFINITY) ? true : (a.u <= fminf(1.f, exp2f(lp - lq)));
             }
         }
+        if (extra_bits & BS_DEV_DRAFT_MISSING) acc = false;   // no draft statistics: nothing is accepted
     }
     if (!GREEDY && j == g) {              // the bonus row's normaliser is used by the resampler
         const float2 ts = stats(g);
@@ -260,5 +288,10 @@ __device__ __forceinline__ void accept_scan_warp(const VerifyParams& p, int b, S
 
 template <typename T, bool GREEDY>
 bs_status launch_verify_stream(const VerifyParams& p, cudaStream_t st);   // pipelined kernel, aligned rows
+
+bs_status run_verify(const void* target_logits, const void* draft_logits, bs_dtype dtype, const int32_t* draft_tokens,
+                     const int32_t* gamma, const float* u_accept, float temperature, int B, int Gmax, int V,
+                     int32_t* accept_len, float* p_tok, float* q_tok, void* workspace, size_t workspace_bytes,
+                     void* stream, int mode, int position, int32_t* draft_out);
 
 }  // namespace bs

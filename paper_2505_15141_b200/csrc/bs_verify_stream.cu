@@ -91,7 +91,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) verify_stream_kernel(const 
         int local = 0;
         for (int k = 0; k < per; ++k) {
             const int b = b0 + k;
-            if (b < p.B) local += seq_rows<GREEDY>(p.gamma[b], p.Gmax) * p.nseg;
+            if (b < p.B) local += mode_rows<GREEDY>(p, clamp_gamma(p.gamma[b], p.Gmax)) * p.nseg;
         }
         int incl = local;
 #pragma unroll
@@ -108,7 +108,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) verify_stream_kernel(const 
             const int b = b0 + k;
             if (b < p.B) {
                 s_prefix[b] = run;
-                run += seq_rows<GREEDY>(p.gamma[b], p.Gmax) * p.nseg;
+                run += mode_rows<GREEDY>(p, clamp_gamma(p.gamma[b], p.Gmax)) * p.nseg;
             }
         }
         if (tid == kStreamThreads - 1) s_prefix[p.B] = run;
@@ -136,16 +136,13 @@ __global__ void __launch_bounds__(kStreamThreads, 2) verify_stream_kernel(const 
             lr = local / p.nseg;
             sg = local - lr * p.nseg;
             g = clamp_gamma(p.gamma[b], p.Gmax);
-            rows_b = GREEDY ? g + 1 : 2 * g + 1;
+            rows_b = mode_rows<GREEDY>(p, g);
         }
         int slot = 0;
         uint32_t ph = 0;
         for (int k = 0; k < count; ++k) {
             if (!mbar_wait(smem_u32(&s_empty[slot]), ph ^ 1u)) { atomicExch(p.abort_flag, 1); return; }
-            const bool is_target = lr <= g;
-            const T* rowp = is_target
-                ? row_ptr(static_cast<const T*>(p.target), b, p.Gmax + 1, lr, p.V)
-                : row_ptr(static_cast<const T*>(p.draft), b, p.Gmax, lr - g - 1, p.V);
+            const T* rowp = mode_row<T>(p, b, lr, g);
             const int e0 = sg * p.seg;
             const int n = min(p.seg, p.V - e0);
             const uint32_t bytes = (uint32_t)n * (uint32_t)sizeof(T);
@@ -162,11 +159,13 @@ __global__ void __launch_bounds__(kStreamThreads, 2) verify_stream_kernel(const 
                 sg = 0;
                 if (++lr == rows_b) {
                     lr = 0;
-                    ++b;
-                    if (b < p.B) {
-                        g = clamp_gamma(p.gamma[b], p.Gmax);
-                        rows_b = GREEDY ? g + 1 : 2 * g + 1;
-                    }
+                    do {                                      // next sequence that contributes rows
+                        ++b;
+                        if (b < p.B) {
+                            g = clamp_gamma(p.gamma[b], p.Gmax);
+                            rows_b = mode_rows<GREEDY>(p, g);
+                        }
+                    } while (b < p.B && rows_b == 0);
                 }
             }
             if (++slot == nstages) { slot = 0; ph ^= 1u; }
@@ -202,9 +201,9 @@ __global__ void __launch_bounds__(kStreamThreads, 2) verify_stream_kernel(const 
             const int first_sg = pm.first_sg & 0xffff;
             const int graw = p.gamma[m_b];
             const int gb = clamp_gamma(graw, p.Gmax);
-            const int r = row_slot(m_lr, gb, p.Gmax);
+            const int r = mode_slot(p, m_lr, gb);
             const int piece_len = m_sg - first_sg + 1;
-            const int rows_mb = GREEDY ? gb + 1 : 2 * gb + 1;
+            const int rows_mb = mode_rows<GREEDY>(p, gb);
             {
                 float2* pp = p.partial + ((size_t)m_b * p.R + r) * p.S;
                 // slot of the piece's first segment carries the result, the rest are neutral
@@ -213,7 +212,8 @@ __global__ void __launch_bounds__(kStreamThreads, 2) verify_stream_kernel(const 
             }
             // the loads of the accept test do not depend on the statistics: start them now, so
             // that they travel while the arrival counter does
-            const AcceptLoads al = accept_prefetch<T, GREEDY>(p, m_b, gb);
+            AcceptLoads al{0, 0.f, 0.f, 2.f, 0};
+            if (p.mode != kModeDraft) al = accept_prefetch<T, GREEDY>(p, m_b, gb);
             __threadfence();
             __syncwarp();
             unsigned old = 0;
@@ -225,7 +225,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) verify_stream_kernel(const 
                 for (int lr0 = 0; lr0 < rows_mb; lr0 += 32) {
                     const int lr = lr0 + lane;
                     if (lr < rows_mb) {
-                        const int rr = row_slot(lr, gb, p.Gmax);
+                        const int rr = mode_slot(p, lr, gb);
                         const float2* pp = p.partial + ((size_t)m_b * p.R + rr) * p.S;
                         float2 st;
                         if (GREEDY) {
@@ -251,7 +251,26 @@ __global__ void __launch_bounds__(kStreamThreads, 2) verify_stream_kernel(const 
                     }
                 }
                 __syncwarp();
-                accept_finish<T, GREEDY>(p, m_b, graw, gb, al, [&](int rr) { return s_fin[rr]; });
+                if (p.mode == kModeDraft) {
+                    // the draft row's statistics are in place; greedy drafting ends here
+                    if (lane == 0) {
+                        if (GREEDY) p.draft_out[(size_t)m_b * p.Gmax + p.position] = __float_as_int(s_fin[r].y);
+                        __threadfence();
+                        atomicOr(p.draft_ready + m_b, 1u << p.position);
+                    }
+                } else if (p.mode == kModeDrafted) {
+                    // target rows were merged just now, the draft rows' statistics were left by the drafting calls
+                    const unsigned need = gb >= 32 ? 0xffffffffu : ((1u << gb) - 1u);
+                    const unsigned have = GREEDY ? need : __ldcg(p.draft_ready + m_b);
+                    const float2* rsb = p.row_stats + (size_t)m_b * p.R;
+                    const int G1 = p.Gmax + 1;
+                    accept_finish<T, GREEDY>(p, m_b, graw, gb, al,
+                                             [&](int rr) { return rr < G1 ? s_fin[rr] : __ldcg(rsb + rr); },
+                                             (have & need) == need ? 0 : BS_DEV_DRAFT_MISSING);
+                    if (lane == 0) p.draft_ready[m_b] = 0u;       // consumed: a later round must draft again
+                } else {
+                    accept_finish<T, GREEDY>(p, m_b, graw, gb, al, [&](int rr) { return s_fin[rr]; });
+                }
                 if (lane == 0) p.ticket[m_b] = 0u;                // leave the counter clear for the next call
             }
             if (pm.first_sg >> 16) break;                     // that was the CTA's last piece
