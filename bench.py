@@ -67,6 +67,9 @@ def parse_args():
     ap.add_argument("--fixed-gamma", type=int, default=0,
                     help="replace the workload's arms by one arm of this speculation length, so that the bytes "
                          "of every launch are known exactly (profiler captures)")
+    ap.add_argument("--drafted", action="store_true",
+                    help="the round with drafting on the device: select -> bs_draft_sample per position -> "
+                         "bs_softmax_verify_drafted -> bs_residual_sample -> update")
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="budget of the CPU-oracle sample")
@@ -255,7 +258,8 @@ def run_cuda(args, w):
             target=rnd.target, draft=rnd.draft, tokens=rnd.tokens.contiguous(),
             u_accept=torch.as_tensor(rnd.uniforms.u_accept, device=dev),
             u_resample=torch.as_tensor(rnd.uniforms.u_resample, device=dev),
-            u_arm=torch.as_tensor(rnd.uniforms.u_arm, device=dev), rnd=rnd))
+            u_arm=torch.as_tensor(rnd.uniforms.u_arm, device=dev),
+            u_draft=torch.as_tensor(rnd.uniforms.u_draft, device=dev), rnd=rnd))
     state = bs.new_bandit(alg, B, w.arm_gamma, w.delta, dev)
     ws = bs.new_workspace(B, G, V, dev)
     arm_d = torch.zeros(B, dtype=torch.int32, device=dev)
@@ -266,10 +270,28 @@ def run_cuda(args, w):
     out_tokens = torch.zeros(B, G + 1, dtype=torch.int32, device=dev)
     out_len = torch.zeros(B, dtype=torch.int32, device=dev)
 
+    drafted = args.drafted
+    rows_per_gamma = (arm_gamma + 1) if drafted else (2 * arm_gamma + 1)     # rows the verify call streams
+    tok_d = torch.zeros(B, G, dtype=torch.int32, device=dev)                 # tokens drafted on the device
+
+    def verify_call(s):
+        if drafted:
+            bs.bs_softmax_verify_drafted(s["target"], s["draft"], tok_d, gamma_d, s["u_accept"], w.temperature,
+                                         accept_len, p_tok, q_tok, ws)
+        else:
+            bs.bs_softmax_verify(s["target"], s["draft"], s["tokens"], gamma_d, s["u_accept"], w.temperature,
+                                 accept_len, p_tok, q_tok, ws)
+
+    def draft_calls(s):
+        for j in range(G):
+            bs.bs_draft_sample(s["draft"], j, gamma_d, s["u_draft"], w.temperature, tok_d, ws)
+
     def step_calls(s):
         bs.bs_bandit_select(state, alg, B, K, s["u_arm"], None, arm_d, gamma_d)
-        bs.bs_softmax_verify(s["target"], s["draft"], s["tokens"], gamma_d, s["u_accept"], w.temperature,
-                             accept_len, p_tok, q_tok, ws)
+        if drafted:
+            draft_calls(s)
+            s = dict(s, tokens=tok_d)
+        verify_call(s)
         bs.bs_residual_sample(s["target"], s["draft"], s["tokens"], gamma_d, accept_len, s["u_resample"],
                               w.temperature, out_tokens, out_len, ws)
         bs.bs_bandit_update(state, alg, B, K, arm_d, out_len)
@@ -328,7 +350,7 @@ def run_cuda(args, w):
     n1 = pulls()
     dn = (n1 - n0)                                             # [B, K] pulls inside the timed region
     assert dn.sum() == B * args.steps, "every sequence must have played every timed round"
-    rows_timed = int((dn * (2 * arm_gamma + 1)[None, :]).sum())
+    rows_timed = int((dn * (2 * arm_gamma + 1)[None, :]).sum())     # drafted or not: every valid row once
     bytes_timed = rows_timed * V * es
     ms, bytes_all = reduce_over_ranks(ms, bytes_timed, dev)
     value = job_rounds_per_s(world, args.steps, ms)
@@ -337,14 +359,18 @@ def run_cuda(args, w):
     ksteps = min(args.steps, 50)
     evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(ksteps)]
     rsd = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(ksteps)]
+    dft = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(ksteps)]
     nk0 = pulls()
-    y_total = 0
     for i in range(ksteps):
         s = sets[(args.warmup + args.steps + i) % ring]
         bs.bs_bandit_select(state, alg, B, K, s["u_arm"], None, arm_d, gamma_d)
+        if drafted:
+            dft[i][0].record(stream)
+            draft_calls(s)
+            dft[i][1].record(stream)
+            s = dict(s, tokens=tok_d)
         evs[i][0].record(stream)
-        bs.bs_softmax_verify(s["target"], s["draft"], s["tokens"], gamma_d, s["u_accept"], w.temperature,
-                             accept_len, p_tok, q_tok, ws)
+        verify_call(s)
         evs[i][1].record(stream)
         rsd[i][0].record(stream)
         bs.bs_residual_sample(s["target"], s["draft"], s["tokens"], gamma_d, accept_len, s["u_resample"],
@@ -356,7 +382,9 @@ def run_cuda(args, w):
     verify_ms = sum(a.elapsed_time(b) for a, b in evs) / ksteps
     resid_ms = sum(a.elapsed_time(b) for a, b in rsd) / ksteps
     dk = pulls() - nk0
-    verify_bytes = float((dk * (2 * arm_gamma + 1)[None, :]).sum()) * V * es / ksteps   # per launch
+    verify_bytes = float((dk * rows_per_gamma[None, :]).sum()) * V * es / ksteps   # per launch
+    draft_ms = sum(a.elapsed_time(b) for a, b in dft) / ksteps if drafted else None
+    draft_bytes = float((dk * arm_gamma[None, :]).sum()) * V * es / ksteps if drafted else None
     mean_y = float(y_sum.item()) / (B * ksteps)
     status = bs.bs_get_device_status(ws, B, G, V)
     assert (status & ~bs.BS_DEV_RESIDUAL_FALLBACK == 0).all(), f"device status {status}"
@@ -373,7 +401,7 @@ def run_cuda(args, w):
     if args.e2e_steps > 0:
         s0 = sets[0]
         host = {k: torch.empty(s0[k].shape, dtype=s0[k].dtype, pin_memory=True).copy_(s0[k])
-                for k in ("target", "draft", "tokens", "u_accept", "u_resample", "u_arm")}
+                for k in ("target", "draft", "tokens", "u_accept", "u_resample", "u_arm", "u_draft")}
         devb = {k: torch.empty_like(s0[k]) for k in host}
         h_tokens = torch.empty(out_tokens.shape, dtype=out_tokens.dtype, pin_memory=True)
         h_len = torch.empty(out_len.shape, dtype=out_len.dtype, pin_memory=True)
@@ -426,6 +454,8 @@ def run_cuda(args, w):
                        "logits_dtype": w.dtype, "temperature": w.temperature,
                        "l2": f"ring of {ring} input sets, {ring * set_bytes / 1e6:.0f} MB > 2 x L2",
                        "launch": "one CUDA graph per step" if graphs else "direct launches",
+                       "path": ("select, draft x Gmax, verify on drafted statistics, resample, update"
+                                if drafted else "select, verify, resample, update"),
                        "multi_gpu": "one independent batch per rank, no collective on the data path"},
             "tokens_per_s": mean_y * B * value,
             "mean_accepted_len": mean_y,
@@ -435,8 +465,12 @@ def run_cuda(args, w):
                          "traffic": ncu_traffic(w.name, verify_bytes), "bytes_per_launch": verify_bytes,
                          "ms_per_launch": verify_ms, "residual_ms_per_launch": resid_ms},
             "e2e": e2e, "cpu_baseline": cpu, "clocks": clocks,
-            "gpu_launches": 4 * args.steps,
+            "gpu_launches": (4 + (2 * G if drafted else 0)) * args.steps,
         }
+        if drafted:
+            line["drafting"] = {"ms_per_round": draft_ms, "calls": G, "row_bytes_per_round": draft_bytes,
+                                "note": "each call reads its draft rows once for the statistics and once more "
+                                        "(mostly from L2) for the inverse CDF"}
         print(json.dumps(line))
     if world > 1:
         dist.barrier()

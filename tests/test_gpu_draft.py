@@ -128,3 +128,33 @@ def test_verify_drafted_without_drafting_is_reported(lib):
         lib.bs_draft_sample(d_odd, 0, torch.ones(2, dtype=torch.int32, device=DEV), torch.full((2, 2), 0.5, device=DEV),
                             1.0, torch.zeros(2, 2, dtype=torch.int32, device=DEV), lib.new_workspace(2, 2, 1001, DEV))
     assert e.value.code == lib.BS_ERR_UNSUPPORTED
+
+
+def test_drafted_round_full_size(lib):
+    """64 sequences, 128256-entry vocabulary, bf16, ragged speculation lengths up to 8 (the launch
+    configuration the benchmark's --drafted round times): drafted tokens of sampled sequences against
+    the oracle, the drafted verification against the plain one for every sequence."""
+    w = wl.WORKLOADS["llama3_ucb"]
+    B, G, V, T = w.B, w.Gmax, w.V, w.temperature
+    arm = np.arange(B) % w.K
+    rnd = wl.make_round(w, 5, arm, device=DEV)
+    gamma_d = torch.as_tensor(rnd.gamma, device=DEV)
+    ws = lib.new_workspace(B, G, V, DEV); ws2 = lib.new_workspace(B, G, V, DEV)
+    tok = _draft_all(lib, rnd.draft, gamma_d, torch.as_tensor(rnd.uniforms.u_draft, device=DEV), T, ws)
+    sample = [0, 3, 17, 42, 63]
+    sub = torch.as_tensor(sample, device=DEV)
+    assert _check_tokens(tok[sub], rnd.draft[sub], rnd.gamma[sample], rnd.uniforms.u_draft[sample], T) <= 1
+    tk = tok.cpu().numpy()
+    for b in range(B):
+        assert ((tk[b, :rnd.gamma[b]] >= 0) & (tk[b, :rnd.gamma[b]] < V)).all() and (tk[b, rnd.gamma[b]:] == -5).all()
+    tok = torch.where(tok < 0, torch.zeros_like(tok), tok).contiguous()
+    u_acc = torch.as_tensor(rnd.uniforms.u_accept, device=DEV)
+    res = []
+    for fn, w_ in ((lib.bs_softmax_verify_drafted, ws), (lib.bs_softmax_verify, ws2)):
+        acc = torch.zeros(B, dtype=torch.int32, device=DEV); p = torch.zeros(B, G, device=DEV); q = torch.zeros(B, G, device=DEV)
+        fn(rnd.target, rnd.draft, tok, gamma_d, u_acc, T, acc, p, q, w_)
+        torch.cuda.synchronize()
+        assert (lib.bs_get_device_status(w_, B, G, V) == 0).all()
+        res.append((acc, p, q))
+    assert torch.equal(res[0][0], res[1][0])
+    assert torch.allclose(res[0][1], res[1][1], atol=1e-6, rtol=0) and torch.allclose(res[0][2], res[1][2], atol=1e-6, rtol=0)
