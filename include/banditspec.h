@@ -161,6 +161,30 @@ bs_status bs_softmax_verify_noalloc(const void* target_logits, const void* draft
                                     float temperature, int B, int Gmax, int V,
                                     int32_t* accept_len, float* p_tok, float* q_tok, void* stream);
 
+/* ---- verification and resampling in one launch, with early exit ------------------------------- */
+
+/* Algorithm 6 from its second line on in the algorithm's own order: position after position,
+ * stopping at the first rejection (its "break"), then the resampling step -- bs_softmax_verify
+ * followed by bs_residual_sample, but rows behind the first rejected draft are never read: a
+ * sequence that stops at position tau costs 2 (tau + 1) rows (2 gamma + 1 when everything
+ * passes) plus a second pass over the rows of the stop position, instead of 2 gamma + 1 + 2.
+ *
+ *  arguments as bs_softmax_verify and bs_residual_sample; sampling mode only (temperature > 0,
+ *  BS_ERR_UNSUPPORTED otherwise: greedy rounds take the two separate calls)
+ *  p_tok, q_tok  [B, Gmax] fp32 out or NULL: filled for the positions that were examined
+ *                (j <= tau_b, j < gamma_b); the entries behind the stop are set to 0
+ *  accept_len, out_tokens, out_len: as the two separate calls
+ * The CTAs that share a sequence wait for one another, so the kernel is launched cooperatively
+ * and the call fails with BS_ERR_CUDA where that is not possible.  A wait that does not end
+ * within about a second makes bs_get_device_status return BS_ERR_TIMEOUT.
+ * Requirement: rows on 16-byte boundaries (V * element size a multiple of 16, base pointers
+ * 16-byte aligned), else BS_ERR_UNSUPPORTED. */
+bs_status bs_verify_walk(const void* target_logits, const void* draft_logits, bs_dtype dtype,
+                         const int32_t* draft_tokens, const int32_t* gamma, const float* u_accept,
+                         const float* u_resample, float temperature, int B, int Gmax, int V,
+                         int32_t* accept_len, float* p_tok, float* q_tok, int32_t* out_tokens, int32_t* out_len,
+                         void* workspace, size_t workspace_bytes, void* stream);
+
 /* ---- drafting on the device (Algorithm 6, first line: x~_{j+1} ~ Q(. | pt, x~_{1:j})) ------------ */
 
 /* Draws the drafted token of ONE position for every sequence that drafts it (position < gamma_b):

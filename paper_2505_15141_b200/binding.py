@@ -41,6 +41,7 @@ SIGNATURES = {
     "bs_softmax_verify": (_i, [_vp, _vp, _i, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bs_residual_sample": (_i, [_vp, _vp, _i, _vp, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _sz, _vp]),
     "bs_softmax_verify_noalloc": (_i, [_vp, _vp, _i, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _vp]),
+    "bs_verify_walk": (_i, [_vp, _vp, _i, _vp, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bs_draft_sample": (_i, [_vp, _i, _i, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _sz, _vp]),
     "bs_softmax_verify_drafted": (_i, [_vp, _vp, _i, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bs_lmhead_workspace_bytes": (_sz, [_i, _i, _i]),
@@ -183,6 +184,34 @@ def verify_round(target_logits, draft_logits, draft_tokens, gamma, u_accept, u_r
                       accept_len, p_tok, q_tok, workspace)
     bs_residual_sample(target_logits, draft_logits, draft_tokens, gamma, accept_len, u_resample,
                        temperature, out_tokens, out_len, workspace)
+    return RoundOutput(accept_len, p_tok, q_tok, out_tokens, out_len, workspace)
+
+
+def bs_verify_walk(target_logits, draft_logits, draft_tokens, gamma, u_accept, u_resample, temperature: float,
+                   accept_len, p_tok, q_tok, out_tokens, out_len, workspace, stream=None) -> None:
+    """Verification with early exit and resampling in one launch (sampling mode)."""
+    B, G1, V = target_logits.shape
+    _check(_lib.bs_verify_walk(_ptr(target_logits), _ptr(draft_logits), _dtype_code(target_logits),
+                               _ptr(draft_tokens), _ptr(gamma), _ptr(u_accept), _ptr(u_resample), float(temperature),
+                               B, G1 - 1, V, _ptr(accept_len), _ptr(p_tok), _ptr(q_tok), _ptr(out_tokens),
+                               _ptr(out_len), _ptr(workspace), workspace.numel(), _stream(stream)), "bs_verify_walk")
+
+
+def verify_round_walk(target_logits, draft_logits, draft_tokens, gamma, u_accept, u_resample,
+                      temperature: float, workspace: Optional[torch.Tensor] = None) -> RoundOutput:
+    """Allocates the outputs and calls bs_verify_walk."""
+    B, G1, V = target_logits.shape
+    G = G1 - 1
+    dev = target_logits.device
+    if workspace is None:
+        workspace = new_workspace(B, G, V, dev)
+    accept_len = torch.full((B,), -9, dtype=torch.int32, device=dev)
+    p_tok = torch.full((B, G), -1.0, dtype=torch.float32, device=dev)
+    q_tok = torch.full((B, G), -1.0, dtype=torch.float32, device=dev)
+    out_tokens = torch.full((B, G + 1), -9, dtype=torch.int32, device=dev)
+    out_len = torch.full((B,), -9, dtype=torch.int32, device=dev)
+    bs_verify_walk(target_logits, draft_logits, draft_tokens, gamma, u_accept, u_resample, temperature,
+                   accept_len, p_tok, q_tok, out_tokens, out_len, workspace)
     return RoundOutput(accept_len, p_tok, q_tok, out_tokens, out_len, workspace)
 
 

@@ -29,7 +29,8 @@ __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a -
 //   ticket_verify [B] u32     per-sequence arrival counters of the statistics kernel (zero between calls)
 //   ticket_resid  [B] u32     per-sequence arrival counters of the resampling kernel (zero between calls)
 //   ticket_row    [B, R] u32  first B words: bit j set = the statistics of draft row j were left by a
-//                             drafting call (bs_draft_sample) and not yet consumed; rest unused
+//                             drafting call (bs_draft_sample) and not yet consumed; second B words: decision
+//                             words of bs_verify_walk (zero between calls); rest unused
 //   status        [B] i32     device-data status bits of the last call pair
 //   abort         [1] i32     set when a bounded pipeline wait gave up (reported as BS_ERR_TIMEOUT)
 //   row_stats     [B, R, 2] f32, R = 2*Gmax+1: (raw max logit, Z) per row; greedy: (max, arg-max bits)
@@ -51,7 +52,7 @@ __host__ __device__ inline Workspace workspace_layout(int B, int Gmax, int V) {
     size_t o = 0;
     w.off_ticket_verify = o; o = align_up(o + sizeof(uint32_t) * (size_t)B, 256);
     w.off_ticket_resid = o;  o = align_up(o + sizeof(uint32_t) * (size_t)B, 256);
-    w.off_ticket_row = o;    o = align_up(o + sizeof(uint32_t) * (size_t)B * w.R, 256);
+    w.off_ticket_row = o;    o = align_up(o + sizeof(uint32_t) * (size_t)B * (w.R < 2 ? 2 : w.R), 256);
     w.off_status = o;        o = align_up(o + sizeof(int32_t) * (size_t)B, 256);
     w.off_abort = o;         o = align_up(o + sizeof(int32_t), 256);
     w.off_row_stats = o;     o = align_up(o + sizeof(float) * 2 * (size_t)B * w.R, 256);

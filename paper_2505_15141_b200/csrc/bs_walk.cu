@@ -1,0 +1,489 @@
+// bs_verify_walk: Algorithm 6 from its second line on, in one launch and in the algorithm's own
+// order -- position after position, stopping at the first rejection ("break"), so the rows behind
+// the first rejected draft are never read.
+//
+// Every sequence belongs to a fixed group of CTAs (nG = CTAs / B of them, 1 when there are more
+// sequences than CTAs, which then take several sequences each, one after the other).  For
+// position k the group streams target row k and draft row k (bulk async copies into a ring of
+// 32 KB stages, 16 consumer warps, online softmax: the pipeline of the row-statistics kernel),
+// every CTA its contiguous share of the 2 * nseg segments.  A finisher warp per CTA publishes the
+// pieces and counts them on the sequence's ticket; the finisher that completes position k merges
+// the two rows, tests r <= min{1, P/Q} for the drafted token and publishes the decision word of
+// the sequence.  The producers of the group wait for that word (bounded), then stream position
+// k + 1, or -- at the first rejection, or after the bonus row when everything passed -- the row
+// pair of the stop position again (it has just been read: L2) for the residual masses; the
+// finisher that completes that count runs the inverse CDF (level 2 of the resampling kernel).
+//
+// CTAs of one group wait for one another, so the kernel is launched cooperatively (all CTAs
+// resident).  Every wait is bounded; a wait that gives up sets the abort word and the CTA drains.
+#include "bs_verify_common.cuh"
+#include "bs_residual_level2.cuh"
+#include "bs_pipeline.cuh"
+
+namespace bs {
+
+constexpr int kWkWarps = 16;
+constexpr int kWkConsumers = kWkWarps * 32;
+constexpr int kWkThreads = kWkConsumers + 64;                    // + producer warp + finisher warp
+constexpr int kWkStages = 3;
+constexpr int kWkRing = 8;                                       // events the consumers may run ahead of the finisher
+constexpr int kWkVecPerThread = kSegBytes / 16 / kWkConsumers;   // 4
+static_assert(kSegBytes == 2 * kResSegBytes && kWkWarps == kRsWarps, "one stage holds a segment or a pair of half segments");
+
+constexpr int kItemStats = 0, kItemMass = 1, kItemEnd = 2;
+
+struct WalkParams {
+    VerifyParams v;        // logits, tokens, uniforms, outputs of the accept test, statistics and partials
+    ResidParams r;         // the same logits for the residual pass, its outputs, piece masses
+    uint32_t* dec;         // [B] decision word: (positions decided << 1) | last one accepted
+    int nG;                // CTAs per sequence
+};
+
+// Per-stage record, written by the producer.
+struct WkMeta {
+    int type, b, k;
+    int row;               // stats: 0 = target row k, 1 = draft row k;  mass: 1 = target row only (bonus)
+    int sg, nvec, flags;   // flags bit 0: first stage of a row piece, bit 1: last stage of a piece / of the CTA's share
+    float kt, kd;
+};
+// Per event handed to the finisher (written by consumer warp 0).
+struct WkEvent {
+    int type, b, k, row, first_sg, last_sg;
+};
+
+// Stats items counted on the sequence's ticket once position k is complete.
+__device__ __forceinline__ unsigned wk_cum(int k, int g, int nseg) {
+    return k < g ? (unsigned)(2 * nseg * (k + 1)) : (unsigned)(2 * nseg * g + nseg);
+}
+__device__ __forceinline__ unsigned ld_volatile_u32(const uint32_t* p) {
+    return *reinterpret_cast<const volatile uint32_t*>(p);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkParams p) {
+    extern __shared__ __align__(128) unsigned char ring[];    // kWkStages * 32 KB
+    __shared__ __align__(8) unsigned long long s_full[kWkStages];
+    __shared__ __align__(8) unsigned long long s_empty[kWkStages];
+    __shared__ __align__(8) unsigned long long s_evbar[kWkRing];
+    __shared__ __align__(8) unsigned long long s_evfree[kWkRing];
+    __shared__ WkMeta s_meta[kWkStages];
+    __shared__ WkEvent s_ev[kWkRing];
+    __shared__ float2 s_red[kWkRing][kWkWarps];
+    __shared__ float2 s_fin[2];
+
+    const VerifyParams& v = p.v;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int kVec = Elem<T>::kVec;
+
+    if (tid == 0) {
+        for (int s = 0; s < kWkStages; ++s) {
+            mbar_init(smem_u32(&s_full[s]), 1);
+            mbar_init(smem_u32(&s_empty[s]), kWkWarps);
+        }
+        for (int s = 0; s < kWkRing; ++s) {
+            mbar_init(smem_u32(&s_evbar[s]), kWkWarps);
+            mbar_init(smem_u32(&s_evfree[s]), 1);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    // sequences of this CTA: one (shared with nG - 1 other CTAs) or every gridDim.x-th
+    const int part = blockIdx.x % p.nG;
+    const int b_first = blockIdx.x / p.nG;
+    const int b_step = p.nG > 1 ? v.B : (int)gridDim.x;
+
+    if (warp == kWkWarps) {
+        // =============================== producer ===============================
+        if (lane != 0) return;
+        int slot = 0;
+        uint32_t ph = 0;
+        bool ok = true;
+        // one stage: wait for the slot, write the record, arm the barrier, copy
+        auto issue = [&](const WkMeta& m, const T* src0, const T* src1, uint32_t bytes) -> bool {
+            if (!mbar_wait(smem_u32(&s_empty[slot]), ph ^ 1u)) return false;
+            s_meta[slot] = m;
+            const uint32_t bar = smem_u32(&s_full[slot]);
+            const uint32_t dst = smem_u32(ring + (size_t)slot * kSegBytes);
+            if (m.type == kItemEnd) {
+                mbar_arrive(bar);                              // nothing to copy: the phase completes at once
+            } else {
+                mbar_arrive_expect_tx(bar, src1 ? 2u * bytes : bytes);
+                bulk_load(dst, src0, bytes, bar);
+                if (src1) bulk_load(dst + kResSegBytes, src1, bytes, bar);
+            }
+            if (++slot == kWkStages) { slot = 0; ph ^= 1u; }
+            return true;
+        };
+        for (int b = b_first; b < v.B && ok; b += b_step) {
+            const int g = clamp_gamma(v.gamma[b], v.Gmax);
+            for (int k = 0; ok; ++k) {
+                // ---- position k: target row k and, below gamma, draft row k ----
+                const int nrows = k < g ? 2 : 1;
+                const int items = nrows * v.nseg;
+                const int i0 = (int)((long long)items * part / p.nG), i1 = (int)((long long)items * (part + 1) / p.nG);
+                for (int i = i0; i < i1 && ok; ++i) {
+                    const int row = i / v.nseg, sg = i - row * v.nseg;
+                    const T* rowp = row == 0 ? row_ptr(static_cast<const T*>(v.target), b, v.Gmax + 1, k, v.V)
+                                             : row_ptr(static_cast<const T*>(v.draft), b, v.Gmax, k, v.V);
+                    const int e0 = sg * v.seg;
+                    const int n = min(v.seg, v.V - e0);
+                    WkMeta m;
+                    m.type = kItemStats; m.b = b; m.k = k; m.row = row; m.sg = sg; m.nvec = n / kVec;
+                    m.flags = ((sg == 0 || i == i0) ? 1 : 0) | ((sg == v.nseg - 1 || i == i1 - 1) ? 2 : 0);
+                    m.kt = m.kd = 0.f;
+                    ok = issue(m, rowp + e0, nullptr, (uint32_t)n * (uint32_t)sizeof(T));
+                }
+                if (!ok) break;
+                // ---- the decision for position k (made by whichever finisher of the group completes it) ----
+                unsigned d;
+                {
+                    const long long t0 = clock64();
+                    while (((d = ld_volatile_u32(p.dec + b)) >> 1) != (unsigned)(k + 1)) {
+                        if (clock64() - t0 > kWaitCycles) { ok = false; break; }
+                        __nanosleep(32);
+                    }
+                }
+                if (!ok) break;
+                __threadfence();
+                if (k < g && (d & 1u)) continue;               // accepted: on to the next position
+                // ---- stop at k: residual [P_k - Q_k]_+ (rejected) or the bonus row P_k (k == gamma) ----
+                const bool bonus = k >= g;
+                const T* tp = row_ptr(static_cast<const T*>(v.target), b, v.Gmax + 1, k, v.V);
+                const T* dp = bonus ? nullptr : row_ptr(static_cast<const T*>(v.draft), b, v.Gmax, k, v.V);
+                const float2 ts = __ldcg(v.row_stats + (size_t)b * v.R + k);
+                float kt = -(ts.x * v.c + log2f(ts.y)), kd = 0.f;
+                if (!bonus) {
+                    const float2 ds = __ldcg(v.row_stats + (size_t)b * v.R + v.Gmax + 1 + k);
+                    kd = -(ds.x * v.c + log2f(ds.y));
+                }
+                const int rseg = p.r.seg, rnseg = p.r.nseg;
+                const int j0 = (int)((long long)rnseg * part / p.nG), j1 = (int)((long long)rnseg * (part + 1) / p.nG);
+                for (int sg = j0; sg < j1 && ok; ++sg) {
+                    const int e0 = sg * rseg;
+                    const int n = min(rseg, v.V - e0);
+                    WkMeta m;
+                    m.type = kItemMass; m.b = b; m.k = k; m.row = bonus ? 1 : 0; m.sg = sg; m.nvec = n / kVec;
+                    m.flags = (sg == j0 ? 1 : 0) | (sg == j1 - 1 ? 2 : 0);
+                    m.kt = kt; m.kd = kd;
+                    ok = issue(m, tp + e0, bonus ? nullptr : dp + e0, (uint32_t)n * (uint32_t)sizeof(T));
+                }
+                break;                                          // this sequence is done for the producer
+            }
+        }
+        if (!ok) atomicExch(v.abort_flag, 1);
+        // the end marker lets the consumers and the finisher leave (also after a failed wait, if a slot frees up)
+        WkMeta e;
+        e.type = kItemEnd; e.b = 0; e.k = 0; e.row = 0; e.sg = 0; e.nvec = 0; e.flags = 2; e.kt = e.kd = 0.f;
+        issue(e, nullptr, nullptr, 0);
+        return;
+    }
+
+    if (warp == kWkWarps + 1) {
+        // =============================== finisher ===============================
+        for (int ev = 0;; ++ev) {
+            const int rs = ev % kWkRing;
+            if (!mbar_wait_warp(smem_u32(&s_evbar[rs]), (uint32_t)(ev / kWkRing) & 1u)) {
+                if (lane == 0) atomicExch(v.abort_flag, 1);
+                return;
+            }
+            const WkEvent e = s_ev[rs];
+            float2 mine = make_float2(-INFINITY, 0.f);
+            if (lane < kWkWarps) mine = s_red[rs][lane];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&s_evfree[rs]));   // the slot may be reused
+            if (e.type == kItemEnd) return;
+            const int b = e.b, k = e.k;
+            const int graw = v.gamma[b];
+            const int g = clamp_gamma(graw, v.Gmax);
+            const int len = e.last_sg - e.first_sg + 1;
+
+            if (e.type == kItemStats) {
+                // ---- a piece of target row k (row 0) or draft row k (row 1) ----
+                const float2 out = warp_merge(Online{mine.x, mine.y}, v.c);
+                const int slot_r = e.row == 0 ? k : v.Gmax + 1 + k;
+                float2* pp = v.partial + ((size_t)b * v.R + slot_r) * v.S;
+                for (int q = e.first_sg + lane; q <= e.last_sg; q += 32)
+                    pp[q] = (q == e.first_sg) ? out : make_float2(-INFINITY, 0.f);
+                // the loads of the accept test do not depend on the statistics: start them now
+                int x = 0;
+                float tl = 0.f, dl = 0.f, u = 2.f;
+                bool bad = false;
+                if (k < g) {
+                    x = v.tokens[(size_t)b * v.Gmax + k];
+                    bad = x < 0 || x >= v.V;
+                    if (!bad) {
+                        tl = Elem<T>::load(row_ptr(static_cast<const T*>(v.target), b, v.Gmax + 1, k, v.V) + x);
+                        dl = Elem<T>::load(row_ptr(static_cast<const T*>(v.draft), b, v.Gmax, k, v.V) + x);
+                        u = v.u_accept[(size_t)b * v.Gmax + k];
+                    }
+                }
+                __threadfence();
+                __syncwarp();
+                unsigned old = 0;
+                if (lane == 0) old = atomicAdd(v.ticket + b, (unsigned)len);
+                old = __shfl_sync(0xffffffffu, old, 0);
+                if (old + (unsigned)len != wk_cum(k, g, v.nseg)) continue;
+                // ---- position k is complete: merge its rows (lane 0: target, lane 1: draft), decide ----
+                __threadfence();
+                const int nrows = k < g ? 2 : 1;
+                if (lane < nrows) {
+                    const int rr = lane == 0 ? k : v.Gmax + 1 + k;
+                    const float2* qq = v.partial + ((size_t)b * v.R + rr) * v.S;
+                    Online o{-INFINITY, 0.f};
+#pragma unroll 4
+                    for (int q = 0; q < v.nseg; ++q) {
+                        const float2 t = __ldcg(qq + q);
+                        o.merge(t.x, t.y, v.c);
+                    }
+                    s_fin[lane] = make_float2(o.m, o.s);
+                    v.row_stats[(size_t)b * v.R + rr] = make_float2(o.m, o.s);
+                }
+                __syncwarp();
+                const float2 ts = s_fin[0];
+                int bits = (k == 0 && graw != g) ? BS_DEV_BAD_GAMMA : 0;
+                if (!(ts.y > 0.f) || !isfinite(ts.y) || !isfinite(ts.x)) bits |= BS_DEV_NONFINITE;
+                bool acc = false;
+                float pj = 0.f, qj = 0.f;
+                if (k < g) {
+                    const float2 ds = s_fin[1];
+                    if (!(ds.y > 0.f) || !isfinite(ds.y) || !isfinite(ds.x)) bits |= BS_DEV_NONFINITE;
+                    if (bad) {
+                        bits |= BS_DEV_BAD_TOKEN;
+                    } else {
+                        // log2 of the two probabilities; the ratio is formed in the log domain
+                        const float lp = (tl - ts.x) * v.c - log2f(ts.y);
+                        const float lq = (dl - ds.x) * v.c - log2f(ds.y);
+                        pj = exp2f(lp);
+                        qj = exp2f(lq);
+                        // r <= min{1, P/Q}; Q(x) = 0 counts as an infinite ratio
+                        acc = (lq == -INFINITY) ? true : (u <= fminf(1.f, exp2f(lp - lq)));
+                    }
+                }
+                if (lane == 0) {
+                    if (k < g) {
+                        if (v.p_tok) v.p_tok[(size_t)b * v.Gmax + k] = pj;
+                        if (v.q_tok) v.q_tok[(size_t)b * v.Gmax + k] = qj;
+                    }
+                    if (k == 0) v.status[b] = bits; else if (bits) atomicOr(v.status + b, bits);
+                    if (!acc) v.accept_len[b] = k;             // first rejection, or k == gamma: everything passed
+                }
+                if (!acc) {                                    // positions behind the stop were not looked at
+                    for (int j = (k < g ? k + 1 : k) + lane; j < v.Gmax; j += 32) {
+                        if (v.p_tok) v.p_tok[(size_t)b * v.Gmax + j] = 0.f;
+                        if (v.q_tok) v.q_tok[(size_t)b * v.Gmax + j] = 0.f;
+                    }
+                }
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) atomicExch(p.dec + b, ((unsigned)(k + 1) << 1) | (acc ? 1u : 0u));
+            } else {
+                // ---- this CTA's share of the residual masses of the stop position k is written ----
+                __threadfence();
+                unsigned old = 0;
+                if (lane == 0) old = atomicAdd(p.r.ticket + b, (unsigned)len);
+                old = __shfl_sync(0xffffffffu, old, 0);
+                if (old + (unsigned)len != (unsigned)p.r.nseg) continue;
+                __threadfence();
+                RsSeq sq;
+                sq.tau = k; sq.bonus = k >= g; sq.wgt = sq.bonus ? 1 : 2;
+                MassFn f;
+                f.c = v.c; f.bonus = sq.bonus != 0;
+                const float2 ts = __ldcg(v.row_stats + (size_t)b * v.R + k);
+                f.kt = -(ts.x * v.c + log2f(ts.y));
+                f.kd = 0.f;
+                if (!f.bonus) {
+                    const float2 ds = __ldcg(v.row_stats + (size_t)b * v.R + v.Gmax + 1 + k);
+                    f.kd = -(ds.x * v.c + log2f(ds.y));
+                }
+                rs_level2<T>(p.r, b, sq, f);                   // token, out_tokens, out_len; clears the mass ticket
+                if (lane == 0) {                               // leave the workspace clean for the next call
+                    v.ticket[b] = 0u;
+                    p.dec[b] = 0u;
+                }
+            }
+        }
+    }
+
+    // ================================= consumers =================================
+    Online on{-INFINITY, 0.f};
+    int first_sg = 0;
+    int ev = 0;                                               // events posted by this CTA
+    int slot = 0;
+    uint32_t ph = 0;
+    for (;;) {
+        if (!mbar_wait_warp(smem_u32(&s_full[slot]), ph)) { atomicExch(v.abort_flag, 1); return; }
+        const WkMeta m = s_meta[slot];
+        const uint32_t base = smem_u32(ring + (size_t)slot * kSegBytes);
+        if (m.flags & 1) first_sg = m.sg;
+        float2 wr = make_float2(-INFINITY, 0.f);
+        if (m.type == kItemStats) {
+            // one 32 KB segment of one row: online softmax statistics, one exp per logit
+            uint4 x[kWkVecPerThread];
+#pragma unroll
+            for (int q = 0; q < kWkVecPerThread; ++q)
+                x[q] = (q * kWkConsumers + tid < m.nvec) ? lds128(base + (uint32_t)(q * kWkConsumers + tid) * 16u)
+                                                         : neg_inf_vec<T>();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&s_empty[slot]));
+            online_add<T, kWkVecPerThread>(on, x, v.c);
+            if (m.flags & 2) {
+                wr = warp_merge(on, v.c);
+                on = Online{-INFINITY, 0.f};
+            }
+        } else if (m.type == kItemMass) {
+            // a 16 KB segment of the row pair: warp w owns the w-th 1 KB piece and writes its mass
+            MassFn f;
+            f.c = v.c; f.kt = m.kt; f.kd = m.kd; f.bonus = m.row != 0;
+            const uint32_t pb = base + (uint32_t)(warp * kRsPieceBytes + lane * 16);
+            uint4 a[kRsVecPerLane], d[kRsVecPerLane];
+            bool valid[kRsVecPerLane];
+#pragma unroll
+            for (int q = 0; q < kRsVecPerLane; ++q) {
+                valid[q] = warp * kRsPieceVecs + q * 32 + lane < m.nvec;
+                if (valid[q]) {
+                    a[q] = lds128(pb + (uint32_t)(q * 512));
+                    d[q] = f.bonus ? a[q] : lds128(pb + (uint32_t)(kResSegBytes + q * 512));
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&s_empty[slot]));
+            float acc = 0.f;
+#pragma unroll
+            for (int q = 0; q < kRsVecPerLane; ++q) {
+                if (valid[q]) {
+                    float r[kVec];
+                    RsElems<T>::masses(a[q], d[q], f, r);
+                    float vs = 0.f;
+#pragma unroll
+                    for (int i = 0; i < kVec; ++i) vs += r[i];
+                    acc += vs;
+                }
+            }
+            acc = warp_sum(acc);
+            if (lane == 0) {
+                p.r.resid_partial[(size_t)m.b * p.r.S + m.sg * kRsWarps + warp] = acc;
+                if (m.flags & 2) __threadfence();             // the share's masses are visible before the event
+            }
+        } else {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&s_empty[slot]));
+        }
+        if (++slot == kWkStages) { slot = 0; ph ^= 1u; }
+
+        if (m.flags & 2) {
+            // ---- end of a row piece / of the share / of the work: one event for the finisher ----
+            const int rs = ev % kWkRing;
+            if (ev >= kWkRing && !mbar_wait_warp(smem_u32(&s_evfree[rs]), (uint32_t)(ev / kWkRing - 1) & 1u)) {
+                atomicExch(v.abort_flag, 1);
+                return;
+            }
+            if (lane == 0) {
+                s_red[rs][warp] = wr;
+                if (warp == 0) s_ev[rs] = WkEvent{m.type, m.b, m.k, m.row, first_sg, m.sg};
+                mbar_arrive(smem_u32(&s_evbar[rs]));          // release: the writes above are visible to the finisher
+            }
+            ++ev;
+            if (m.type == kItemEnd) return;
+        }
+    }
+}
+
+static int g_wk_blocks[2][64];        // resident CTAs per SM (0 = not queried)
+
+template <typename T>
+static bs_status launch_walk(WalkParams& p, cudaStream_t st) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64) dev = 0;
+    const int variant = Elem<T>::kDtype == BS_F32 ? 0 : 1;
+    const size_t smem = (size_t)kWkStages * kSegBytes;
+    if (!g_wk_blocks[variant][dev]) {
+        if (cudaFuncSetAttribute(verify_walk_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+            cudaSuccess)
+            return cuda_status(cudaGetLastError());
+        int nb = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_walk_kernel<T>, kWkThreads, smem) != cudaSuccess)
+            return cuda_status(cudaGetLastError());
+        if (nb < 1) return BS_ERR_UNSUPPORTED;
+        g_wk_blocks[variant][dev] = nb > 2 ? 2 : nb;
+    }
+    // groups of CTAs wait for one another: never more CTAs than can be resident together
+    const int max_grid = g_wk_blocks[variant][dev] * sm_count();
+    int nG = max_grid / p.v.B;
+    if (nG > p.v.nseg) nG = p.v.nseg;                        // every CTA of a group gets a segment of every row
+    if (nG < 1) nG = 1;
+    p.nG = nG;
+    const int grid = nG > 1 ? p.v.B * nG : (p.v.B < max_grid ? p.v.B : max_grid);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kWkThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeCooperative;
+    at[0].val.cooperative = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cuda_status(cudaLaunchKernelEx(&cfg, verify_walk_kernel<T>, p));
+}
+
+}  // namespace bs
+
+using namespace bs;
+
+extern "C" bs_status bs_verify_walk(const void* target_logits, const void* draft_logits, bs_dtype dtype,
+                                    const int32_t* draft_tokens, const int32_t* gamma, const float* u_accept,
+                                    const float* u_resample, float temperature, int B, int Gmax, int V,
+                                    int32_t* accept_len, float* p_tok, float* q_tok, int32_t* out_tokens,
+                                    int32_t* out_len, void* workspace, size_t workspace_bytes, void* stream) {
+    if (B < 1 || Gmax < 0 || V < 1) return BS_ERR_INVALID_ARG;
+    if (B > BS_MAX_BATCH || Gmax > BS_MAX_GAMMA || V > BS_MAX_VOCAB) return BS_ERR_UNSUPPORTED;
+    if (dtype != BS_F32 && dtype != BS_BF16) return BS_ERR_INVALID_ARG;
+    if (!(temperature >= 0.f) || !isfinite(temperature)) return BS_ERR_INVALID_ARG;
+    if (temperature == 0.f) return BS_ERR_UNSUPPORTED;       // greedy rounds: bs_softmax_verify + bs_residual_sample
+    if (!target_logits || !gamma || !accept_len || !out_tokens || !out_len || !u_resample || !workspace)
+        return BS_ERR_INVALID_ARG;
+    if (Gmax > 0 && (!draft_tokens || !draft_logits || !u_accept)) return BS_ERR_INVALID_ARG;
+    const size_t es = dtype == BS_F32 ? 4 : 2;
+    if (((size_t)V * es) % 16 != 0 || (reinterpret_cast<uintptr_t>(target_logits) & 15) ||
+        (reinterpret_cast<uintptr_t>(draft_logits) & 15))
+        return BS_ERR_UNSUPPORTED;                           // rows must start on 16-byte boundaries
+    const Workspace w = workspace_layout(B, Gmax, V);
+    if (workspace_bytes < w.total || (reinterpret_cast<uintptr_t>(workspace) & 255)) return BS_ERR_WORKSPACE;
+
+    char* ws = static_cast<char*>(workspace);
+    WalkParams p;
+    VerifyParams& v = p.v;
+    v.target = target_logits; v.draft = draft_logits; v.tokens = draft_tokens; v.gamma = gamma;
+    v.u_accept = u_accept; v.accept_len = accept_len; v.p_tok = p_tok; v.q_tok = q_tok;
+    v.ticket = reinterpret_cast<uint32_t*>(ws + w.off_ticket_verify);
+    v.ticket_row = reinterpret_cast<uint32_t*>(ws + w.off_ticket_row);
+    v.status = reinterpret_cast<int32_t*>(ws + w.off_status);
+    v.abort_flag = reinterpret_cast<int32_t*>(ws + w.off_abort);
+    v.row_stats = reinterpret_cast<float2*>(ws + w.off_row_stats);
+    v.partial = reinterpret_cast<float2*>(ws + w.off_partial);
+    v.B = B; v.Gmax = Gmax; v.V = V; v.R = w.R; v.S = w.S;
+    v.seg = seg_elems(dtype);
+    v.nseg = div_up(V, v.seg);
+    v.c = kLog2e / temperature;
+    v.mode = kModeVerify; v.position = 0; v.draft_ready = v.ticket_row; v.draft_out = nullptr;
+    ResidParams& r = p.r;
+    r.target = target_logits; r.draft = draft_logits; r.tokens = draft_tokens; r.gamma = gamma;
+    r.accept_len = accept_len; r.u_resample = u_resample; r.out_tokens = out_tokens; r.out_len = out_len;
+    r.ticket = reinterpret_cast<uint32_t*>(ws + w.off_ticket_resid);
+    r.status = v.status;
+    r.abort_flag = v.abort_flag;
+    r.row_stats = v.row_stats;
+    r.resid_partial = reinterpret_cast<float*>(ws + w.off_resid_partial);
+    r.B = B; r.Gmax = Gmax; r.V = V; r.R = w.R; r.S = w.Sr;
+    r.seg = res_seg_elems(dtype);
+    r.nseg = div_up(V, r.seg);
+    r.c = v.c;
+    r.mode = kResidVerify; r.position = 0; r.draft_out = nullptr;
+    // decision words: the second B words of the per-row counter slot (the first B mark drafted positions)
+    p.dec = v.ticket_row + B;
+    p.nG = 1;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return dtype == BS_F32 ? launch_walk<float>(p, st) : launch_walk<__nv_bfloat16>(p, st);
+}

@@ -55,17 +55,21 @@ def to_np(t: torch.Tensor) -> np.ndarray:
 
 def check_sequence(ref: ov.SequenceResult, tau_gpu: int, out_tokens_gpu: np.ndarray, out_len_gpu: int,
                    p_gpu: np.ndarray, q_gpu: np.ndarray, *, target_rows, draft_rows, tokens, gamma: int,
-                   u_accept, u_resample: float, temperature: float, tally: Tally, where="") -> ov.SequenceResult:
-    """Checks one sequence; returns the oracle result the trajectory should continue from."""
+                   u_accept, u_resample: float, temperature: float, tally: Tally, where="",
+                   walk: bool = False) -> ov.SequenceResult:
+    """Checks one sequence; returns the oracle result the trajectory should continue from.
+    walk: the early-exit path examines positions up to the first rejection only, so its token
+    probabilities are compared there and must be zero behind it."""
     G1 = len(out_tokens_gpu)
     tally.sequences += 1
     tally.positions += gamma
     greedy = temperature == 0.0
-    if not greedy and gamma:
-        err = max(np.abs(p_gpu[:gamma] - ref.p_tok).max(), np.abs(q_gpu[:gamma] - ref.q_tok).max())
+    seen = min(tau_gpu + 1, gamma) if walk else gamma            # positions whose probabilities were formed
+    if not greedy and seen:
+        err = max(np.abs(p_gpu[:seen] - ref.p_tok[:seen]).max(), np.abs(q_gpu[:seen] - ref.q_tok[:seen]).max())
         tally.max_p_err = max(tally.max_p_err, float(err))
         assert err <= P_TOL, f"{where}: token probability off by {err}"
-    assert (p_gpu[gamma:] == 0).all() and (q_gpu[gamma:] == 0).all(), f"{where}: padded p/q not zero"
+    assert (p_gpu[seen:] == 0).all() and (q_gpu[seen:] == 0).all(), f"{where}: padded p/q not zero"
     if tau_gpu != ref.tau:
         j = min(tau_gpu, ref.tau)                      # first position where the decisions differ
         assert not greedy, f"{where}: greedy accept_len {tau_gpu} != {ref.tau}"
@@ -98,7 +102,7 @@ def check_sequence(ref: ov.SequenceResult, tau_gpu: int, out_tokens_gpu: np.ndar
 
 
 def check_round(out, rnd: wl.RoundInputs, temperature: float, tally: Tally,
-                seqs: Optional[Sequence[int]] = None, where="") -> List[Optional[ov.SequenceResult]]:
+                seqs: Optional[Sequence[int]] = None, where="", walk: bool = False) -> List[Optional[ov.SequenceResult]]:
     """Compares a RoundOutput with the oracle on the sequences `seqs` (default: all)."""
     B = rnd.target.shape[0]
     seqs = range(B) if seqs is None else seqs
@@ -115,7 +119,7 @@ def check_round(out, rnd: wl.RoundInputs, temperature: float, tally: Tally,
         res[b] = check_sequence(ref, int(tau[b]), ot[b], int(ol[b]), pg[b], qg[b],
                                 target_rows=t_rows, draft_rows=d_rows, tokens=toks[b], gamma=g,
                                 u_accept=rnd.uniforms.u_accept[b], u_resample=float(rnd.uniforms.u_resample[b]),
-                                temperature=temperature, tally=tally, where=f"{where} b={b}")
+                                temperature=temperature, tally=tally, where=f"{where} b={b}", walk=walk)
     return res
 
 

@@ -1,0 +1,107 @@
+"""bs_verify_walk (verification with early exit + resampling in one launch) against the CPU oracle,
+through the C ABI (needs a B200).  Same rules as the two-call path: accepted lengths and tokens
+bit-exact except at flagged near-ties, probabilities of the examined positions within 1e-5."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2505_15141_b200 import workloads as wl
+import parity
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _round(rng, B, G, V, dtype, T, sigma=1.0, gamma=None, std=3.0):
+    g = torch.Generator(device="cpu"); g.manual_seed(int(rng.integers(1 << 30)))
+    t = torch.randn(B, G + 1, V, generator=g) * std
+    d = t[:, :G] + sigma * torch.randn(B, G, V, generator=g)
+    t, d = t.to(dtype).to(DEV), d.to(dtype).to(DEV)
+    gamma = rng.integers(0, G + 1, size=B).astype(np.int32) if gamma is None else np.asarray(gamma, np.int32)
+    un = wl.RoundUniforms(rng.random((B, G)).astype(np.float32) * 0.999 + 0.0005,
+                          rng.random(B).astype(np.float32) * 0.999 + 0.0005,
+                          rng.random(B).astype(np.float32), rng.random((B, G)).astype(np.float32) * 0.999 + 0.0005)
+    tok = wl.draw_draft_tokens(d, T, un.u_draft)
+    return wl.RoundInputs(target=t, draft=d, tokens=tok.contiguous(), gamma=gamma, uniforms=un)
+
+
+def _walk(lib, rnd, T, ws=None):
+    dev = rnd.target.device
+    out = lib.verify_round_walk(rnd.target, rnd.draft, rnd.tokens,
+                                torch.as_tensor(np.asarray(rnd.gamma, np.int32), device=dev),
+                                torch.as_tensor(rnd.uniforms.u_accept, device=dev),
+                                torch.as_tensor(rnd.uniforms.u_resample, device=dev), T, workspace=ws)
+    torch.cuda.synchronize()
+    return out
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("B,G,V", [(5, 4, 1000), (3, 6, 40000), (40, 3, 8200), (700, 2, 256), (2, 8, 128256)])
+def test_walk_parity(lib, dtype, B, G, V):
+    """One CTA per sequence, several CTAs per sequence, several sequences per CTA; one and many segments."""
+    rng = np.random.default_rng(B * 7 + V)
+    tally = parity.Tally()
+    for T in (1.0, 0.6):
+        rnd = _round(rng, B, G, V, dtype, T, sigma=0.7)
+        out = _walk(lib, rnd, T)
+        st = lib.bs_get_device_status(out.workspace, B, G, V)
+        assert (st & ~lib.BS_DEV_RESIDUAL_FALLBACK == 0).all(), st
+        seqs = range(B) if B <= 64 else list(range(0, B, 23))
+        parity.check_round(out, rnd, T, tally, seqs=seqs, where=f"walk B={B} V={V} T={T}", walk=True)
+        y = out.out_len.cpu().numpy(); tau = out.accept_len.cpu().numpy()
+        assert ((y == tau + 1) & (tau >= 0) & (tau <= rnd.gamma)).all()
+    assert tally.flagged_accept + tally.flagged_token <= 2 + tally.sequences // 100
+
+
+def test_walk_edge_cases_and_reuse(lib):
+    rng = np.random.default_rng(17)
+    B, G, V = 8, 6, 3000
+    rnd = _round(rng, B, G, V, torch.float32, 1.0, gamma=[0, G, G, G, 3, 3, 2, 1])
+    rnd.draft[2] = rnd.target[2, :G]                                     # q == p: everything passes, bonus row
+    rnd.draft[3] = -rnd.target[3, :G] * 3                                # far apart: stops at once
+    rnd.target[5] = 1.25; rnd.draft[5] = -0.5                            # constant rows
+    rnd.tokens = wl.draw_draft_tokens(rnd.draft, 1.0, rnd.uniforms.u_draft).contiguous()
+    ws = lib.new_workspace(B, G, V, DEV)
+    tally = parity.Tally()
+    out = _walk(lib, rnd, 1.0, ws)
+    refs = parity.check_round(out, rnd, 1.0, tally, where="walk edge", walk=True)
+    assert refs[0].y == 1 and refs[2].tau == G and refs[3].tau <= 1
+    # the same workspace again, and then the two-call path on it: counters were left clean
+    out2 = _walk(lib, rnd, 1.0, ws)
+    assert torch.equal(out.out_tokens, out2.out_tokens) and torch.equal(out.p_tok, out2.p_tok)
+    out3 = parity.gpu_round(lib, rnd, 1.0, ws)
+    assert torch.equal(out3.accept_len, out.accept_len) and torch.equal(out3.out_tokens, out.out_tokens)
+    # data errors are reported, not fatal
+    rnd.tokens[4, 1] = V + 3
+    rnd.gamma = np.array([0, G, G, G, 3, 3, 99, 1], np.int32)
+    out4 = _walk(lib, rnd, 1.0, ws)
+    st = lib.bs_get_device_status(ws, B, G, V)
+    assert st[4] & lib.BS_DEV_BAD_TOKEN and int(out4.accept_len[4]) <= 1
+    assert st[6] & lib.BS_DEV_BAD_GAMMA and int(out4.out_len[6]) == 1
+    parity.check_round(out4, rnd, 1.0, tally, seqs=[0, 1, 2, 3, 5, 7], where="walk after errors", walk=True)
+    # greedy and unaligned rows are refused on the host
+    with pytest.raises(lib.BanditSpecError) as e:
+        _walk(lib, rnd, 0.0, ws)
+    assert e.value.code == lib.BS_ERR_UNSUPPORTED
+
+
+def test_walk_full_size(lib):
+    """The launch configurations the benchmark times: 64 x 128256 bf16 (four CTAs per sequence) and
+    256 x 152064 fp32 (one CTA per sequence); sampled sequences against the oracle, all against
+    the invariants, and accepted lengths against the two-call path."""
+    for name, sample in (("llama3_ucb", [0, 1, 17, 40, 63]), ("qwen_exp3", [0, 100, 255])):
+        w = wl.WORKLOADS[name]
+        arm = np.arange(w.B) % w.K
+        rnd = wl.make_round(w, 7, arm, device=DEV)
+        out = _walk(lib, rnd, w.temperature)
+        st = lib.bs_get_device_status(out.workspace, w.B, w.Gmax, w.V)
+        assert (st & ~lib.BS_DEV_RESIDUAL_FALLBACK == 0).all()
+        tally = parity.Tally()
+        parity.check_round(out, rnd, w.temperature, tally, seqs=sample, where=f"walk {name}", walk=True)
+        ref = parity.gpu_round(lib, rnd, w.temperature)
+        same = (ref.accept_len == out.accept_len).cpu().numpy()
+        assert same.mean() > 0.98                    # the two paths merge statistics in different orders: near-ties only
+        y = out.out_len.cpu().numpy(); tau = out.accept_len.cpu().numpy(); ot = out.out_tokens.cpu().numpy()
+        assert ((y == tau + 1) & (tau <= rnd.gamma)).all()
+        for b in range(w.B):
+            assert 0 <= ot[b, tau[b]] < w.V and (ot[b, y[b]:] == -1).all()
