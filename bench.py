@@ -70,6 +70,9 @@ def parse_args():
     ap.add_argument("--drafted", action="store_true",
                     help="the round with drafting on the device: select -> bs_draft_sample per position -> "
                          "bs_softmax_verify_drafted -> bs_residual_sample -> update")
+    ap.add_argument("--walk", action="store_true",
+                    help="the round with early exit: select -> bs_verify_walk (verification up to the first "
+                         "rejection + resampling in one launch) -> update")
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="budget of the CPU-oracle sample")
@@ -286,8 +289,18 @@ def run_cuda(args, w):
         for j in range(G):
             bs.bs_draft_sample(s["draft"], j, gamma_d, s["u_draft"], w.temperature, tok_d, ws)
 
+    walk = args.walk
+
+    def walk_call(s):
+        bs.bs_verify_walk(s["target"], s["draft"], s["tokens"], gamma_d, s["u_accept"], s["u_resample"],
+                          w.temperature, accept_len, p_tok, q_tok, out_tokens, out_len, ws)
+
     def step_calls(s):
         bs.bs_bandit_select(state, alg, B, K, s["u_arm"], None, arm_d, gamma_d)
+        if walk:
+            walk_call(s)
+            bs.bs_bandit_update(state, alg, B, K, arm_d, out_len)
+            return
         if drafted:
             draft_calls(s)
             s = dict(s, tokens=tok_d)
@@ -360,6 +373,7 @@ def run_cuda(args, w):
     evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(ksteps)]
     rsd = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(ksteps)]
     dft = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(ksteps)]
+    walk_rows = torch.zeros((), dtype=torch.int64, device=dev)
     nk0 = pulls()
     for i in range(ksteps):
         s = sets[(args.warmup + args.steps + i) % ring]
@@ -370,12 +384,19 @@ def run_cuda(args, w):
             dft[i][1].record(stream)
             s = dict(s, tokens=tok_d)
         evs[i][0].record(stream)
-        verify_call(s)
+        if walk:
+            walk_call(s)
+        else:
+            verify_call(s)
         evs[i][1].record(stream)
         rsd[i][0].record(stream)
-        bs.bs_residual_sample(s["target"], s["draft"], s["tokens"], gamma_d, accept_len, s["u_resample"],
-                              w.temperature, out_tokens, out_len, ws)
+        if not walk:
+            bs.bs_residual_sample(s["target"], s["draft"], s["tokens"], gamma_d, accept_len, s["u_resample"],
+                                  w.temperature, out_tokens, out_len, ws)
         rsd[i][1].record(stream)
+        if walk:                                               # rows the walk had to read: up to the stop position
+            tau = accept_len.to(torch.int64); gm = gamma_d.to(torch.int64)
+            walk_rows += torch.where(tau < gm, 2 * (tau + 1), 2 * gm + 1).sum()
         bs.bs_bandit_update(state, alg, B, K, arm_d, out_len)
         y_sum += out_len.sum()
     torch.cuda.synchronize()
@@ -383,6 +404,9 @@ def run_cuda(args, w):
     resid_ms = sum(a.elapsed_time(b) for a, b in rsd) / ksteps
     dk = pulls() - nk0
     verify_bytes = float((dk * rows_per_gamma[None, :]).sum()) * V * es / ksteps   # per launch
+    full_bytes = verify_bytes
+    if walk:
+        verify_bytes = float(walk_rows.item()) * V * es / ksteps
     draft_ms = sum(a.elapsed_time(b) for a, b in dft) / ksteps if drafted else None
     draft_bytes = float((dk * arm_gamma[None, :]).sum()) * V * es / ksteps if drafted else None
     mean_y = float(y_sum.item()) / (B * ksteps)
@@ -454,7 +478,8 @@ def run_cuda(args, w):
                        "logits_dtype": w.dtype, "temperature": w.temperature,
                        "l2": f"ring of {ring} input sets, {ring * set_bytes / 1e6:.0f} MB > 2 x L2",
                        "launch": "one CUDA graph per step" if graphs else "direct launches",
-                       "path": ("select, draft x Gmax, verify on drafted statistics, resample, update"
+                       "path": ("select, verify with early exit + resample in one launch, update" if walk else
+                                "select, draft x Gmax, verify on drafted statistics, resample, update"
                                 if drafted else "select, verify, resample, update"),
                        "multi_gpu": "one independent batch per rank, no collective on the data path"},
             "tokens_per_s": mean_y * B * value,
@@ -465,8 +490,14 @@ def run_cuda(args, w):
                          "traffic": ncu_traffic(w.name, verify_bytes), "bytes_per_launch": verify_bytes,
                          "ms_per_launch": verify_ms, "residual_ms_per_launch": resid_ms},
             "e2e": e2e, "cpu_baseline": cpu, "clocks": clocks,
-            "gpu_launches": (4 + (2 * G if drafted else 0)) * args.steps,
+            "gpu_launches": (3 if walk else 4 + (2 * G if drafted else 0)) * args.steps,
         }
+        if walk:
+            line["roofline"]["kernel"] = "verify_walk_kernel (bs_verify_walk)"
+            line["roofline"]["traffic"] = None
+            line["early_exit"] = {"bytes_per_launch": verify_bytes, "bytes_without_early_exit": full_bytes,
+                                  "note": "rows up to the stop position only; the second pass over the stop "
+                                          "position's rows (mostly L2) is not credited"}
         if drafted:
             line["drafting"] = {"ms_per_round": draft_ms, "calls": G, "row_bytes_per_round": draft_bytes,
                                 "note": "each call reads its draft rows once for the statistics and once more "

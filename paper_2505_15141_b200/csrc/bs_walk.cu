@@ -2,9 +2,9 @@
 // order -- position after position, stopping at the first rejection ("break"), so the rows behind
 // the first rejected draft are never read.
 //
-// Every sequence belongs to a fixed group of CTAs (nG = CTAs / B of them, 1 when there are more
-// sequences than CTAs, which then take several sequences each, one after the other).  For
-// position k the group streams target row k and draft row k (bulk async copies into a ring of
+// Every sequence is shared by a fixed group of nG CTAs (up to 8), and every CTA holds a share of
+// several sequences and interleaves them, so that a sequence with a long run of accepted drafts
+// keeps a slice of many CTAs busy rather than one CTA alone.  For position k the group streams target row k and draft row k (bulk async copies into a ring of
 // 32 KB stages, 16 consumer warps, online softmax: the pipeline of the row-statistics kernel),
 // every CTA its contiguous share of the 2 * nseg segments.  A finisher warp per CTA publishes the
 // pieces and counts them on the sequence's ticket; the finisher that completes position k merges
@@ -50,6 +50,12 @@ struct WkMeta {
 struct WkEvent {
     int type, b, k, row, first_sg, last_sg;
 };
+// A sequence in the producer's table: its share, the position it is at, and what it is waiting for.
+struct WkSeq {
+    int b, part, k, g;
+    int stage;             // 0: position k to be streamed, 1: waiting for its decision, 2: done
+};
+constexpr int kWkMaxSeqs = 32;
 
 // Stats items counted on the sequence's ticket once position k is complete.
 __device__ __forceinline__ unsigned wk_cum(int k, int g, int nseg) {
@@ -70,6 +76,7 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
     __shared__ WkEvent s_ev[kWkRing];
     __shared__ float2 s_red[kWkRing][kWkWarps];
     __shared__ float2 s_fin[2];
+    __shared__ WkSeq s_seq[kWkMaxSeqs];
 
     const VerifyParams& v = p.v;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -88,13 +95,11 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
     }
     __syncthreads();
 
-    // sequences of this CTA: one (shared with nG - 1 other CTAs) or every gridDim.x-th
-    const int part = blockIdx.x % p.nG;
-    const int b_first = blockIdx.x / p.nG;
-    const int b_step = p.nG > 1 ? v.B : (int)gridDim.x;
-
     if (warp == kWkWarps) {
         // =============================== producer ===============================
+        // This CTA holds one share (part of nG) of several sequences: pair q = b * nG + part belongs
+        // to CTA q % gridDim.x.  The producer keeps all of them moving: it streams whatever is
+        // ready and only sleeps when every one of its sequences is waiting for a decision.
         if (lane != 0) return;
         int slot = 0;
         uint32_t ph = 0;
@@ -115,60 +120,86 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
             if (++slot == kWkStages) { slot = 0; ph ^= 1u; }
             return true;
         };
-        for (int b = b_first; b < v.B && ok; b += b_step) {
-            const int g = clamp_gamma(v.gamma[b], v.Gmax);
-            for (int k = 0; ok; ++k) {
-                // ---- position k: target row k and, below gamma, draft row k ----
-                const int nrows = k < g ? 2 : 1;
-                const int items = nrows * v.nseg;
-                const int i0 = (int)((long long)items * part / p.nG), i1 = (int)((long long)items * (part + 1) / p.nG);
-                for (int i = i0; i < i1 && ok; ++i) {
-                    const int row = i / v.nseg, sg = i - row * v.nseg;
-                    const T* rowp = row == 0 ? row_ptr(static_cast<const T*>(v.target), b, v.Gmax + 1, k, v.V)
-                                             : row_ptr(static_cast<const T*>(v.draft), b, v.Gmax, k, v.V);
-                    const int e0 = sg * v.seg;
-                    const int n = min(v.seg, v.V - e0);
-                    WkMeta m;
-                    m.type = kItemStats; m.b = b; m.k = k; m.row = row; m.sg = sg; m.nvec = n / kVec;
-                    m.flags = ((sg == 0 || i == i0) ? 1 : 0) | ((sg == v.nseg - 1 || i == i1 - 1) ? 2 : 0);
-                    m.kt = m.kd = 0.f;
-                    ok = issue(m, rowp + e0, nullptr, (uint32_t)n * (uint32_t)sizeof(T));
-                }
-                if (!ok) break;
-                // ---- the decision for position k (made by whichever finisher of the group completes it) ----
-                unsigned d;
-                {
-                    const long long t0 = clock64();
-                    while (((d = ld_volatile_u32(p.dec + b)) >> 1) != (unsigned)(k + 1)) {
-                        if (clock64() - t0 > kWaitCycles) { ok = false; break; }
-                        __nanosleep(32);
+        const int npairs = v.B * p.nG;
+        int nmine = 0;
+        for (int q = blockIdx.x; q < npairs && nmine < kWkMaxSeqs; q += gridDim.x) {
+            const int b = q / p.nG;
+            s_seq[nmine++] = WkSeq{b, q - b * p.nG, 0, clamp_gamma(v.gamma[b], v.Gmax), 0};
+        }
+        int alive = nmine;
+        long long t_last = clock64();
+        while (alive > 0 && ok) {
+            bool progress = false;
+            for (int si = 0; si < nmine && ok; ++si) {
+                WkSeq sq = s_seq[si];
+                if (sq.stage == 2) continue;
+                const int b = sq.b, g = sq.g, part = sq.part;
+                if (sq.stage == 1) {
+                    // ---- has position k been decided (by whichever finisher of the group completed it)? ----
+                    const unsigned d = ld_volatile_u32(p.dec + b);
+                    if ((d >> 1) != (unsigned)(sq.k + 1)) continue;
+                    __threadfence();
+                    progress = true;
+                    if (sq.k < g && (d & 1u)) {                // accepted: on to the next position
+                        sq.k += 1;
+                        sq.stage = 0;
+                    } else {
+                        // ---- stop at k: residual [P_k - Q_k]_+ (rejected) or the bonus row P_k (k == gamma) ----
+                        const int k = sq.k;
+                        const bool bonus = k >= g;
+                        const T* tp = row_ptr(static_cast<const T*>(v.target), b, v.Gmax + 1, k, v.V);
+                        const T* dp = bonus ? nullptr : row_ptr(static_cast<const T*>(v.draft), b, v.Gmax, k, v.V);
+                        const float2 ts = __ldcg(v.row_stats + (size_t)b * v.R + k);
+                        float kt = -(ts.x * v.c + log2f(ts.y)), kd = 0.f;
+                        if (!bonus) {
+                            const float2 ds = __ldcg(v.row_stats + (size_t)b * v.R + v.Gmax + 1 + k);
+                            kd = -(ds.x * v.c + log2f(ds.y));
+                        }
+                        const int rseg = p.r.seg, rnseg = p.r.nseg;
+                        const int j0 = (int)((long long)rnseg * part / p.nG), j1 = (int)((long long)rnseg * (part + 1) / p.nG);
+                        for (int sg = j0; sg < j1 && ok; ++sg) {
+                            const int e0 = sg * rseg;
+                            const int n = min(rseg, v.V - e0);
+                            WkMeta m;
+                            m.type = kItemMass; m.b = b; m.k = k; m.row = bonus ? 1 : 0; m.sg = sg; m.nvec = n / kVec;
+                            m.flags = (sg == j0 ? 1 : 0) | (sg == j1 - 1 ? 2 : 0);
+                            m.kt = kt; m.kd = kd;
+                            ok = issue(m, tp + e0, bonus ? nullptr : dp + e0, (uint32_t)n * (uint32_t)sizeof(T));
+                        }
+                        sq.stage = 2;                          // this sequence is done for the producer
+                        --alive;
+                        s_seq[si] = sq;
+                        continue;
                     }
                 }
-                if (!ok) break;
-                __threadfence();
-                if (k < g && (d & 1u)) continue;               // accepted: on to the next position
-                // ---- stop at k: residual [P_k - Q_k]_+ (rejected) or the bonus row P_k (k == gamma) ----
-                const bool bonus = k >= g;
-                const T* tp = row_ptr(static_cast<const T*>(v.target), b, v.Gmax + 1, k, v.V);
-                const T* dp = bonus ? nullptr : row_ptr(static_cast<const T*>(v.draft), b, v.Gmax, k, v.V);
-                const float2 ts = __ldcg(v.row_stats + (size_t)b * v.R + k);
-                float kt = -(ts.x * v.c + log2f(ts.y)), kd = 0.f;
-                if (!bonus) {
-                    const float2 ds = __ldcg(v.row_stats + (size_t)b * v.R + v.Gmax + 1 + k);
-                    kd = -(ds.x * v.c + log2f(ds.y));
+                // ---- position k: this CTA's share of target row k and, below gamma, draft row k ----
+                {
+                    const int k = sq.k;
+                    const int nrows = k < g ? 2 : 1;
+                    const int items = nrows * v.nseg;
+                    const int i0 = (int)((long long)items * part / p.nG), i1 = (int)((long long)items * (part + 1) / p.nG);
+                    for (int i = i0; i < i1 && ok; ++i) {
+                        const int row = i / v.nseg, sg = i - row * v.nseg;
+                        const T* rowp = row == 0 ? row_ptr(static_cast<const T*>(v.target), b, v.Gmax + 1, k, v.V)
+                                                 : row_ptr(static_cast<const T*>(v.draft), b, v.Gmax, k, v.V);
+                        const int e0 = sg * v.seg;
+                        const int n = min(v.seg, v.V - e0);
+                        WkMeta m;
+                        m.type = kItemStats; m.b = b; m.k = k; m.row = row; m.sg = sg; m.nvec = n / kVec;
+                        m.flags = ((sg == 0 || i == i0) ? 1 : 0) | ((sg == v.nseg - 1 || i == i1 - 1) ? 2 : 0);
+                        m.kt = m.kd = 0.f;
+                        ok = issue(m, rowp + e0, nullptr, (uint32_t)n * (uint32_t)sizeof(T));
+                    }
+                    sq.stage = 1;
+                    s_seq[si] = sq;
+                    progress = true;
                 }
-                const int rseg = p.r.seg, rnseg = p.r.nseg;
-                const int j0 = (int)((long long)rnseg * part / p.nG), j1 = (int)((long long)rnseg * (part + 1) / p.nG);
-                for (int sg = j0; sg < j1 && ok; ++sg) {
-                    const int e0 = sg * rseg;
-                    const int n = min(rseg, v.V - e0);
-                    WkMeta m;
-                    m.type = kItemMass; m.b = b; m.k = k; m.row = bonus ? 1 : 0; m.sg = sg; m.nvec = n / kVec;
-                    m.flags = (sg == j0 ? 1 : 0) | (sg == j1 - 1 ? 2 : 0);
-                    m.kt = kt; m.kd = kd;
-                    ok = issue(m, tp + e0, bonus ? nullptr : dp + e0, (uint32_t)n * (uint32_t)sizeof(T));
-                }
-                break;                                          // this sequence is done for the producer
+            }
+            if (progress) {
+                t_last = clock64();
+            } else {
+                if (clock64() - t_last > kWaitCycles) ok = false;
+                __nanosleep(64);
             }
         }
         if (!ok) atomicExch(v.abort_flag, 1);
@@ -205,7 +236,15 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                 float2* pp = v.partial + ((size_t)b * v.R + slot_r) * v.S;
                 for (int q = e.first_sg + lane; q <= e.last_sg; q += 32)
                     pp[q] = (q == e.first_sg) ? out : make_float2(-INFINITY, 0.f);
-                // the loads of the accept test do not depend on the statistics: start them now
+                __threadfence();
+                __syncwarp();
+                unsigned old = 0;
+                if (lane == 0) old = atomicAdd(v.ticket + b, (unsigned)len);
+                old = __shfl_sync(0xffffffffu, old, 0);
+                if (old + (unsigned)len != wk_cum(k, g, v.nseg)) continue;
+                // ---- position k is complete: merge its rows (lane 0: target, lane 1: draft), decide ----
+                __threadfence();
+                // the drafted token, its two logits, the uniform (in flight while the rows are merged)
                 int x = 0;
                 float tl = 0.f, dl = 0.f, u = 2.f;
                 bool bad = false;
@@ -218,14 +257,6 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                         u = v.u_accept[(size_t)b * v.Gmax + k];
                     }
                 }
-                __threadfence();
-                __syncwarp();
-                unsigned old = 0;
-                if (lane == 0) old = atomicAdd(v.ticket + b, (unsigned)len);
-                old = __shfl_sync(0xffffffffu, old, 0);
-                if (old + (unsigned)len != wk_cum(k, g, v.nseg)) continue;
-                // ---- position k is complete: merge its rows (lane 0: target, lane 1: draft), decide ----
-                __threadfence();
                 const int nrows = k < g ? 2 : 1;
                 if (lane < nrows) {
                     const int rr = lane == 0 ? k : v.Gmax + 1 + k;
@@ -410,11 +441,18 @@ static bs_status launch_walk(WalkParams& p, cudaStream_t st) {
     }
     // groups of CTAs wait for one another: never more CTAs than can be resident together
     const int max_grid = g_wk_blocks[variant][dev] * sm_count();
-    int nG = max_grid / p.v.B;
+    // every sequence is shared by nG CTAs and every CTA holds a share of about B * nG / grid sequences,
+    // so a long run of accepted drafts keeps a slice of many CTAs busy instead of one whole CTA
+    // (measured on 256 x 152064 fp32: 3.5 shares per CTA is the best trade between the time a
+    // sequence waits for its CTAs' other work and the time it takes to stream a share)
+    int nG = (int)((7LL * max_grid + p.v.B) / (2LL * p.v.B));
+    if (nG > 8) nG = 8;
     if (nG > p.v.nseg) nG = p.v.nseg;                        // every CTA of a group gets a segment of every row
     if (nG < 1) nG = 1;
+    while (nG > 1 && (long long)p.v.B * nG > (long long)max_grid * kWkMaxSeqs) --nG;
     p.nG = nG;
-    const int grid = nG > 1 ? p.v.B * nG : (p.v.B < max_grid ? p.v.B : max_grid);
+    const long long pairs = (long long)p.v.B * nG;
+    const int grid = pairs < max_grid ? (int)pairs : max_grid;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(kWkThreads);
