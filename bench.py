@@ -420,6 +420,28 @@ def run_cuda(args, w):
         peak, peak_src = FALLBACK_HBM_GBS, "fallback"
     achieved = verify_bytes / (verify_ms * 1e-3) / 1e9
 
+    # ---- the same rounds through the early-exit entry point, for comparison (plain runs only) ----
+    variants = None
+    if not walk and not drafted and w.temperature > 0.0:
+        def walk_step(s):
+            bs.bs_bandit_select(state, alg, B, K, s["u_arm"], None, arm_d, gamma_d)
+            walk_call(s)
+            bs.bs_bandit_update(state, alg, B, K, arm_d, out_len)
+        for i in range(min(args.warmup, 5)):
+            walk_step(sets[i % ring])
+        sync_all()
+        a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        nw = min(args.steps, 100)
+        a.record(stream)
+        for i in range(nw):
+            walk_step(sets[i % ring])
+        b_.record(stream)
+        sync_all()
+        wms, _ = reduce_over_ranks(a.elapsed_time(b_), 0.0, dev)
+        variants = {"early_exit": {"value": job_rounds_per_s(world, nw, wms), "unit": UNIT, "ms_per_step": wms / nw,
+                                   "steps": nw, "launch": "direct launches",
+                                   "path": "select, bs_verify_walk, update (see --walk)"}}
+
     # ---- end to end from pinned host buffers ----
     e2e = None
     if args.e2e_steps > 0:
@@ -485,11 +507,11 @@ def run_cuda(args, w):
             "tokens_per_s": mean_y * B * value,
             "mean_accepted_len": mean_y,
             "algorithmic_gbs": bytes_all / (ms * 1e-3) / 1e9,
-            "roofline": {"bound": "hbm", "kernel": "verify_kernel (bs_softmax_verify)", "achieved": achieved,
+            "roofline": {"bound": "hbm", "kernel": "verify_stream_kernel (bs_softmax_verify)", "achieved": achieved,
                          "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": ncu_traffic(w.name, verify_bytes), "bytes_per_launch": verify_bytes,
                          "ms_per_launch": verify_ms, "residual_ms_per_launch": resid_ms},
-            "e2e": e2e, "cpu_baseline": cpu, "clocks": clocks,
+            "e2e": e2e, "cpu_baseline": cpu, "clocks": clocks, "variants": variants,
             "gpu_launches": (3 if walk else 4 + (2 * G if drafted else 0)) * args.steps,
         }
         if walk:
