@@ -236,15 +236,8 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                 float2* pp = v.partial + ((size_t)b * v.R + slot_r) * v.S;
                 for (int q = e.first_sg + lane; q <= e.last_sg; q += 32)
                     pp[q] = (q == e.first_sg) ? out : make_float2(-INFINITY, 0.f);
-                __threadfence();
-                __syncwarp();
-                unsigned old = 0;
-                if (lane == 0) old = atomicAdd(v.ticket + b, (unsigned)len);
-                old = __shfl_sync(0xffffffffu, old, 0);
-                if (old + (unsigned)len != wk_cum(k, g, v.nseg)) continue;
-                // ---- position k is complete: merge its rows (lane 0: target, lane 1: draft), decide ----
-                __threadfence();
-                // the drafted token, its two logits, the uniform (in flight while the rows are merged)
+                // the drafted token, its two logits, the uniform (they do not depend on the statistics:
+                // in flight while the ticket is)
                 int x = 0;
                 float tl = 0.f, dl = 0.f, u = 2.f;
                 bool bad = false;
@@ -257,18 +250,36 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                         u = v.u_accept[(size_t)b * v.Gmax + k];
                     }
                 }
-                const int nrows = k < g ? 2 : 1;
-                if (lane < nrows) {
-                    const int rr = lane == 0 ? k : v.Gmax + 1 + k;
-                    const float2* qq = v.partial + ((size_t)b * v.R + rr) * v.S;
+                __threadfence();
+                __syncwarp();
+                unsigned old = 0;
+                if (lane == 0) old = atomicAdd(v.ticket + b, (unsigned)len);
+                old = __shfl_sync(0xffffffffu, old, 0);
+                if (old + (unsigned)len != wk_cum(k, g, v.nseg)) continue;
+                // ---- position k is complete: merge its rows (lane 0: target, lane 1: draft), decide ----
+                __threadfence();
+                // lanes 0..15 merge the partials of target row k, lanes 16..31 those of draft row k
+                {
+                    const int half = lane >> 4, hl = lane & 15;
+                    const int rr = half == 0 ? k : v.Gmax + 1 + k;
                     Online o{-INFINITY, 0.f};
-#pragma unroll 4
-                    for (int q = 0; q < v.nseg; ++q) {
-                        const float2 t = __ldcg(qq + q);
-                        o.merge(t.x, t.y, v.c);
+                    if (half == 0 || k < g) {
+                        const float2* qq = v.partial + ((size_t)b * v.R + rr) * v.S;
+                        for (int q = hl; q < v.nseg; q += 16) {
+                            const float2 t = __ldcg(qq + q);
+                            o.merge(t.x, t.y, v.c);
+                        }
                     }
-                    s_fin[lane] = make_float2(o.m, o.s);
-                    v.row_stats[(size_t)b * v.R + rr] = make_float2(o.m, o.s);
+                    float M = o.m;
+#pragma unroll
+                    for (int off = 8; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
+                    float Z = o.s * rescale(o.m, M, v.c);
+#pragma unroll
+                    for (int off = 8; off > 0; off >>= 1) Z += __shfl_xor_sync(0xffffffffu, Z, off);
+                    if (hl == 0 && (half == 0 || k < g)) {
+                        s_fin[half] = make_float2(M, Z);
+                        v.row_stats[(size_t)b * v.R + rr] = make_float2(M, Z);
+                    }
                 }
                 __syncwarp();
                 const float2 ts = s_fin[0];
