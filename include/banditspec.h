@@ -48,7 +48,7 @@ typedef enum {
     BS_ERR_CUDA = 2,          /* a CUDA runtime call or launch failed */
     BS_ERR_UNSUPPORTED = 3,   /* valid request outside the implemented limits */
     BS_ERR_WORKSPACE = 4,     /* workspace too small or misaligned */
-    BS_ERR_TIMEOUT = 5,       /* a bounded device-side wait gave up (LM-head pipeline) */
+    BS_ERR_TIMEOUT = 5,       /* bs_get_device_status: a bounded wait inside a kernel gave up */
     BS_ERR_DEVICE_DATA = 6    /* bs_get_device_status: some sequence carries a data error */
 } bs_status;
 
