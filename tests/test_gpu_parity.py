@@ -308,3 +308,23 @@ def test_full_size_invariants_all_sequences(lib):
         assert (ot[b, :tau[b]] == tk[b, :tau[b]]).all() and 0 <= ot[b, tau[b]] < w.V and (ot[b, y[b]:] == -1).all()
     p = out.p_tok.cpu().numpy(); q = out.q_tok.cpu().numpy()
     assert np.allclose(p[:8], q[:8], atol=1e-7) and (p >= 0).all() and (p <= 1 + 1e-6).all()
+
+
+@pytest.mark.parametrize("B,G,V,dtype", [(2, 1, 1 << 20, torch.float32), (2, 2, 1 << 20, torch.bfloat16),
+                                         (4096, 1, 64, torch.float32)])
+def test_largest_supported_sizes(lib, B, G, V, dtype):
+    """The limits the header states: a vocabulary of 2^20 entries (128 / 64 segments per row, 4096
+    residual pieces per sequence) and a batch of 4096 sequences."""
+    assert lib.bs_workspace_bytes(B, G, V) > 0
+    rng = np.random.default_rng(B + V)
+    rnd = _random_round(rng, B, G, V, dtype, 1.0, sigma=0.5, std=2.0)
+    out = parity.gpu_round(lib, rnd, 1.0)
+    st = lib.bs_get_device_status(out.workspace, B, G, V)
+    assert (st & ~lib.BS_DEV_RESIDUAL_FALLBACK == 0).all()
+    tally = parity.Tally()
+    seqs = range(B) if B <= 8 else list(range(0, B, 257))
+    parity.check_round(out, rnd, 1.0, tally, seqs=seqs, where=f"max sizes B={B} V={V}")
+    y = out.out_len.cpu().numpy(); tau = out.accept_len.cpu().numpy()
+    assert ((y == tau + 1) & (tau >= 0) & (tau <= rnd.gamma)).all()
+    # one more than the limits is refused on the host
+    assert lib.bs_workspace_bytes(B, G, (1 << 20) + 8) == 0 and lib.bs_workspace_bytes(4097, G, V) == 0
