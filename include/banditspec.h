@@ -169,10 +169,11 @@ bs_status bs_softmax_verify_noalloc(const void* target_logits, const void* draft
  * sequence that stops at position tau costs 2 (tau + 1) rows (2 gamma + 1 when everything
  * passes) plus a second pass over the rows of the stop position, instead of 2 gamma + 1 + 2.
  *
- *  arguments as bs_softmax_verify and bs_residual_sample; sampling mode only (temperature > 0,
- *  BS_ERR_UNSUPPORTED otherwise: greedy rounds take the two separate calls)
+ *  arguments as bs_softmax_verify and bs_residual_sample (temperature 0 = greedy mode: target rows
+ *  only, the emitted token is the arg-max of the stop row, draft logits and uniforms may be NULL)
  *  p_tok, q_tok  [B, Gmax] fp32 out or NULL: filled for the positions that were examined
- *                (j <= tau_b, j < gamma_b); the entries behind the stop are set to 0
+ *                (j <= tau_b, j < gamma_b); the entries behind the stop are set to 0 (all of them
+ *                in greedy mode)
  *  accept_len, out_tokens, out_len: as the two separate calls
  * The CTAs that share a sequence wait for one another, so the kernel is launched cooperatively
  * and the call fails with BS_ERR_CUDA where that is not possible.  A wait that does not end

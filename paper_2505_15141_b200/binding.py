@@ -189,7 +189,7 @@ def verify_round(target_logits, draft_logits, draft_tokens, gamma, u_accept, u_r
 
 def bs_verify_walk(target_logits, draft_logits, draft_tokens, gamma, u_accept, u_resample, temperature: float,
                    accept_len, p_tok, q_tok, out_tokens, out_len, workspace, stream=None) -> None:
-    """Verification with early exit and resampling in one launch (sampling mode)."""
+    """Verification with early exit and resampling in one launch."""
     B, G1, V = target_logits.shape
     _check(_lib.bs_verify_walk(_ptr(target_logits), _ptr(draft_logits), _dtype_code(target_logits),
                                _ptr(draft_tokens), _ptr(gamma), _ptr(u_accept), _ptr(u_resample), float(temperature),

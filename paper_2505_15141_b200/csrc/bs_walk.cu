@@ -30,7 +30,7 @@ constexpr int kWkRing = 8;                                       // events the c
 constexpr int kWkVecPerThread = kSegBytes / 16 / kWkConsumers;   // 4
 static_assert(kSegBytes == 2 * kResSegBytes && kWkWarps == kRsWarps, "one stage holds a segment or a pair of half segments");
 
-constexpr int kItemStats = 0, kItemMass = 1, kItemEnd = 2;
+constexpr int kItemStats = 0, kItemMass = 1, kItemEnd = 2, kItemAck = 3;
 
 struct WalkParams {
     VerifyParams v;        // logits, tokens, uniforms, outputs of the accept test, statistics and partials
@@ -58,14 +58,16 @@ struct WkSeq {
 constexpr int kWkMaxSeqs = 32;
 
 // Stats items counted on the sequence's ticket once position k is complete.
+template <bool GREEDY>
 __device__ __forceinline__ unsigned wk_cum(int k, int g, int nseg) {
+    if (GREEDY) return (unsigned)(nseg * (k + 1));           // target rows only
     return k < g ? (unsigned)(2 * nseg * (k + 1)) : (unsigned)(2 * nseg * g + nseg);
 }
 __device__ __forceinline__ unsigned ld_volatile_u32(const uint32_t* p) {
     return *reinterpret_cast<const volatile uint32_t*>(p);
 }
 
-template <typename T>
+template <typename T, bool GREEDY>
 __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkParams p) {
     extern __shared__ __align__(128) unsigned char ring[];    // kWkStages * 32 KB
     __shared__ __align__(8) unsigned long long s_full[kWkStages];
@@ -110,7 +112,7 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
             s_meta[slot] = m;
             const uint32_t bar = smem_u32(&s_full[slot]);
             const uint32_t dst = smem_u32(ring + (size_t)slot * kSegBytes);
-            if (m.type == kItemEnd) {
+            if (m.type == kItemEnd || m.type == kItemAck) {
                 mbar_arrive(bar);                              // nothing to copy: the phase completes at once
             } else {
                 mbar_arrive_expect_tx(bar, src1 ? 2u * bytes : bytes);
@@ -144,6 +146,18 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                         sq.k += 1;
                         sq.stage = 0;
                     } else {
+                        if (GREEDY) {
+                            // the deciding finisher has emitted the arg-max already; this share only
+                            // reports that it has seen the decision, so that the words can be cleared
+                            WkMeta m;
+                            m.type = kItemAck; m.b = b; m.k = sq.k; m.row = 0; m.sg = 0; m.nvec = 0; m.flags = 3;
+                            m.kt = m.kd = 0.f;
+                            ok = issue(m, nullptr, nullptr, 0);
+                            sq.stage = 2;
+                            --alive;
+                            s_seq[si] = sq;
+                            continue;
+                        }
                         // ---- stop at k: residual [P_k - Q_k]_+ (rejected) or the bonus row P_k (k == gamma) ----
                         const int k = sq.k;
                         const bool bonus = k >= g;
@@ -175,7 +189,7 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                 // ---- position k: this CTA's share of target row k and, below gamma, draft row k ----
                 {
                     const int k = sq.k;
-                    const int nrows = k < g ? 2 : 1;
+                    const int nrows = (!GREEDY && k < g) ? 2 : 1;
                     const int items = nrows * v.nseg;
                     const int i0 = (int)((long long)items * part / p.nG), i1 = (int)((long long)items * (part + 1) / p.nG);
                     for (int i = i0; i < i1 && ok; ++i) {
@@ -219,7 +233,7 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                 return;
             }
             const WkEvent e = s_ev[rs];
-            float2 mine = make_float2(-INFINITY, 0.f);
+            float2 mine = make_float2(-INFINITY, GREEDY ? __int_as_float(INT_MAX) : 0.f);
             if (lane < kWkWarps) mine = s_red[rs][lane];
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&s_evfree[rs]));   // the slot may be reused
@@ -228,6 +242,69 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
             const int graw = v.gamma[b];
             const int g = clamp_gamma(graw, v.Gmax);
             const int len = e.last_sg - e.first_sg + 1;
+
+            if (e.type == kItemAck) {
+                // ---- greedy: one more share has seen the stop decision; the last one clears the words ----
+                unsigned old = 0;
+                if (lane == 0) old = atomicAdd(p.r.ticket + b, 1u);
+                old = __shfl_sync(0xffffffffu, old, 0);
+                if (old + 1u == (unsigned)p.nG && lane == 0) {
+                    p.r.ticket[b] = 0u;
+                    v.ticket[b] = 0u;
+                    p.dec[b] = 0u;
+                }
+                continue;
+            }
+            if (GREEDY && e.type == kItemStats) {
+                // ---- a piece of target row k: (max, arg-max); the drafted token passes iff it is the arg-max ----
+                ArgMax a = warp_best(ArgMax{mine.x, __float_as_int(mine.y)});
+                float2* pp = v.partial + ((size_t)b * v.R + k) * v.S;
+                for (int q = e.first_sg + lane; q <= e.last_sg; q += 32)
+                    pp[q] = (q == e.first_sg) ? make_float2(a.m, __int_as_float(a.idx))
+                                              : make_float2(-INFINITY, __int_as_float(INT_MAX));
+                int x = 0;
+                if (k < g) x = v.tokens[(size_t)b * v.Gmax + k];
+                __threadfence();
+                __syncwarp();
+                unsigned old = 0;
+                if (lane == 0) old = atomicAdd(v.ticket + b, (unsigned)len);
+                old = __shfl_sync(0xffffffffu, old, 0);
+                if (old + (unsigned)len != wk_cum<true>(k, g, v.nseg)) continue;
+                __threadfence();
+                ArgMax best{-INFINITY, INT_MAX};
+                for (int q = lane; q < v.nseg; q += 32) {
+                    const float2 t = __ldcg(pp + q);
+                    best = better(best, ArgMax{t.x, __float_as_int(t.y)});
+                }
+                best = warp_best(best);
+                if (best.idx == INT_MAX) best.idx = 0;        // row of -inf / NaN only
+                const bool bad = k < g && (x < 0 || x >= v.V);
+                const bool acc = k < g && !bad && x == best.idx;
+                int bits = (k == 0 && graw != g) ? BS_DEV_BAD_GAMMA : 0;
+                if (bad) bits |= BS_DEV_BAD_TOKEN;
+                if (lane == 0) {
+                    v.row_stats[(size_t)b * v.R + k] = make_float2(best.m, __int_as_float(best.idx));
+                    if (k == 0) v.status[b] = bits; else if (bits) atomicOr(v.status + b, bits);
+                }
+                if (!acc) {
+                    // stop at k: the emitted token is the arg-max of target row k (Section 2, temperature 0)
+                    int32_t* ot = p.r.out_tokens + (size_t)b * (v.Gmax + 1);
+                    for (int j = lane; j <= v.Gmax; j += 32)
+                        ot[j] = j < k ? v.tokens[(size_t)b * v.Gmax + j] : (j == k ? best.idx : -1);
+                    for (int j = lane; j < v.Gmax; j += 32) {
+                        if (v.p_tok) v.p_tok[(size_t)b * v.Gmax + j] = 0.f;
+                        if (v.q_tok) v.q_tok[(size_t)b * v.Gmax + j] = 0.f;
+                    }
+                    if (lane == 0) {
+                        v.accept_len[b] = k;
+                        p.r.out_len[b] = k + 1;
+                    }
+                }
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) atomicExch(p.dec + b, ((unsigned)(k + 1) << 1) | (acc ? 1u : 0u));
+                continue;
+            }
 
             if (e.type == kItemStats) {
                 // ---- a piece of target row k (row 0) or draft row k (row 1) ----
@@ -255,7 +332,7 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                 unsigned old = 0;
                 if (lane == 0) old = atomicAdd(v.ticket + b, (unsigned)len);
                 old = __shfl_sync(0xffffffffu, old, 0);
-                if (old + (unsigned)len != wk_cum(k, g, v.nseg)) continue;
+                if (old + (unsigned)len != wk_cum<false>(k, g, v.nseg)) continue;
                 // ---- position k is complete: merge its rows (lane 0: target, lane 1: draft), decide ----
                 __threadfence();
                 // lanes 0..15 merge the partials of target row k, lanes 16..31 those of draft row k
@@ -349,6 +426,7 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
 
     // ================================= consumers =================================
     Online on{-INFINITY, 0.f};
+    ArgMax am{-INFINITY, INT_MAX};
     int first_sg = 0;
     int ev = 0;                                               // events posted by this CTA
     int slot = 0;
@@ -368,10 +446,19 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                                                          : neg_inf_vec<T>();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&s_empty[slot]));
-            online_add<T, kWkVecPerThread>(on, x, v.c);
-            if (m.flags & 2) {
-                wr = warp_merge(on, v.c);
-                on = Online{-INFINITY, 0.f};
+            if (GREEDY) {
+                argmax_add<T, kWkVecPerThread>(am, x, m.sg * v.seg + tid * kVec, kWkConsumers * kVec);
+                if (m.flags & 2) {
+                    am = warp_best(am);
+                    wr = make_float2(am.m, __int_as_float(am.idx));
+                    am = ArgMax{-INFINITY, INT_MAX};
+                }
+            } else {
+                online_add<T, kWkVecPerThread>(on, x, v.c);
+                if (m.flags & 2) {
+                    wr = warp_merge(on, v.c);
+                    on = Online{-INFINITY, 0.f};
+                }
             }
         } else if (m.type == kItemMass) {
             // a 16 KB segment of the row pair: warp w owns the w-th 1 KB piece and writes its mass
@@ -431,21 +518,21 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
     }
 }
 
-static int g_wk_blocks[2][64];        // resident CTAs per SM (0 = not queried)
+static int g_wk_blocks[4][64];        // resident CTAs per SM (0 = not queried)
 
-template <typename T>
+template <typename T, bool GREEDY>
 static bs_status launch_walk(WalkParams& p, cudaStream_t st) {
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64) dev = 0;
-    const int variant = Elem<T>::kDtype == BS_F32 ? 0 : 1;
+    const int variant = (Elem<T>::kDtype == BS_F32 ? 0 : 2) + (GREEDY ? 1 : 0);
     const size_t smem = (size_t)kWkStages * kSegBytes;
     if (!g_wk_blocks[variant][dev]) {
-        if (cudaFuncSetAttribute(verify_walk_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+        if (cudaFuncSetAttribute(verify_walk_kernel<T, GREEDY>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
             cudaSuccess)
             return cuda_status(cudaGetLastError());
         int nb = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_walk_kernel<T>, kWkThreads, smem) != cudaSuccess)
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, verify_walk_kernel<T, GREEDY>, kWkThreads, smem) != cudaSuccess)
             return cuda_status(cudaGetLastError());
         if (nb < 1) return BS_ERR_UNSUPPORTED;
         g_wk_blocks[variant][dev] = nb > 2 ? 2 : nb;
@@ -474,7 +561,7 @@ static bs_status launch_walk(WalkParams& p, cudaStream_t st) {
     at[0].val.cooperative = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    return cuda_status(cudaLaunchKernelEx(&cfg, verify_walk_kernel<T>, p));
+    return cuda_status(cudaLaunchKernelEx(&cfg, verify_walk_kernel<T, GREEDY>, p));
 }
 
 }  // namespace bs
@@ -490,10 +577,10 @@ extern "C" bs_status bs_verify_walk(const void* target_logits, const void* draft
     if (B > BS_MAX_BATCH || Gmax > BS_MAX_GAMMA || V > BS_MAX_VOCAB) return BS_ERR_UNSUPPORTED;
     if (dtype != BS_F32 && dtype != BS_BF16) return BS_ERR_INVALID_ARG;
     if (!(temperature >= 0.f) || !isfinite(temperature)) return BS_ERR_INVALID_ARG;
-    if (temperature == 0.f) return BS_ERR_UNSUPPORTED;       // greedy rounds: bs_softmax_verify + bs_residual_sample
-    if (!target_logits || !gamma || !accept_len || !out_tokens || !out_len || !u_resample || !workspace)
-        return BS_ERR_INVALID_ARG;
-    if (Gmax > 0 && (!draft_tokens || !draft_logits || !u_accept)) return BS_ERR_INVALID_ARG;
+    const bool greedy = temperature == 0.f;
+    if (!target_logits || !gamma || !accept_len || !out_tokens || !out_len || !workspace) return BS_ERR_INVALID_ARG;
+    if (Gmax > 0 && !draft_tokens) return BS_ERR_INVALID_ARG;
+    if (!greedy && (!u_resample || (Gmax > 0 && (!draft_logits || !u_accept)))) return BS_ERR_INVALID_ARG;
     const size_t es = dtype == BS_F32 ? 4 : 2;
     if (((size_t)V * es) % 16 != 0 || (reinterpret_cast<uintptr_t>(target_logits) & 15) ||
         (reinterpret_cast<uintptr_t>(draft_logits) & 15))
@@ -515,7 +602,7 @@ extern "C" bs_status bs_verify_walk(const void* target_logits, const void* draft
     v.B = B; v.Gmax = Gmax; v.V = V; v.R = w.R; v.S = w.S;
     v.seg = seg_elems(dtype);
     v.nseg = div_up(V, v.seg);
-    v.c = kLog2e / temperature;
+    v.c = greedy ? 1.f : kLog2e / temperature;
     v.mode = kModeVerify; v.position = 0; v.draft_ready = v.ticket_row; v.draft_out = nullptr;
     ResidParams& r = p.r;
     r.target = target_logits; r.draft = draft_logits; r.tokens = draft_tokens; r.gamma = gamma;
@@ -534,5 +621,6 @@ extern "C" bs_status bs_verify_walk(const void* target_logits, const void* draft
     p.dec = v.ticket_row + B;
     p.nG = 1;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    return dtype == BS_F32 ? launch_walk<float>(p, st) : launch_walk<__nv_bfloat16>(p, st);
+    if (greedy) return dtype == BS_F32 ? launch_walk<float, true>(p, st) : launch_walk<__nv_bfloat16, true>(p, st);
+    return dtype == BS_F32 ? launch_walk<float, false>(p, st) : launch_walk<__nv_bfloat16, false>(p, st);
 }

@@ -79,10 +79,37 @@ def test_walk_edge_cases_and_reuse(lib):
     assert st[4] & lib.BS_DEV_BAD_TOKEN and int(out4.accept_len[4]) <= 1
     assert st[6] & lib.BS_DEV_BAD_GAMMA and int(out4.out_len[6]) == 1
     parity.check_round(out4, rnd, 1.0, tally, seqs=[0, 1, 2, 3, 5, 7], where="walk after errors", walk=True)
-    # greedy and unaligned rows are refused on the host
+    # rows that are not 16-byte aligned are refused on the host
+    odd = _round(rng, 2, 2, 1001, torch.float32, 1.0)
     with pytest.raises(lib.BanditSpecError) as e:
-        _walk(lib, rnd, 0.0, ws)
+        _walk(lib, odd, 1.0)
     assert e.value.code == lib.BS_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_walk_greedy_with_ties(lib, dtype):
+    """Temperature 0: a draft passes iff it is the arg-max of its target row (lowest index among equal
+    maxima), the emitted token is the arg-max of the stop row; bit-exact, no flags."""
+    rng = np.random.default_rng(23)
+    tally = parity.Tally()
+    for B, G, V in ((6, 5, 4096), (3, 4, 33336), (300, 2, 512)):
+        # coarse values -> many exact ties for the arg-max
+        t = torch.as_tensor(rng.integers(-4, 5, size=(B, G + 1, V)).astype(np.float32)).to(dtype).to(DEV)
+        gamma = rng.integers(0, G + 1, size=B).astype(np.int32)
+        tok = t[:, :G].float().argmax(dim=-1).to(torch.int32)
+        flip = torch.as_tensor(rng.random((B, G)) < 0.3, device=DEV)
+        tok = torch.where(flip, (tok + 1) % V, tok).to(torch.int32).contiguous()
+        rnd = wl.RoundInputs(target=t, draft=t[:, :G].contiguous(), tokens=tok, gamma=gamma,
+                             uniforms=wl.round_uniforms(1, 1, B, G))
+        ws = lib.new_workspace(B, G, V, DEV)
+        out = _walk(lib, rnd, 0.0, ws)
+        assert (lib.bs_get_device_status(ws, B, G, V) == 0).all()
+        seqs = range(B) if B <= 16 else list(range(0, B, 17))
+        parity.check_round(out, rnd, 0.0, tally, seqs=seqs, where=f"walk greedy V={V}", walk=True)
+        ref = parity.gpu_round(lib, rnd, 0.0, ws)            # the two-call path on the same workspace
+        assert torch.equal(ref.accept_len, out.accept_len) and torch.equal(ref.out_tokens, out.out_tokens)
+        assert torch.equal(ref.out_len, out.out_len)
+    assert tally.flagged_accept == 0 and tally.flagged_token == 0
 
 
 def test_walk_full_size(lib):
