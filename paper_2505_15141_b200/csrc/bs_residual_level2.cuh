@@ -119,14 +119,38 @@ __device__ void rs_level2(const ResidParams& p, int b, const RsSeq sq, MassFn f)
         if (lane == 0) excl = 0.0;
         int ps = -1;
         double before = 0.0;
-        if (incl > target && !(excl > target)) {              // the lane in whose pieces the crossing falls
-            double run = excl;
-            for (int i = s0; i < s1; ++i) {
-                const double m = (double)__ldcg(pm + i);
-                if (m > 0.0) { ps = i; before = run; }        // so far: the last piece with mass
-                if (run + m > target && m > 0.0) break;       // the first piece whose end passes the target
-                run += m;
+        // the lane in whose pieces the crossing falls; its pieces are then searched by the whole
+        // warp, 32 at a time (one load latency per round instead of one per piece)
+        const unsigned cross = __ballot_sync(0xffffffffu, incl > target && !(excl > target));
+        if (cross) {
+            const int L = __ffs(cross) - 1;
+            const int c0 = __shfl_sync(0xffffffffu, s0, L), c1 = __shfl_sync(0xffffffffu, s1, L);
+            double run0 = __shfl_sync(0xffffffffu, excl, L);  // mass in front of the lane's pieces
+            int lastp = -1;                                   // so far: the last piece with mass
+            double lastbefore = 0.0;
+            for (int r0 = c0; r0 < c1 && ps < 0; r0 += 32) {
+                const int i = r0 + lane;
+                const double m = i < c1 ? (double)__ldcg(pm + i) : 0.0;
+                const double sc = warp_scan_incl(m);
+                double sx = __shfl_up_sync(0xffffffffu, sc, 1);
+                if (lane == 0) sx = 0.0;
+                // the first piece whose end passes the target
+                const unsigned hit = __ballot_sync(0xffffffffu, run0 + sc > target && !(run0 + sx > target) && m > 0.0);
+                if (hit) {
+                    const int src = __ffs(hit) - 1;
+                    ps = __shfl_sync(0xffffffffu, i, src);
+                    before = __shfl_sync(0xffffffffu, run0 + sx, src);
+                } else {
+                    const unsigned pos = __ballot_sync(0xffffffffu, m > 0.0);
+                    if (pos) {
+                        const int src = 31 - __clz(pos);
+                        lastp = __shfl_sync(0xffffffffu, i, src);
+                        lastbefore = __shfl_sync(0xffffffffu, run0 + sx, src);
+                    }
+                    run0 += __shfl_sync(0xffffffffu, sc, 31);
+                }
             }
+            if (ps < 0 && lastp >= 0) { ps = lastp; before = lastbefore; }   // rounding only
         }
         // the lane that found the piece tells the others
         const unsigned found = __ballot_sync(0xffffffffu, ps >= 0);
