@@ -73,6 +73,8 @@ def parse_args():
     ap.add_argument("--walk", action="store_true",
                     help="the round with early exit: select -> bs_verify_walk (verification up to the first "
                          "rejection + resampling in one launch) -> update")
+    ap.add_argument("--no-others", action="store_true",
+                    help="skip the short runs of the other workloads that the default invocation adds to its line")
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="budget of the CPU-oracle sample")
@@ -512,6 +514,7 @@ def run_cuda(args, w):
                          "traffic": ncu_traffic(w.name, verify_bytes), "bytes_per_launch": verify_bytes,
                          "ms_per_launch": verify_ms, "residual_ms_per_launch": resid_ms},
             "e2e": e2e, "cpu_baseline": cpu, "clocks": clocks, "variants": variants,
+            "other_workloads": getattr(args, "others", None),
             "gpu_launches": (3 if walk else 4 + (2 * G if drafted else 0)) * args.steps,
         }
         if walk:
@@ -752,9 +755,35 @@ def run_lmhead(args, w):
         dist.destroy_process_group()
 
 
+OTHER_WORKLOADS = ("llama3_ucb", "llama2_fixed", "lmhead_llama3", "lmhead_llama3_b128")
+
+
+def other_workloads_summary():
+    """Short runs of the other workloads, each in a process of its own before this one touches the
+    GPU: rounds/s and the dominant kernel's roofline line, for the record next to the main line."""
+    out = {}
+    for name in OTHER_WORKLOADS:
+        cmd = [sys.executable, os.path.abspath(__file__), "--workload", name, "--steps", "200", "--warmup", "20",
+               "--no-cpu-baseline", "--e2e-steps", "0", "--no-others"]
+        try:
+            res = subprocess.run(cmd, capture_output=True, text=True, timeout=240)
+            d = json.loads(res.stdout.strip().splitlines()[-1])
+            r = d["roofline"]
+            out[name] = {"value": d["value"], "unit": d["unit"], "ms_per_step": d["ms_per_step"],
+                         "roofline": {k: r.get(k) for k in ("bound", "kernel", "achieved", "peak", "unit", "frac",
+                                                            "ms_per_launch")},
+                         "variants": d.get("variants")}
+        except Exception as e:                                   # the main line must not depend on these
+            out[name] = {"error": f"{type(e).__name__}: {e}"[:200]}
+    return out
+
+
 def main():
     args = parse_args()
     from paper_2505_15141_b200 import workloads as wl
+    plain_default = (args.workload == "qwen_exp3" and args.impl == "cuda" and not (args.batch or args.fixed_gamma
+                     or args.walk or args.drafted or args.no_others) and int(os.environ.get("WORLD_SIZE", "1")) == 1)
+    args.others = other_workloads_summary() if plain_default else None
     if args.workload in wl.LMHEAD_WORKLOADS:
         w = wl.LMHEAD_WORKLOADS[args.workload]
         if args.batch:
