@@ -88,7 +88,9 @@ bs_status bs_workspace_init(void* workspace, size_t workspace_bytes, void* strea
 
 /* Copies the per-sequence status words of the LAST verify/residual call to host memory.
  * Synchronises the stream.  host_status: host array [B].  Returns BS_ERR_DEVICE_DATA if any
- * word is non-zero, BS_OK otherwise. */
+ * word is non-zero, BS_ERR_TIMEOUT if a bounded wait inside a kernel of that call gave up (its
+ * outputs are then undefined and its arrival counters may be left non-zero: clear the workspace
+ * with bs_workspace_init before using it again), BS_OK otherwise. */
 bs_status bs_get_device_status(const void* workspace, size_t workspace_bytes, int B, int Gmax, int V,
                                int32_t* host_status, void* stream);
 
