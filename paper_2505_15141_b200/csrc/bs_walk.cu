@@ -96,6 +96,7 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    pdl_enter();                                              // gamma comes from the kernel before this one
 
     if (warp == kWkWarps) {
         // =============================== producer ===============================
@@ -556,11 +557,13 @@ static bs_status launch_walk(WalkParams& p, cudaStream_t st) {
     cfg.blockDim = dim3(kWkThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute at[1];
+    cudaLaunchAttribute at[2];
     at[0].id = cudaLaunchAttributeCooperative;
     at[0].val.cooperative = 1;
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // set-up overlaps the previous kernel's drain
+    at[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return cuda_status(cudaLaunchKernelEx(&cfg, verify_walk_kernel<T, GREEDY>, p));
 }
 
