@@ -4,15 +4,18 @@
 //
 // Every sequence is shared by a fixed group of nG CTAs (up to 8), and every CTA holds a share of
 // several sequences and interleaves them, so that a sequence with a long run of accepted drafts
-// keeps a slice of many CTAs busy rather than one CTA alone.  For position k the group streams target row k and draft row k (bulk async copies into a ring of
-// 32 KB stages, 16 consumer warps, online softmax: the pipeline of the row-statistics kernel),
-// every CTA its contiguous share of the 2 * nseg segments.  A finisher warp per CTA publishes the
+// keeps a slice of many CTAs busy rather than one CTA alone.  For position k the group streams
+// target row k and draft row k (bulk async copies into a ring of 32 KB stages, 16 consumer warps,
+// online softmax: the pipeline of the row-statistics kernel), every CTA its contiguous share of
+// the 2 * nseg segments (greedy mode: target rows only, arg-max instead of the statistics).  A finisher warp per CTA publishes the
 // pieces and counts them on the sequence's ticket; the finisher that completes position k merges
 // the two rows, tests r <= min{1, P/Q} for the drafted token and publishes the decision word of
 // the sequence.  The producers of the group wait for that word (bounded), then stream position
 // k + 1, or -- at the first rejection, or after the bonus row when everything passed -- the row
-// pair of the stop position again (it has just been read: L2) for the residual masses; the
-// finisher that completes that count runs the inverse CDF (level 2 of the resampling kernel).
+// pair of the stop position again (it has just been read: partly still in L2) for the residual
+// masses; the finisher that completes that count runs the inverse CDF (level 2 of the resampling
+// kernel).  In greedy mode the deciding finisher emits the arg-max of the stop row itself and the
+// shares only acknowledge the decision, so that the last one can clear the sequence's words.
 //
 // CTAs of one group wait for one another, so the kernel is launched cooperatively (all CTAs
 // resident).  Every wait is bounded; a wait that gives up sets the abort word and the CTA drains.
