@@ -132,3 +132,27 @@ def test_walk_full_size(lib):
         assert ((y == tau + 1) & (tau <= rnd.gamma)).all()
         for b in range(w.B):
             assert 0 <= ot[b, tau[b]] < w.V and (ot[b, y[b]:] == -1).all()
+
+
+def test_walk_wait_that_cannot_end_is_reported_and_the_context_survives(lib):
+    """The CTAs that share a sequence wait for its decision word.  With the sequence's arrival counter
+    spoilt beforehand (the workspace's first B words are those counters) no finisher ever completes
+    the count, so nobody decides: the producers' bounded wait must give up after about a second, the
+    kernel must drain, bs_get_device_status must say BS_ERR_TIMEOUT, and after bs_workspace_init the
+    same workspace must work again."""
+    rng = np.random.default_rng(41)
+    B, G, V = 4, 3, 4096
+    rnd = _round(rng, B, G, V, torch.float32, 1.0, gamma=[3, 2, 3, 1])
+    ws = lib.new_workspace(B, G, V, DEV)
+    ws.view(torch.int32)[2] = 5                                  # sequence 2 can never reach its count
+    out = _walk(lib, rnd, 1.0, ws)                               # returns: every wait is bounded
+    with pytest.raises(lib.BanditSpecError) as e:
+        lib.bs_get_device_status(ws, B, G, V)
+    assert e.value.code == lib.BS_ERR_TIMEOUT
+    # the other sequences were finished all the same
+    tally = parity.Tally()
+    parity.check_round(out, rnd, 1.0, tally, seqs=[0, 1, 3], where="walk beside a stuck sequence", walk=True)
+    lib.bs_workspace_init(ws)
+    out2 = _walk(lib, rnd, 1.0, ws)
+    assert (lib.bs_get_device_status(ws, B, G, V) == 0).all()
+    parity.check_round(out2, rnd, 1.0, tally, where="walk after re-initialising the workspace", walk=True)
