@@ -512,6 +512,7 @@ def run_cuda(args, w):
             "roofline": {"bound": "hbm", "kernel": "verify_stream_kernel (bs_softmax_verify)", "achieved": achieved,
                          "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": ncu_traffic(w.name, verify_bytes), "bytes_per_launch": verify_bytes,
+                         "nominal_peak": 8000.0, "frac_of_nominal": achieved / 8000.0,
                          "ms_per_launch": verify_ms, "residual_ms_per_launch": resid_ms},
             "e2e": e2e, "cpu_baseline": cpu, "clocks": clocks, "variants": variants,
             "other_workloads": getattr(args, "others", None),
@@ -689,6 +690,8 @@ def run_lmhead(args, w):
     roof = ({"bound": "hbm", "achieved": gbs, "peak": hbm_peak, "unit": "GB/s", "frac": gbs / hbm_peak}
             if hbm_bound else
             {"bound": "tensor", "achieved": tfs, "peak": tc_peak, "unit": "TFLOP/s", "frac": tfs / tc_peak})
+    roof.update({"nominal_hbm_gbs": 8000.0, "hbm_frac_of_nominal": gbs / 8000.0,
+                 "nominal_bf16_tflops": 2250.0, "tensor_frac_of_nominal": tfs / 2250.0})
     roof.update({"kernel": "lmhead_gemm_kernel (bs_lmhead_verify)", "peak_source": src,
                  "traffic": ncu_traffic(w.name, 2.0 * w.V * (w.d_t + w.d_d) + 2.0 * w.B * ((w.gamma + 1) * w.d_t + w.gamma * w.d_d)),
                  "bytes_per_launch": nbytes, "flops_per_launch": flops,
