@@ -294,12 +294,15 @@ def run_cuda(args, w):
     walk = args.walk
 
     def walk_call(s):
-        bs.bs_verify_walk(s["target"], s["draft"], s["tokens"], gamma_d, s["u_accept"], s["u_resample"],
-                          w.temperature, accept_len, p_tok, q_tok, out_tokens, out_len, ws)
+        fn = bs.bs_verify_walk_drafted if drafted else bs.bs_verify_walk
+        fn(s["target"], s["draft"], tok_d if drafted else s["tokens"], gamma_d, s["u_accept"], s["u_resample"],
+           w.temperature, accept_len, p_tok, q_tok, out_tokens, out_len, ws)
 
     def step_calls(s):
         bs.bs_bandit_select(state, alg, B, K, s["u_arm"], None, arm_d, gamma_d)
         if walk:
+            if drafted:
+                draft_calls(s)
             walk_call(s)
             bs.bs_bandit_update(state, alg, B, K, arm_d, out_len)
             return
@@ -398,7 +401,7 @@ def run_cuda(args, w):
         rsd[i][1].record(stream)
         if walk:                                               # rows the walk had to read: up to the stop position
             tau = accept_len.to(torch.int64); gm = gamma_d.to(torch.int64)
-            walk_rows += torch.where(tau < gm, 2 * (tau + 1), 2 * gm + 1).sum()
+            walk_rows += (tau + 1).sum() if drafted else torch.where(tau < gm, 2 * (tau + 1), 2 * gm + 1).sum()
         bs.bs_bandit_update(state, alg, B, K, arm_d, out_len)
         y_sum += out_len.sum()
     torch.cuda.synchronize()
@@ -502,7 +505,9 @@ def run_cuda(args, w):
                        "logits_dtype": w.dtype, "temperature": w.temperature,
                        "l2": f"ring of {ring} input sets, {ring * set_bytes / 1e6:.0f} MB > 2 x L2",
                        "launch": "one CUDA graph per step" if graphs else "direct launches",
-                       "path": ("select, verify with early exit + resample in one launch, update" if walk else
+                       "path": ("select, draft x Gmax, verify with early exit on drafted statistics + resample "
+                                "in one launch, update" if walk and drafted else
+                                "select, verify with early exit + resample in one launch, update" if walk else
                                 "select, draft x Gmax, verify on drafted statistics, resample, update"
                                 if drafted else "select, verify, resample, update"),
                        "multi_gpu": "one independent batch per rank, no collective on the data path"},
@@ -516,7 +521,7 @@ def run_cuda(args, w):
                          "ms_per_launch": verify_ms, "residual_ms_per_launch": resid_ms},
             "e2e": e2e, "cpu_baseline": cpu, "clocks": clocks, "variants": variants,
             "other_workloads": getattr(args, "others", None),
-            "gpu_launches": (3 if walk else 4 + (2 * G if drafted else 0)) * args.steps,
+            "gpu_launches": ((3 if walk else 4) + (2 * G if drafted else 0)) * args.steps,
         }
         if walk:
             line["roofline"]["kernel"] = "verify_walk_kernel (bs_verify_walk)"

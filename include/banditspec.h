@@ -225,6 +225,18 @@ bs_status bs_softmax_verify_drafted(const void* target_logits, const void* draft
                                     int32_t* accept_len, float* p_tok, float* q_tok,
                                     void* workspace, size_t workspace_bytes, void* stream);
 
+/* bs_verify_walk for a round whose draft rows went through bs_draft_sample on the same workspace
+ * (see bs_softmax_verify_drafted): only target rows are walked, position after position; of each
+ * draft row the statistics left by drafting and the logit of the drafted token are used, and the
+ * draft row of the stop position is read once for the residual.  Same arguments, outputs and
+ * requirements as bs_verify_walk; an undrafted position stops the sequence there with
+ * BS_DEV_DRAFT_MISSING; the drafted marks are consumed. */
+bs_status bs_verify_walk_drafted(const void* target_logits, const void* draft_logits, bs_dtype dtype,
+                                 const int32_t* draft_tokens, const int32_t* gamma, const float* u_accept,
+                                 const float* u_resample, float temperature, int B, int Gmax, int V,
+                                 int32_t* accept_len, float* p_tok, float* q_tok, int32_t* out_tokens,
+                                 int32_t* out_len, void* workspace, size_t workspace_bytes, void* stream);
+
 /* ---- fused LM head (Algorithm 6, second line: the models are evaluated on all drafted positions
  *      in parallel; the last step of that evaluation is logits = H W) -------------------------- */
 

@@ -42,6 +42,8 @@ SIGNATURES = {
     "bs_residual_sample": (_i, [_vp, _vp, _i, _vp, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _sz, _vp]),
     "bs_softmax_verify_noalloc": (_i, [_vp, _vp, _i, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _vp]),
     "bs_verify_walk": (_i, [_vp, _vp, _i, _vp, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "bs_verify_walk_drafted": (_i, [_vp, _vp, _i, _vp, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _sz,
+                                    _vp]),
     "bs_draft_sample": (_i, [_vp, _i, _i, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _sz, _vp]),
     "bs_softmax_verify_drafted": (_i, [_vp, _vp, _i, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bs_lmhead_workspace_bytes": (_sz, [_i, _i, _i]),
@@ -195,6 +197,17 @@ def bs_verify_walk(target_logits, draft_logits, draft_tokens, gamma, u_accept, u
                                _ptr(draft_tokens), _ptr(gamma), _ptr(u_accept), _ptr(u_resample), float(temperature),
                                B, G1 - 1, V, _ptr(accept_len), _ptr(p_tok), _ptr(q_tok), _ptr(out_tokens),
                                _ptr(out_len), _ptr(workspace), workspace.numel(), _stream(stream)), "bs_verify_walk")
+
+
+def bs_verify_walk_drafted(target_logits, draft_logits, draft_tokens, gamma, u_accept, u_resample, temperature: float,
+                           accept_len, p_tok, q_tok, out_tokens, out_len, workspace, stream=None) -> None:
+    """bs_verify_walk on the statistics bs_draft_sample left in the workspace: target rows only."""
+    B, G1, V = target_logits.shape
+    _check(_lib.bs_verify_walk_drafted(_ptr(target_logits), _ptr(draft_logits), _dtype_code(target_logits),
+                                       _ptr(draft_tokens), _ptr(gamma), _ptr(u_accept), _ptr(u_resample),
+                                       float(temperature), B, G1 - 1, V, _ptr(accept_len), _ptr(p_tok), _ptr(q_tok),
+                                       _ptr(out_tokens), _ptr(out_len), _ptr(workspace), workspace.numel(),
+                                       _stream(stream)), "bs_verify_walk_drafted")
 
 
 def verify_round_walk(target_logits, draft_logits, draft_tokens, gamma, u_accept, u_resample,

@@ -40,6 +40,7 @@ struct WalkParams {
     ResidParams r;         // the same logits for the residual pass, its outputs, piece masses
     uint32_t* dec;         // [B] decision word: (positions decided << 1) | last one accepted
     int nG;                // CTAs per sequence
+    int drafted;           // 1: the draft rows' statistics were left by bs_draft_sample: stream target rows only
 };
 
 // Per-stage record, written by the producer.
@@ -193,7 +194,7 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                 // ---- position k: this CTA's share of target row k and, below gamma, draft row k ----
                 {
                     const int k = sq.k;
-                    const int nrows = (!GREEDY && k < g) ? 2 : 1;
+                    const int nrows = (!GREEDY && !p.drafted && k < g) ? 2 : 1;
                     const int items = nrows * v.nseg;
                     const int i0 = (int)((long long)items * part / p.nG), i1 = (int)((long long)items * (part + 1) / p.nG);
                     for (int i = i0; i < i1 && ok; ++i) {
@@ -336,7 +337,7 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                 unsigned old = 0;
                 if (lane == 0) old = atomicAdd(v.ticket + b, (unsigned)len);
                 old = __shfl_sync(0xffffffffu, old, 0);
-                if (old + (unsigned)len != wk_cum<false>(k, g, v.nseg)) continue;
+                if (old + (unsigned)len != (p.drafted ? wk_cum<true>(k, g, v.nseg) : wk_cum<false>(k, g, v.nseg))) continue;
                 // ---- position k is complete: merge its rows (lane 0: target, lane 1: draft), decide ----
                 __threadfence();
                 // lanes 0..15 merge the partials of target row k, lanes 16..31 those of draft row k
@@ -344,7 +345,7 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                     const int half = lane >> 4, hl = lane & 15;
                     const int rr = half == 0 ? k : v.Gmax + 1 + k;
                     Online o{-INFINITY, 0.f};
-                    if (half == 0 || k < g) {
+                    if (half == 0 || (k < g && !p.drafted)) {
                         const float2* qq = v.partial + ((size_t)b * v.R + rr) * v.S;
                         for (int q = hl; q < v.nseg; q += 16) {
                             const float2 t = __ldcg(qq + q);
@@ -357,7 +358,7 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                     float Z = o.s * rescale(o.m, M, v.c);
 #pragma unroll
                     for (int off = 8; off > 0; off >>= 1) Z += __shfl_xor_sync(0xffffffffu, Z, off);
-                    if (hl == 0 && (half == 0 || k < g)) {
+                    if (hl == 0 && (half == 0 || (k < g && !p.drafted))) {
                         s_fin[half] = make_float2(M, Z);
                         v.row_stats[(size_t)b * v.R + rr] = make_float2(M, Z);
                     }
@@ -365,6 +366,13 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                 __syncwarp();
                 const float2 ts = s_fin[0];
                 int bits = (k == 0 && graw != g) ? BS_DEV_BAD_GAMMA : 0;
+                bool missing = false;                          // drafted mode: position k was never drafted
+                if (p.drafted && k < g) {
+                    if (lane == 0) s_fin[1] = __ldcg(v.row_stats + (size_t)b * v.R + v.Gmax + 1 + k);
+                    missing = ((__ldcg(v.draft_ready + b) >> k) & 1u) == 0u;
+                    if (missing) bits |= BS_DEV_DRAFT_MISSING;
+                    __syncwarp();
+                }
                 if (!(ts.y > 0.f) || !isfinite(ts.y) || !isfinite(ts.x)) bits |= BS_DEV_NONFINITE;
                 bool acc = false;
                 float pj = 0.f, qj = 0.f;
@@ -373,7 +381,7 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                     if (!(ds.y > 0.f) || !isfinite(ds.y) || !isfinite(ds.x)) bits |= BS_DEV_NONFINITE;
                     if (bad) {
                         bits |= BS_DEV_BAD_TOKEN;
-                    } else {
+                    } else if (!missing) {
                         // log2 of the two probabilities; the ratio is formed in the log domain
                         const float lp = (tl - ts.x) * v.c - log2f(ts.y);
                         const float lq = (dl - ds.x) * v.c - log2f(ds.y);
@@ -423,6 +431,7 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                 if (lane == 0) {                               // leave the workspace clean for the next call
                     v.ticket[b] = 0u;
                     p.dec[b] = 0u;
+                    if (p.drafted) v.draft_ready[b] = 0u;      // consumed: a later round must draft again
                 }
             }
         }
@@ -574,11 +583,11 @@ static bs_status launch_walk(WalkParams& p, cudaStream_t st) {
 
 using namespace bs;
 
-extern "C" bs_status bs_verify_walk(const void* target_logits, const void* draft_logits, bs_dtype dtype,
-                                    const int32_t* draft_tokens, const int32_t* gamma, const float* u_accept,
-                                    const float* u_resample, float temperature, int B, int Gmax, int V,
-                                    int32_t* accept_len, float* p_tok, float* q_tok, int32_t* out_tokens,
-                                    int32_t* out_len, void* workspace, size_t workspace_bytes, void* stream) {
+static bs_status run_walk(const void* target_logits, const void* draft_logits, bs_dtype dtype,
+                          const int32_t* draft_tokens, const int32_t* gamma, const float* u_accept,
+                          const float* u_resample, float temperature, int B, int Gmax, int V,
+                          int32_t* accept_len, float* p_tok, float* q_tok, int32_t* out_tokens,
+                          int32_t* out_len, void* workspace, size_t workspace_bytes, void* stream, int drafted) {
     if (B < 1 || Gmax < 0 || V < 1) return BS_ERR_INVALID_ARG;
     if (B > BS_MAX_BATCH || Gmax > BS_MAX_GAMMA || V > BS_MAX_VOCAB) return BS_ERR_UNSUPPORTED;
     if (dtype != BS_F32 && dtype != BS_BF16) return BS_ERR_INVALID_ARG;
@@ -626,7 +635,26 @@ extern "C" bs_status bs_verify_walk(const void* target_logits, const void* draft
     // decision words: the second B words of the per-row counter slot (the first B mark drafted positions)
     p.dec = v.ticket_row + B;
     p.nG = 1;
+    p.drafted = (drafted && !greedy) ? 1 : 0;         // greedy rounds never read draft rows anyway
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (greedy) return dtype == BS_F32 ? launch_walk<float, true>(p, st) : launch_walk<__nv_bfloat16, true>(p, st);
     return dtype == BS_F32 ? launch_walk<float, false>(p, st) : launch_walk<__nv_bfloat16, false>(p, st);
+}
+
+extern "C" bs_status bs_verify_walk(const void* target_logits, const void* draft_logits, bs_dtype dtype,
+                                    const int32_t* draft_tokens, const int32_t* gamma, const float* u_accept,
+                                    const float* u_resample, float temperature, int B, int Gmax, int V,
+                                    int32_t* accept_len, float* p_tok, float* q_tok, int32_t* out_tokens,
+                                    int32_t* out_len, void* workspace, size_t workspace_bytes, void* stream) {
+    return run_walk(target_logits, draft_logits, dtype, draft_tokens, gamma, u_accept, u_resample, temperature, B, Gmax,
+                    V, accept_len, p_tok, q_tok, out_tokens, out_len, workspace, workspace_bytes, stream, 0);
+}
+
+extern "C" bs_status bs_verify_walk_drafted(const void* target_logits, const void* draft_logits, bs_dtype dtype,
+                                            const int32_t* draft_tokens, const int32_t* gamma, const float* u_accept,
+                                            const float* u_resample, float temperature, int B, int Gmax, int V,
+                                            int32_t* accept_len, float* p_tok, float* q_tok, int32_t* out_tokens,
+                                            int32_t* out_len, void* workspace, size_t workspace_bytes, void* stream) {
+    return run_walk(target_logits, draft_logits, dtype, draft_tokens, gamma, u_accept, u_resample, temperature, B, Gmax,
+                    V, accept_len, p_tok, q_tok, out_tokens, out_len, workspace, workspace_bytes, stream, 1);
 }

@@ -158,3 +158,40 @@ def test_drafted_round_full_size(lib):
         res.append((acc, p, q))
     assert torch.equal(res[0][0], res[1][0])
     assert torch.allclose(res[0][1], res[1][1], atol=1e-6, rtol=0) and torch.allclose(res[0][2], res[1][2], atol=1e-6, rtol=0)
+
+
+def test_drafted_walk_equals_plain_walk_and_the_oracle(lib):
+    """draft -> bs_verify_walk_drafted against bs_verify_walk on the same tokens and against the oracle;
+    two rounds on one workspace; an undrafted position is reported."""
+    rng = np.random.default_rng(8)
+    B, G, V, T = 10, 5, 40000, 0.9
+    ws = lib.new_workspace(B, G, V, DEV); ws2 = lib.new_workspace(B, G, V, DEV)
+    for rnd_i in range(2):
+        t, d = _logits(300 + rnd_i, B, G, V, torch.float32, sigma=0.6)
+        gamma = rng.integers(0, G + 1, size=B).astype(np.int32); gamma[0] = G
+        un = wl.round_uniforms(13, rnd_i + 1, B, G)
+        gamma_d = torch.as_tensor(gamma, device=DEV)
+        u_acc = torch.as_tensor(un.u_accept, device=DEV); u_res = torch.as_tensor(un.u_resample, device=DEV)
+        tok = _draft_all(lib, d, gamma_d, torch.as_tensor(un.u_draft, device=DEV), T, ws)
+        tok = torch.where(tok < 0, torch.zeros_like(tok), tok).contiguous()
+        outs = []
+        for fn, w_ in ((lib.bs_verify_walk_drafted, ws), (lib.bs_verify_walk, ws2)):
+            acc = torch.zeros(B, dtype=torch.int32, device=DEV); p = torch.zeros(B, G, device=DEV); q = torch.zeros(B, G, device=DEV)
+            ot = torch.zeros(B, G + 1, dtype=torch.int32, device=DEV); ol = torch.zeros(B, dtype=torch.int32, device=DEV)
+            fn(t, d, tok, gamma_d, u_acc, u_res, T, acc, p, q, ot, ol, w_)
+            torch.cuda.synchronize()
+            assert (lib.bs_get_device_status(w_, B, G, V) & ~lib.BS_DEV_RESIDUAL_FALLBACK == 0).all()
+            outs.append(lib.RoundOutput(acc, p, q, ot, ol, w_))
+        a, b_ = outs
+        assert torch.equal(a.accept_len, b_.accept_len) and torch.equal(a.out_tokens, b_.out_tokens)
+        assert torch.allclose(a.p_tok, b_.p_tok, atol=1e-6, rtol=0) and torch.allclose(a.q_tok, b_.q_tok, atol=1e-6, rtol=0)
+        rin = wl.RoundInputs(target=t, draft=d, tokens=tok, gamma=gamma, uniforms=un)
+        tally = parity.Tally()
+        parity.check_round(a, rin, T, tally, where=f"drafted walk round {rnd_i}", walk=True)
+    # nothing drafted this time: every sequence with gamma > 0 is reported and accepts nothing
+    acc = torch.full((B,), -1, dtype=torch.int32, device=DEV)
+    ot = torch.zeros(B, G + 1, dtype=torch.int32, device=DEV); ol = torch.zeros(B, dtype=torch.int32, device=DEV)
+    lib.bs_verify_walk_drafted(t, d, tok, gamma_d, u_acc, u_res, T, acc, None, None, ot, ol, ws)
+    st = lib.bs_get_device_status(ws, B, G, V)
+    for b in range(B):
+        assert bool(st[b] & lib.BS_DEV_DRAFT_MISSING) == (gamma[b] > 0) and (gamma[b] == 0 or int(acc[b]) == 0)
