@@ -142,3 +142,25 @@ def test_lmhead_full_size(lib):
     # a second call on the same inputs is bit-identical
     out2, lt2, ld2 = run_lmhead(lib, inp, B, G, V, w.temperature)
     assert torch.equal(lt, lt2) and torch.equal(ld, ld2) and torch.equal(out.out_tokens, out2.out_tokens)
+
+
+def _lm_shapes(n, seed):
+    rng = np.random.default_rng(seed)
+    return [(int(rng.integers(1, 60)), int(rng.integers(0, 6)), int(rng.choice([8, 264, 1000, 2056, 4104, 8200])),
+             int(rng.choice([8, 72, 200, 264, 520])), int(rng.choice([8, 64, 136, 328]))) for _ in range(n)]
+
+
+@pytest.mark.parametrize("B,G,V,d_t,d_d", _lm_shapes(12, 7))
+def test_lmhead_random_shapes(lib, B, G, V, d_t, d_d):
+    """Row counts on both sides of one and two 128-row tiles, k-extents that are not multiples of the
+    64-deep stage, vocabularies that end inside a tile, speculation length 0 (no draft product)."""
+    w = wl.LmHeadWorkload("r", B=B, gamma=G, V=V, d_t=d_t, d_d=d_d, temperature=1.0, seed=B * 100 + V)
+    rng = np.random.default_rng(B + V + d_t)
+    gam = rng.integers(0, G + 1, size=B).astype(np.int32)
+    inp = wl.make_lmhead_inputs(w, 1, DEV, gamma=gam)
+    out, lt, ld = run_lmhead(lib, inp, B, G, V, 1.0)
+    check_logits(lt.view(-1, V), inp.H_t, inp.W_t, slice(None), "target")
+    if G > 0:
+        check_logits(ld.view(-1, V), inp.H_d, inp.W_d, slice(None), "draft")
+    t = check_verify(lib, out, lt, ld, inp, 1.0, f"lmhead random B={B} G={G} V={V}")
+    assert t.sequences == B
