@@ -46,6 +46,13 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
+// Hands a ring slot back safely: a bulk copy writes shared memory through the asynchronous proxy,
+// which is not ordered after this thread's ordinary shared loads by the mbarrier arrive alone.  Every
+// lane that read the slot runs this fence before the warp's arrive on the slot's "empty" barrier, so
+// the refill cannot overtake a load that is still in flight.
+__device__ __forceinline__ void fence_reads_before_refill() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));

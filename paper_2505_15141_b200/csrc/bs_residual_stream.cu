@@ -223,6 +223,7 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
                 d[q] = f.bonus ? a[q] : lds128(base + (uint32_t)(kResSegBytes + q * 512));
             }
         }
+        fence_reads_before_refill();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&s_empty[slot]));  // the slot's data is in registers now
         float acc = 0.f;

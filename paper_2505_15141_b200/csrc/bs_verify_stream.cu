@@ -301,6 +301,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) verify_stream_kernel(const 
             for (int q = 0; q < kVecPerThread; ++q)
                 v[q] = (q * kConsumers + tid < nvec) ? lds128(base + (uint32_t)(q * kConsumers) * 16u) : neg_inf_vec<T>();
         }
+        fence_reads_before_refill();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&s_empty[slot]));  // the slot's data is in registers now
         if (GREEDY) argmax_add<T, kVecPerThread>(am, v, m_sg * p.seg + tid * kVec, kConsumers * kVec);

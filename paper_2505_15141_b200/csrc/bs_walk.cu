@@ -457,6 +457,7 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
             for (int q = 0; q < kWkVecPerThread; ++q)
                 x[q] = (q * kWkConsumers + tid < m.nvec) ? lds128(base + (uint32_t)(q * kWkConsumers + tid) * 16u)
                                                          : neg_inf_vec<T>();
+            fence_reads_before_refill();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&s_empty[slot]));
             if (GREEDY) {
@@ -488,6 +489,7 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                     d[q] = f.bonus ? a[q] : lds128(pb + (uint32_t)(kResSegBytes + q * 512));
                 }
             }
+            fence_reads_before_refill();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&s_empty[slot]));
             float acc = 0.f;
