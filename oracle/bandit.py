@@ -16,6 +16,16 @@ eta_t uses the current round index t >= 1; exp(-eta * S) is evaluated after
 subtracting min S (same distribution); I_t ~ p_t is drawn by inverse CDF from
 one uniform, smallest i whose cumulative probability strictly exceeds u.
 
+UCBSpecReward is UCBSpec fed a real-valued reward (Section 6.2 takes the current
+throughput, generated tokens per second, as the reward and gives no formula).  Reading: the
+listing of Algorithm 8 is kept, the history holds the real rewards, and the factor L/2 of the
+confidence radius -- half the width of the interval [1, L+1] the accepted length lives in --
+becomes half the width W of the interval [0, W] the caller declares for its reward.
+throughput_reward is the reward itself: tokens emitted in the round over the seconds the round
+took, per sequence or for the whole batch.  Their pins: UCBSpecReward with W = L and the
+accepted length as reward plays UCBSpec's arms; scaling rewards and W together, or shifting
+every reward, leaves the arms unchanged; a hand-worked trajectory (tests/golden).
+
 Pins (tests/test_oracle_bandit.py): the round-robin prefix, hand-worked arm
 sequences for scripted rewards (tests/golden), a hand-worked radius value,
 monotonicity of the radius, p_1 uniform and sum p = 1, p_t against
@@ -33,7 +43,7 @@ UCB_TIE = 1e-9     # top-two index values closer than this (and not bit-equal): 
 ARM_CDF_TIE = 1e-9  # u_arm within this of an EXP3 CDF edge: flagged
 
 
-def confidence_radius(L: int, K: int, t: int, n: int, delta: float) -> float:
+def confidence_radius(L: float, K: int, t: int, n: int, delta: float) -> float:
     """cr_{i,t} of Algorithm 4: (L/2) sqrt( (1+n)/n^2 * (1 + 2 log(K t^2 (1+n)^(1/2) / delta)) )."""
     return (L / 2.0) * math.sqrt((1.0 + n) / (n * n)
                                  * (1.0 + 2.0 * math.log(K * t * t * math.sqrt(1.0 + n) / delta)))
@@ -151,3 +161,78 @@ class EXP3Spec:
             a = int(arm[b])
             self.S[b, a] += self.loss_estimate(b, a, int(y[b]))
             self.t[b] += 1
+
+
+class UCBSpecReward:
+    """Algorithm 8 with a real reward in [0, W] in place of the accepted length (Section 6.2: the
+    reward is the current throughput; arms are speculation lengths, gamma = 0 being canonical
+    decoding, Algorithm 1)."""
+
+    def __init__(self, B: int, arm_gamma: Sequence[int], width: float, delta: float = 0.5):
+        self.B, self.K = B, len(arm_gamma)
+        self.arm_gamma = np.asarray(arm_gamma, dtype=np.int64)
+        self.W = float(width)
+        self.delta = float(delta)
+        self.n = np.zeros((B, self.K), dtype=np.int64)
+        self.sumR = np.zeros((B, self.K), dtype=np.float64)  # sum of the rewards of arm i, in the order received
+        self.t = np.zeros(B, dtype=np.int64)
+        self.last_index = np.full((B, self.K), np.nan)
+
+    def index_values(self, b: int) -> np.ndarray:
+        t = int(self.t[b])
+        out = np.empty(self.K)
+        for i in range(self.K):
+            n = int(self.n[b, i])
+            out[i] = self.sumR[b, i] / n + confidence_radius(self.W, self.K, t, n, self.delta)
+        return out
+
+    def select(self, active: Optional[np.ndarray] = None):
+        arm = np.full(self.B, -1, dtype=np.int64)
+        flagged = np.zeros(self.B, dtype=bool)
+        for b in range(self.B):
+            if active is not None and not active[b]:
+                continue
+            t = int(self.t[b])
+            if t < self.K:
+                arm[b] = t
+                continue
+            ucb = self.index_values(b)
+            self.last_index[b] = ucb
+            a = int(np.argmax(ucb))
+            arm[b] = a
+            if self.K > 1:
+                second = np.partition(ucb, -2)[-2]
+                flagged[b] = (ucb[a] - second) < UCB_TIE * max(1.0, self.W) and ucb[a] != second
+        gamma = np.where(arm >= 0, self.arm_gamma[np.maximum(arm, 0)], 0)
+        return arm, gamma, flagged
+
+    def update(self, arm: np.ndarray, reward: np.ndarray, active: Optional[np.ndarray] = None):
+        """Rewards outside [0, W] are clamped into it; NaN counts as 0."""
+        for b in range(self.B):
+            if active is not None and not active[b]:
+                continue
+            a = int(arm[b])
+            r = float(reward[b])
+            r = 0.0 if math.isnan(r) else min(max(r, 0.0), self.W)
+            self.n[b, a] += 1
+            self.sumR[b, a] += r
+            self.t[b] += 1
+
+
+def throughput_reward(y: np.ndarray, seconds: float, whole_batch: bool,
+                      active: Optional[np.ndarray] = None) -> np.ndarray:
+    """Tokens per second of the round (Section 6.2).  y[b]: tokens sequence b emitted in the round
+    (accepted drafts plus the resampled or bonus token).  Per sequence: y[b] / seconds.  Whole
+    batch: (sum of y over the active sequences) / seconds for every active sequence, so bandits
+    started together stay together and the batch shares one speculation length.  Inactive: 0."""
+    y = np.asarray(y, dtype=np.int64)
+    act = np.ones(len(y), dtype=bool) if active is None else np.asarray(active, dtype=bool)
+    out = np.zeros(len(y), dtype=np.float64)
+    if whole_batch:
+        total = int(y[act].sum())
+        out[act] = float(total) / float(seconds)
+    else:
+        for b in range(len(y)):
+            if act[b]:
+                out[b] = float(int(y[b])) / float(seconds)
+    return out

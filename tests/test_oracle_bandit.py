@@ -173,3 +173,78 @@ def test_active_mask_freezes_sequences():
     assert arm[1] == -1 and gamma[1] == 0
     u.update(arm, np.array([2, 2]), act)
     assert u.t[0] == 1 and u.t[1] == 0 and u.n[1].sum() == 0
+
+
+# ---- UCBSpec with a real reward (Section 6.2) ----------------------------------------------------
+
+def test_ucbspec_reward_scripted_trajectory():
+    rows = golden_lines("ucbspec_reward_scripted.txt")
+    u = ob.UCBSpecReward(1, [0, 3], width=10.0, delta=0.5)
+    for f in rows:
+        arm, gamma, _ = u.select()
+        assert int(arm[0]) == int(f[1]) and int(gamma[0]) == [0, 3][int(f[1])], f
+        if f[3] != "rr":
+            assert np.allclose(u.last_index[0], [float(f[3]), float(f[4])], atol=2e-6), f
+        u.update(arm, np.array([float(f[2])]))
+    assert list(u.n[0]) == [4, 4] and list(u.sumR[0]) == [13.25, 13.5] and u.t[0] == 8
+
+
+def test_ucbspec_reward_with_accepted_lengths_plays_ucbspec():
+    """W = L and reward = accepted length - 1 (the accepted length lives in [1, L+1], an interval of
+    width L): the listing of UCBSpec with every mean lowered by one, so the same arms."""
+    rng = np.random.default_rng(3)
+    gam = [1, 2, 4, 6]
+    a, r = ob.UCBSpec(5, gam, delta=0.5), ob.UCBSpecReward(5, gam, width=6.0, delta=0.5)
+    for t in range(300):
+        arm_a, g_a, fl = a.select()
+        arm_r, g_r, _ = r.select()
+        same = arm_a == arm_r
+        assert (same | fl).all() and (g_a[same] == g_r[same]).all()
+        if t >= 4:
+            assert np.allclose(a.last_index, r.last_index + 1.0, rtol=0, atol=1e-12)
+        y = np.array([rng.integers(1, gam[i] + 2) for i in arm_a])
+        a.update(arm_a, y)
+        r.update(arm_a, (y - 1).astype(np.float64))
+    assert np.array_equal(a.n, r.n) and np.array_equal((a.sumY - a.n).astype(np.float64), r.sumR)
+
+
+def test_ucbspec_reward_scale_and_shift_leave_the_arms_unchanged():
+    """Index = mean + (W/2) f(n, t): scaling rewards and W by c scales every index by c; adding a
+    constant to every reward adds it to every index.  Either way the arg-max stays."""
+    rng = np.random.default_rng(4)
+    gam = [0, 1, 2, 3, 4]
+    base = ob.UCBSpecReward(1, gam, width=8.0)
+    scaled = ob.UCBSpecReward(1, gam, width=8.0 * 4.0)               # powers of two: exact scaling
+    shifted = ob.UCBSpecReward(1, gam, width=8.0)
+    means = np.array([2.0, 2.6, 3.1, 2.9, 2.2])
+    for t in range(400):
+        arm, _, flagged = base.select()
+        a2, a3 = scaled.select()[0], shifted.select()[0]
+        assert (arm == a2).all()
+        assert (arm == a3).all() or flagged.any()
+        if t >= 5:
+            assert np.array_equal(scaled.last_index, 4.0 * base.last_index)
+            assert np.allclose(shifted.last_index, base.last_index + 0.5, rtol=0, atol=1e-12)
+        r = np.clip(means[arm] + rng.normal(0, 0.7, size=1), 0.0, 7.0)
+        r = np.round(r * 64) / 64                                    # dyadic rewards: sums are exact
+        base.update(arm, r); scaled.update(arm, 4.0 * r); shifted.update(arm, r + 0.5)
+    assert base.n[0].argmax() == 2                                   # and it has found the best arm
+
+
+def test_ucbspec_reward_clamps_into_the_declared_range():
+    u = ob.UCBSpecReward(1, [0, 1], width=5.0)
+    for r in (7.5, -1.0, float("nan"), 2.0):
+        arm, _, _ = u.select() if u.t[0] < 2 else (np.array([0]), None, None)
+        u.update(np.array([0]), np.array([r]))
+    assert u.sumR[0, 0] == 5.0 + 0.0 + 0.0 + 2.0 and u.n[0, 0] == 4
+
+
+def test_throughput_reward_closed_forms():
+    y = np.array([3, 1, 2, 5])
+    assert list(ob.throughput_reward(y, 0.5, whole_batch=False)) == [6.0, 2.0, 4.0, 10.0]
+    assert list(ob.throughput_reward(y, 0.5, whole_batch=True)) == [22.0] * 4
+    act = np.array([1, 0, 1, 1], dtype=bool)
+    assert list(ob.throughput_reward(y, 0.25, whole_batch=False, active=act)) == [12.0, 0.0, 8.0, 20.0]
+    assert list(ob.throughput_reward(y, 0.25, whole_batch=True, active=act)) == [40.0, 0.0, 40.0, 40.0]
+    # gamma = 0 everywhere (canonical decoding): one token per sequence and round
+    assert list(ob.throughput_reward(np.ones(3, dtype=np.int64), 2.0, whole_batch=True)) == [1.5] * 3
