@@ -60,7 +60,7 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--workload", default="qwen_exp3",
-                    choices=["tiny_ucb", "llama2_fixed", "llama3_ucb", "qwen_exp3", "lmhead_llama3",
+                    choices=["tiny_ucb", "llama2_fixed", "llama3_ucb", "qwen_exp3", "llama3_tput", "lmhead_llama3",
                              "lmhead_llama3_b128"])
     ap.add_argument("--batch", type=int, default=0,
                     help="override the workload's batch size (smaller cases for profiler captures)")
@@ -249,7 +249,8 @@ def run_cuda(args, w):
     from paper_2505_15141_b200 import binding as bs, workloads as wl
 
     B, K, G, V = w.B, w.K, w.Gmax, w.V
-    alg = bs.BS_EXP3 if w.alg == "exp3" else bs.BS_UCB        # a fixed arm is a 1-armed UCBSpec
+    alg = {"exp3": bs.BS_EXP3, "ucb_reward": bs.BS_UCB_REWARD}.get(w.alg, bs.BS_UCB)   # a fixed arm is a 1-armed UCBSpec
+    reward = w.alg == "ucb_reward"
     es = w.elem_size
     arm_gamma = np.asarray(w.arm_gamma)
 
@@ -265,8 +266,26 @@ def run_cuda(args, w):
             u_resample=torch.as_tensor(rnd.uniforms.u_resample, device=dev),
             u_arm=torch.as_tensor(rnd.uniforms.u_arm, device=dev),
             u_draft=torch.as_tensor(rnd.uniforms.u_draft, device=dev), rnd=rnd))
-    state = bs.new_bandit(alg, B, w.arm_gamma, w.delta, dev)
+    state = bs.new_bandit(alg, B, w.arm_gamma, w.delta, dev, reward_width=w.reward_width if reward else None)
     ws = bs.new_workspace(B, G, V, dev)
+    reward_d = torch.zeros(B, dtype=torch.float64, device=dev)
+    # Throughput reward: a serving loop passes the duration it measured for the step; the arms are chosen on
+    # the device here and never read back inside the timed region, so the duration is one constant, the
+    # workload's stand-in for a step at the longest speculation length.
+    step_s = wl.step_seconds(w, arm_gamma) if reward else None
+
+    def update_call():
+        if reward:
+            bs.bs_throughput_reward(out_len, None, B, step_s, w.whole_batch, reward_d)
+            bs.bs_bandit_update_reward(state, B, K, arm_d, reward_d)
+        else:
+            bs.bs_bandit_update(state, alg, B, K, arm_d, out_len)
+
+    def init_call():
+        if reward:
+            bs.bs_bandit_init_reward(state, B, K, w.arm_gamma, w.delta, w.reward_width)
+        else:
+            bs.bs_bandit_init(state, alg, B, K, w.arm_gamma, w.delta)
     arm_d = torch.zeros(B, dtype=torch.int32, device=dev)
     gamma_d = torch.zeros(B, dtype=torch.int32, device=dev)
     accept_len = torch.zeros(B, dtype=torch.int32, device=dev)
@@ -304,7 +323,7 @@ def run_cuda(args, w):
             if drafted:
                 draft_calls(s)
             walk_call(s)
-            bs.bs_bandit_update(state, alg, B, K, arm_d, out_len)
+            update_call()
             return
         if drafted:
             draft_calls(s)
@@ -312,7 +331,7 @@ def run_cuda(args, w):
         verify_call(s)
         bs.bs_residual_sample(s["target"], s["draft"], s["tokens"], gamma_d, accept_len, s["u_resample"],
                               w.temperature, out_tokens, out_len, ws)
-        bs.bs_bandit_update(state, alg, B, K, arm_d, out_len)
+        update_call()
 
     side = torch.cuda.Stream(device=dev)
     graphs = []
@@ -327,7 +346,7 @@ def run_cuda(args, w):
                 graphs.append(g)
         torch.cuda.synchronize()
         # start from a clean bandit: the capture warm-up above played one round
-        bs.bs_bandit_init(state, alg, B, K, w.arm_gamma, w.delta)
+        init_call()
 
     def run_step(i):
         if graphs:
@@ -402,7 +421,7 @@ def run_cuda(args, w):
         if walk:                                               # rows the walk had to read: up to the stop position
             tau = accept_len.to(torch.int64); gm = gamma_d.to(torch.int64)
             walk_rows += (tau + 1).sum() if drafted else torch.where(tau < gm, 2 * (tau + 1), 2 * gm + 1).sum()
-        bs.bs_bandit_update(state, alg, B, K, arm_d, out_len)
+        update_call()
         y_sum += out_len.sum()
     torch.cuda.synchronize()
     verify_ms = sum(a.elapsed_time(b) for a, b in evs) / ksteps
@@ -431,7 +450,7 @@ def run_cuda(args, w):
         def walk_step(s):
             bs.bs_bandit_select(state, alg, B, K, s["u_arm"], None, arm_d, gamma_d)
             walk_call(s)
-            bs.bs_bandit_update(state, alg, B, K, arm_d, out_len)
+            update_call()
         for i in range(min(args.warmup, 5)):
             walk_step(sets[i % ring])
         sync_all()
@@ -521,7 +540,7 @@ def run_cuda(args, w):
                          "ms_per_launch": verify_ms, "residual_ms_per_launch": resid_ms},
             "e2e": e2e, "cpu_baseline": cpu, "clocks": clocks, "variants": variants,
             "other_workloads": getattr(args, "others", None),
-            "gpu_launches": ((3 if walk else 4) + (2 * G if drafted else 0)) * args.steps,
+            "gpu_launches": ((3 if walk else 4) + (2 * G if drafted else 0) + (1 if reward else 0)) * args.steps,
         }
         if walk:
             line["roofline"]["kernel"] = "verify_walk_kernel (bs_verify_walk)"
@@ -763,7 +782,7 @@ def run_lmhead(args, w):
         dist.destroy_process_group()
 
 
-OTHER_WORKLOADS = ("llama3_ucb", "llama2_fixed", "lmhead_llama3", "lmhead_llama3_b128")
+OTHER_WORKLOADS = ("llama3_ucb", "llama2_fixed", "llama3_tput", "lmhead_llama3", "lmhead_llama3_b128")
 
 
 def other_workloads_summary():

@@ -53,7 +53,7 @@ typedef enum {
 } bs_status;
 
 typedef enum { BS_F32 = 0, BS_BF16 = 1 } bs_dtype;
-typedef enum { BS_UCB = 0, BS_EXP3 = 1 } bs_alg;
+typedef enum { BS_UCB = 0, BS_EXP3 = 1, BS_UCB_REWARD = 2 } bs_alg;
 
 /* Per-sequence device status bits (bs_get_device_status). */
 #define BS_DEV_BAD_GAMMA   1   /* gamma[b] outside [0, Gmax]; the sequence was processed as gamma = 0 */
@@ -317,6 +317,40 @@ bs_status bs_bandit_update(void* state, size_t state_bytes, bs_alg alg, int B, i
 bs_status bs_bandit_read(const void* state, size_t state_bytes, bs_alg alg, int B, int K,
                          int64_t* n_host, int64_t* sumY_host, double* S_host, int64_t* t_host,
                          void* stream);
+
+/* ---- throughput as the reward (Section 6.2) -------------------------------------------
+ * Section 6.2 runs UCBSpec over the speculation lengths {0, ..., 4} (0 = canonical decoding,
+ * Algorithm 1) with "the current throughput", generated tokens per second, as the reward, and
+ * prints no formula.  Reading: alg = BS_UCB_REWARD is Algorithm 8 with the history holding
+ * real rewards r in [0, W] and the radius factor L/2 (half the width of [1, L+1], where the
+ * accepted length lives) replaced by W/2.  bs_bandit_state_bytes, bs_bandit_select and
+ * bs_bandit_read take BS_UCB_REWARD; bs_bandit_init and bs_bandit_update do not (they return
+ * BS_ERR_INVALID_ARG): use the two calls below.  bs_bandit_read: n_host [B,K] int64 pulls,
+ * S_host [B,K] fp64 reward sums, t_host [B] int64; sumY_host unused. */
+
+/* bs_bandit_init for BS_UCB_REWARD.  reward_width = W > 0, finite.  arm_gamma may be all
+ * zero (L is not used by this algorithm). */
+bs_status bs_bandit_init_reward(void* state, size_t state_bytes, int B, int K,
+                                const int32_t* arm_gamma_host, double delta, double reward_width,
+                                void* stream);
+
+/* n[arm] += 1, sumR[arm] += r, t += 1 for every active sequence.
+ *  arm [B] int32 device, as returned by select;  reward [B] fp64 device: values outside
+ *  [0, W] are clamped into it, NaN counts as 0. */
+bs_status bs_bandit_update_reward(void* state, size_t state_bytes, int B, int K,
+                                  const int32_t* arm, const double* reward, const uint8_t* active,
+                                  void* stream);
+
+/* The round's throughput as a reward, on the device (fp64).
+ *  out_len [B] int32 device: tokens sequence b emitted in the round (bs_residual_sample)
+ *  seconds: HOST scalar > 0, finite: what the caller measured for the round
+ *  whole_batch = 0: reward[b] = out_len[b] / seconds
+ *  whole_batch = 1: reward[b] = (sum of out_len over the active sequences) / seconds for every
+ *                   active b -- bandits that start together then stay together, so the batch
+ *                   shares one speculation length, as one serving step does
+ *  reward [B] fp64 device out; inactive sequences get 0. */
+bs_status bs_throughput_reward(const int32_t* out_len, const uint8_t* active, int B, double seconds,
+                               int whole_batch, double* reward, void* stream);
 
 #ifdef __cplusplus
 }

@@ -25,7 +25,7 @@ _lib = C.CDLL(LIB_PATH)
 BS_OK = 0
 BS_ERR_INVALID_ARG, BS_ERR_CUDA, BS_ERR_UNSUPPORTED, BS_ERR_WORKSPACE, BS_ERR_TIMEOUT, BS_ERR_DEVICE_DATA = 1, 2, 3, 4, 5, 6
 BS_F32, BS_BF16 = 0, 1
-BS_UCB, BS_EXP3 = 0, 1
+BS_UCB, BS_EXP3, BS_UCB_REWARD = 0, 1, 2
 BS_DEV_BAD_GAMMA, BS_DEV_BAD_TOKEN, BS_DEV_NONFINITE, BS_DEV_RESIDUAL_FALLBACK, BS_DEV_DRAFT_MISSING = 1, 2, 4, 8, 16
 BS_MAX_GAMMA, BS_MAX_ARMS, BS_MAX_BATCH = 31, 32, 4096
 
@@ -54,6 +54,9 @@ SIGNATURES = {
     "bs_bandit_select": (_i, [_vp, _sz, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
     "bs_bandit_update": (_i, [_vp, _sz, _i, _i, _i, _vp, _vp, _vp, _vp]),
     "bs_bandit_read": (_i, [_vp, _sz, _i, _i, _i, _vp, _vp, _vp, _vp, _vp]),
+    "bs_bandit_init_reward": (_i, [_vp, _sz, _i, _i, _vp, _d, _d, _vp]),
+    "bs_bandit_update_reward": (_i, [_vp, _sz, _i, _i, _vp, _vp, _vp, _vp]),
+    "bs_throughput_reward": (_i, [_vp, _vp, _i, _d, _i, _vp, _vp]),
 }
 for _name, (_res, _args) in SIGNATURES.items():
     _fn = getattr(_lib, _name)
@@ -308,7 +311,8 @@ def bs_bandit_update(state, alg: int, B: int, K: int, arm, reward_y, active=None
 
 
 def bs_bandit_read(state, alg: int, B: int, K: int, stream=None) -> dict:
-    """Sufficient statistics as host arrays: UCBSpec {n, sumY, t}; EXP3Spec {S, n, t}."""
+    """Sufficient statistics as host arrays: UCBSpec {n, sumY, t}; EXP3Spec {S, n, t}; real-reward
+    UCBSpec {S (the reward sums), n, t}."""
     t = np.zeros(B, dtype=np.int64)
     if alg == BS_UCB:
         n = np.zeros((B, K), dtype=np.int64)
@@ -324,11 +328,35 @@ def bs_bandit_read(state, alg: int, B: int, K: int, stream=None) -> dict:
     return {"S": S, "n": n, "t": t}
 
 
-def new_bandit(alg: int, B: int, arm_gamma: Sequence[int], delta: float = 0.5, device="cuda") -> torch.Tensor:
+def bs_bandit_init_reward(state: torch.Tensor, B: int, K: int, arm_gamma: Sequence[int], delta: float,
+                          reward_width: float, stream=None) -> None:
+    ag = np.ascontiguousarray(np.asarray(arm_gamma, dtype=np.int32))
+    assert ag.shape == (K,)
+    _check(_lib.bs_bandit_init_reward(_ptr(state), state.numel(), B, K, ag.ctypes.data_as(_vp), float(delta),
+                                      float(reward_width), _stream(stream)), "bs_bandit_init_reward")
+
+
+def bs_bandit_update_reward(state, B: int, K: int, arm, reward, active=None, stream=None) -> None:
+    assert reward.dtype == torch.float64
+    _check(_lib.bs_bandit_update_reward(_ptr(state), state.numel(), B, K, _ptr(arm), _ptr(reward), _ptr(active),
+                                        _stream(stream)), "bs_bandit_update_reward")
+
+
+def bs_throughput_reward(out_len, active, B: int, seconds: float, whole_batch: bool, reward, stream=None) -> None:
+    assert out_len.dtype == torch.int32 and reward.dtype == torch.float64
+    _check(_lib.bs_throughput_reward(_ptr(out_len), _ptr(active), B, float(seconds), int(bool(whole_batch)),
+                                     _ptr(reward), _stream(stream)), "bs_throughput_reward")
+
+
+def new_bandit(alg: int, B: int, arm_gamma: Sequence[int], delta: float = 0.5, device="cuda",
+               reward_width: Optional[float] = None) -> torch.Tensor:
     K = len(arm_gamma)
     n = bs_bandit_state_bytes(alg, B, K)
     if n == 0:
         raise BanditSpecError(BS_ERR_UNSUPPORTED, "bs_bandit_state_bytes")
     state = torch.empty(n, dtype=torch.uint8, device=device)
-    bs_bandit_init(state, alg, B, K, arm_gamma, delta)
+    if alg == BS_UCB_REWARD:
+        bs_bandit_init_reward(state, B, K, arm_gamma, delta, reward_width)
+    else:
+        bs_bandit_init(state, alg, B, K, arm_gamma, delta)
     return state

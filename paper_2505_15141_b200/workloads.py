@@ -110,7 +110,7 @@ class Workload:
     temperature: float              # 0.0 = greedy
     rounds: int
     seed: int
-    alg: Optional[str]              # "ucb" | "exp3" | None (fixed arm 0)
+    alg: Optional[str]              # "ucb" | "exp3" | "ucb_reward" (throughput as the reward) | None (fixed arm 0)
     target_std: float = 3.0
     boost_prob: float = 0.05        # Bernoulli probability of a +boost entry
     boost: float = 8.0
@@ -120,6 +120,18 @@ class Workload:
     sigma_arms: Tuple[float, ...] = (0.3, 0.8, 1.5, 3.0)
     phase_len: int = 200
     delta: float = 0.5
+    # "ucb_reward" only: a stand-in for the measured duration of a decoding step, which the paper
+    # measures and this harness has no models to measure: one target pass plus gamma draft passes
+    step_target_s: float = 0.025
+    step_draft_s: float = 0.0015
+    step_verify_s: float = 0.0004   # extra per drafted position inside the target pass
+    whole_batch: bool = True        # the batch shares one reward (and so one speculation length)
+
+    @property
+    def reward_width(self) -> float:
+        """Upper end of the reward range: every sequence emits gamma_max + 1 tokens in the shortest step."""
+        per_seq = (self.Gmax + 1) / self.step_target_s
+        return per_seq * self.B if self.whole_batch else per_seq
 
     @property
     def K(self) -> int:
@@ -155,7 +167,21 @@ WORKLOADS = {
     # 152064-entry vocabulary, EXP3Spec, draft quality per arm rotates every 200 rounds
     "qwen_exp3": Workload("qwen_exp3", B=256, V=152064, arm_gamma=(1, 3, 5, 8), dtype="f32",
                           temperature=1.0, rounds=1000, seed=4, alg="exp3", sigma="per_arm_phase"),
+    # 128256-entry vocabulary, UCBSpec over the speculation lengths 0..4 (0 = canonical decoding) with the
+    # round's throughput as the reward; 48 sequences that share the reward
+    "llama3_tput": Workload("llama3_tput", B=48, V=128256, arm_gamma=(0, 1, 2, 3, 4), dtype="bf16",
+                            temperature=1.0, rounds=300, seed=6, alg="ucb_reward", sigma_fixed=1.2),
+    "tiny_tput": Workload("tiny_tput", B=6, V=1024, arm_gamma=(0, 1, 2, 3), dtype="f32",
+                          temperature=1.0, rounds=120, seed=7, alg="ucb_reward", whole_batch=False,
+                          target_std=2.0, boost_prob=0.0, sigma_fixed=0.7),
 }
+
+
+def step_seconds(w: Workload, gamma: np.ndarray) -> float:
+    """Stand-in for the measured duration of one decoding step of the batch: the draft model runs
+    max(gamma) times, the target model once over max(gamma) + 1 positions."""
+    g = int(np.max(gamma)) if len(gamma) else 0
+    return w.step_target_s + g * (w.step_draft_s + w.step_verify_s)
 
 
 def torch_generator(seed: int, rnd: int, device) -> torch.Generator:

@@ -139,14 +139,18 @@ def closed_loop(bs, w: wl.Workload, rounds: int, device, sample: Optional[Sequen
     the oracle side by side.  `sample`: sequences whose verification the oracle replays (default
     all); the oracle bandit of the others is fed the CUDA reward (teacher forcing)."""
     B, K, G, V = w.B, w.K, w.Gmax, w.V
-    alg = {None: None, "ucb": bs.BS_UCB, "exp3": bs.BS_EXP3}[w.alg]
+    alg = {None: None, "ucb": bs.BS_UCB, "exp3": bs.BS_EXP3, "ucb_reward": bs.BS_UCB_REWARD}[w.alg]
     tally = Tally()
     ws = bs.new_workspace(B, G, V, device)
     if carry is not None and "state" in carry:           # continue a trajectory started by an earlier call
         state, oracle_bandit = carry["state"], carry["oracle_bandit"]
     if alg is not None and state is None:
-        state = bs.new_bandit(alg, B, w.arm_gamma, w.delta, device)
-        oracle_bandit = ob.UCBSpec(B, w.arm_gamma, w.delta) if w.alg == "ucb" else ob.EXP3Spec(B, w.arm_gamma)
+        if w.alg == "ucb_reward":
+            state = bs.new_bandit(alg, B, w.arm_gamma, w.delta, device, reward_width=w.reward_width)
+            oracle_bandit = ob.UCBSpecReward(B, w.arm_gamma, w.reward_width, w.delta)
+        else:
+            state = bs.new_bandit(alg, B, w.arm_gamma, w.delta, device)
+            oracle_bandit = ob.UCBSpec(B, w.arm_gamma, w.delta) if w.alg == "ucb" else ob.EXP3Spec(B, w.arm_gamma)
     if carry is not None:
         carry["state"], carry["oracle_bandit"] = state, oracle_bandit
     arm_d = torch.zeros(B, dtype=torch.int32, device=device)
@@ -157,7 +161,7 @@ def closed_loop(bs, w: wl.Workload, rounds: int, device, sample: Optional[Sequen
             u_arm_d = torch.as_tensor(un.u_arm, device=device)
             bs.bs_bandit_select(state, alg, B, K, u_arm_d, None, arm_d, gamma_d)
             arm_gpu = to_np(arm_d).astype(np.int64)
-            if w.alg == "ucb":
+            if w.alg in ("ucb", "ucb_reward"):
                 arm_ref, _, flagged = oracle_bandit.select()
             else:
                 arm_ref, _, flagged = oracle_bandit.select(un.u_arm)
@@ -182,7 +186,17 @@ def closed_loop(bs, w: wl.Workload, rounds: int, device, sample: Optional[Sequen
             if r is not None:
                 y[b] = r.y                       # equal to the CUDA value unless the check failed
         assert (y == y_gpu).all()
-        if alg is not None:
+        if w.alg == "ucb_reward":
+            # the round's throughput as the reward; the duration is the workload's stand-in for a measurement
+            seconds = wl.step_seconds(w, np.asarray(w.arm_gamma)[arm])
+            rew_d = torch.empty(B, dtype=torch.float64, device=device)
+            bs.bs_throughput_reward(out.out_len, None, B, seconds, w.whole_batch, rew_d)
+            rew = ob.throughput_reward(y, seconds, w.whole_batch)
+            assert np.array_equal(rew_d.cpu().numpy(), rew), f"round {rnd_i}: throughput reward differs"
+            assert rew.max() <= w.reward_width
+            bs.bs_bandit_update_reward(state, B, K, arm_d, rew_d)
+            oracle_bandit.update(arm, rew)
+        elif alg is not None:
             bs.bs_bandit_update(state, alg, B, K, arm_d, out.out_len)
             oracle_bandit.update(arm, y)
     if alg is not None:
@@ -190,6 +204,8 @@ def closed_loop(bs, w: wl.Workload, rounds: int, device, sample: Optional[Sequen
         assert (st["t"] == oracle_bandit.t).all()
         if w.alg == "ucb":
             assert (st["n"] == oracle_bandit.n).all() and (st["sumY"] == oracle_bandit.sumY).all()
+        elif w.alg == "ucb_reward":                      # the same fp64 additions in the same order
+            assert (st["n"] == oracle_bandit.n).all() and np.array_equal(st["S"], oracle_bandit.sumR)
         else:
             rel = np.abs(st["S"] - oracle_bandit.S) / np.maximum(np.abs(oracle_bandit.S), 1e-12)
             tally.max_S_rel = max(tally.max_S_rel, float(rel.max()))
