@@ -42,8 +42,8 @@ FALLBACK_HBM_GBS = 6650.0
 # written per launch).  Captured on smaller cases of the same kernels; read traffic grows with the
 # bytes, the writes (workspace partials, write-backs) do not.  None = not captured.
 NCU_TRAFFIC = {
-    "qwen_exp3": (1.0002, 4.1e6),          # profiles/verify_stream_kernel.md, fp32 column
-    "llama3_ucb": (1.0005, 4.1e6),         # profiles/verify_stream_kernel.md, bf16 column
+    "qwen_exp3": (1.0003, 4.0e6),          # profiles/verify_stream_kernel.md, fp32 column
+    "llama3_ucb": (1.0005, 4.0e6),         # profiles/verify_stream_kernel.md, bf16 column
     "lmhead_llama3": (1.0000, 29.0e6),     # profiles/lmhead_gemm_kernel.md, B=16 (logits still dirty in L2 not counted)
     "lmhead_llama3_b128": (1.0232, 567.6e6),
 }
@@ -721,6 +721,11 @@ def run_lmhead(args, w):
                  "bytes_per_launch": nbytes, "flops_per_launch": flops,
                  "ms_per_launch": lm_ms, "residual_ms_per_launch": res_ms,
                  "hbm_gbs": gbs, "hbm_frac": gbs / hbm_peak, "tensor_tflops": tfs, "tensor_frac": tfs / tc_peak})
+    if peaks and peaks.get("bf16_tflops_sustained"):
+        # `peak` is the burst figure (the stricter one); the launches here run back to back under the
+        # power cap, where the library product itself settles at the sustained figure
+        sus = float(peaks["bf16_tflops_sustained"])
+        roof.update({"bf16_tflops_sustained": sus, "tensor_frac_of_sustained": tfs / sus})
 
     e2e = None
     if args.e2e_steps > 0:

@@ -55,3 +55,40 @@ def test_walk_round_repeats_bit_for_bit(lib):
                 & (o.p_tok == ref.p_tok).all() & (o.q_tok == ref.q_tok).all() & (o.out_len == ref.out_len).all())
         bad += (~same).to(torch.int64)
     assert int(bad) == 0, f"{int(bad)} of {reps} repetitions differ from the first"
+
+
+@pytest.mark.parametrize("name,reps", [("lmhead_llama3", 400), ("lmhead_llama3_b128", 150)])
+def test_lmhead_round_repeats_bit_for_bit(lib, name, reps):
+    """Both tile shapes of the fused LM head (rows <= 128 and > 128): logits, statistics, accepted
+    lengths and the tokens resampled from those logits."""
+    w = wl.LMHEAD_WORKLOADS[name]
+    B, G, V = w.B, w.gamma, w.V
+    inp = wl.make_lmhead_inputs(w, 2, DEV)
+    ws = lib.new_lmhead_workspace(B, G, V, DEV)
+    gam = torch.as_tensor(inp.gamma, device=DEV)
+    ua = torch.as_tensor(inp.uniforms.u_accept, device=DEV); ur = torch.as_tensor(inp.uniforms.u_resample, device=DEV)
+
+    def run():
+        lt = torch.empty(B, G + 1, V, dtype=torch.float32, device=DEV)
+        ld = torch.empty(B, G, V, dtype=torch.float32, device=DEV)
+        acc = torch.empty(B, dtype=torch.int32, device=DEV)
+        p = torch.empty(B, G, dtype=torch.float32, device=DEV); q = torch.empty(B, G, dtype=torch.float32, device=DEV)
+        ot = torch.empty(B, G + 1, dtype=torch.int32, device=DEV); ol = torch.empty(B, dtype=torch.int32, device=DEV)
+        lib.bs_lmhead_verify(inp.H_t, inp.W_t, inp.H_d, inp.W_d, inp.tokens, gam, ua, w.temperature, B, G,
+                             lt, ld, acc, p, q, ws)
+        lib.bs_residual_sample(lt, ld, inp.tokens, gam, acc, ur, w.temperature, ot, ol, ws)
+        return lt, ld, acc, p, q, ot, ol
+
+    ref = run()
+    ref_ws = ws.clone()
+    bad = torch.zeros((), dtype=torch.int64, device=DEV)
+    for i in range(reps):
+        o = run()
+        same = (ws == ref_ws).all()
+        for a, b in zip(o, ref):
+            same = same & (a == b).all()
+        bad += (~same).to(torch.int64)
+        del o
+    assert int(bad) == 0, f"{int(bad)} of {reps} repetitions differ from the first"
+    st = lib.bs_get_device_status(ws, B, G, V)
+    assert (st & ~lib.BS_DEV_RESIDUAL_FALLBACK == 0).all()
