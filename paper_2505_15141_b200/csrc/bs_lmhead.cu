@@ -20,8 +20,10 @@
 //   warps 2..9          epilogue: tcgen05.ld their 32 lanes of the accumulator, 32 columns at a
 //                       time (four lane quarters x two column halves); every thread owns one
 //                       output row, so the running (max, sum exp) or (max, arg-max) of that row
-//                       over its half tile needs no shuffle; the fp32 logits go to global memory,
-//                       the per-(row, half tile) statistics to a partial buffer.
+//                       over its half tile needs no shuffle; the fp32 logits leave through a 4 KB
+//                       staging block per warp and a TMA store of 32 rows x 32 columns (whole
+//                       128-byte lines; a thread storing its own row would touch 32 lines per
+//                       instruction), the per-(row, half tile) statistics go to a partial buffer.
 // A second small kernel merges the partials of every row, stores the row statistics in the
 // workspace (where bs_residual_sample reads them) and runs the accept scan.
 //
@@ -42,6 +44,8 @@ constexpr int kLmThreads = 64 + 32 * kLmEpiWarps;   // producer warp, MMA warp, 
 constexpr int kLmABytes = kLmBM * kLmBK * 2;                      // 16 KB of H per stage
 constexpr int kLmChunkBytes = kLmBK * 128;                        // 64 k-rows x 64 n (128 B) of W = 8 KB
 constexpr int kLmTmemCols = 512;           // two fp32 accumulators of up to 256 columns
+constexpr int kLmOutBoxBytes = 32 * 32 * 4;                       // staging block of one epilogue warp
+constexpr int kLmOutBytes = kLmEpiWarps * kLmOutBoxBytes;         // 32 KB behind the stages
 
 struct LmProduct {
     float* out;            // [M, V] fp32 logits
@@ -69,6 +73,21 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm,
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
         " [%0], [%1, {%2, %3}], [%4], %5;"
         ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar), "l"(policy) : "memory");
+}
+// shared -> global store of one box; completion is tracked by the issuing thread's bulk async-group
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(tm), "r"(x), "r"(y), "r"(src) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void tma_store_wait_read() {        // the stores issued so far have read their source
+    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+__device__ __forceinline__ void tma_store_wait_all() {         // ... and have been written
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 __device__ __forceinline__ uint64_t policy_evict_first() {
     uint64_t p;
@@ -151,6 +170,7 @@ template <int BN, int MH, int STAGES, bool GREEDY>
 __global__ void __launch_bounds__(kLmThreads, 1)
 lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tm_h0, const __grid_constant__ CUtensorMap tm_w0,
                    const __grid_constant__ CUtensorMap tm_h1, const __grid_constant__ CUtensorMap tm_w1,
+                   const __grid_constant__ CUtensorMap tm_o0, const __grid_constant__ CUtensorMap tm_o1,
                    const LmParams p) {
     constexpr int kChunks = BN / 64;
     constexpr int kBBytes = kChunks * kLmChunkBytes;
@@ -164,6 +184,7 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tm_h0, const __grid_const
     // the swizzle pattern is a function of the address bits: stage bases must be 1024-byte aligned
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(lm_smem_raw) + 1023) &
                                                            ~(uintptr_t)1023);
+    unsigned char* out_stage = smem + (size_t)STAGES * kStageBytes;   // 1024-byte aligned like the stages
     __shared__ __align__(8) unsigned long long s_full[STAGES];
     __shared__ __align__(8) unsigned long long s_empty[STAGES];
     __shared__ __align__(8) unsigned long long s_tmem_full[2];
@@ -313,7 +334,8 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tm_h0, const __grid_const
                 const bool row_ok = row < pr.M;
                 const int n0 = tl.nt * BN + chalf * kHalfCols;
                 const int ncols = max(0, min(kHalfCols, p.V - n0));
-                float* orow = pr.out + (size_t)(row_ok ? row : 0) * p.V + n0;
+                const int row0 = m0 + h * kLmBM + quarter * 32;
+                const uint32_t obuf = smem_u32(out_stage + (size_t)(warp - 2) * kLmOutBoxBytes);
                 Online on{-INFINITY, 0.f};
                 ArgMax am{-INFINITY, INT_MAX};
                 if (m0 + h * kLmBM + quarter * 32 < pr.M) {   // some row of this warp exists
@@ -348,11 +370,20 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tm_h0, const __grid_const
                                     on.s += a0 + a1;
                                 }
                             }
-#pragma unroll
-                            for (int i = 0; i < 32; i += 4)
-                                if (i < nv)
-                                    *reinterpret_cast<uint4*>(orow + c0 + i) = make_uint4(v[i], v[i + 1], v[i + 2], v[i + 3]);
                         }
+                        // The 32 x 32 block leaves through shared memory: row = lane, 16-byte chunk j of a
+                        // row sits at j ^ (row % 8) (the 128-byte swizzle the tensor map undoes), so the
+                        // eight lanes of a quarter warp hit eight different chunks.  Rows past M and
+                        // columns past V are clipped by the tensor map.
+                        if (lane == 0) tma_store_wait_read();     // the block before this one has been read
+                        __syncwarp();
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            sts128(obuf + (uint32_t)(lane * 128 + ((j ^ (lane & 7)) << 4)), v[4 * j], v[4 * j + 1],
+                                   v[4 * j + 2], v[4 * j + 3]);
+                        fence_writes_before_bulk_store();
+                        __syncwarp();
+                        if (lane == 0) tma_store_2d(tl.prod ? &tm_o1 : &tm_o0, obuf, n0 + c0, row0);
                     }
                 }
                 // accumulator drained: hand it back before the bookkeeping
@@ -367,6 +398,7 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tm_h0, const __grid_const
                 }
             }
         }
+        if (lane == 0) tma_store_wait_all();                  // shared memory is given up only after the last store
         if (!ok && lane == 0) { s_abort = 1; atomicExch(p.abort_flag, 1); }
     }
 
@@ -477,9 +509,22 @@ static bool make_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t 
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// fp32 matrix [rows, cols] with cols contiguous, written in boxes of 32 x 32 with the 128-byte swizzle
+static bool make_out_map(CUtensorMap* tm, void* base, uint64_t rows, uint64_t cols) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 4};
+    const cuuint32_t box[2] = {32, 32};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
+           CUDA_SUCCESS;
+}
+
 constexpr int kLmBN = 256;
 constexpr size_t lm_smem_bytes(int mh, int stages) {
-    return (size_t)stages * (mh * kLmABytes + (kLmBN / 64) * kLmChunkBytes) + 1024;
+    return (size_t)stages * (mh * kLmABytes + (kLmBN / 64) * kLmChunkBytes) + kLmOutBytes + 1024;
 }
 
 static size_t lm_partial_bytes(int B, int Gmax, int V) {
@@ -505,7 +550,7 @@ static bs_status launch_lmhead(const CUtensorMap* tms, const LmParams& lp, const
     const int tiles = lp.prod[0].MT * lp.NT + (lp.nprod > 1 ? lp.prod[1].MT * lp.NT : 0);
     int grid = sm_count();
     if (grid > tiles) grid = tiles;
-    cudaError_t e = launch_pdl(kern, grid, kLmThreads, smem, st, tms[0], tms[1], tms[2], tms[3], lp);
+    cudaError_t e = launch_pdl(kern, grid, kLmThreads, smem, st, tms[0], tms[1], tms[2], tms[3], tms[4], tms[5], lp);
     if (e != cudaSuccess) return cuda_status(e);
     return cuda_status(launch_pdl(lmhead_finalize_kernel<GREEDY>, vp.B * vp.R, kThreads, 0, st, vp, partial, 2 * lp.NT));
 }
@@ -560,7 +605,7 @@ extern "C" bs_status bs_lmhead_verify(const void* H_t, const void* W_t, int d_t,
     lp.prod[1] = LmProduct{logits_d_out, need_draft ? Md : 0, need_draft ? div_up(d_d, kLmBK) : 0,
                            need_draft ? div_up(Md, kLmBM * mh) : 0, Gmax > 0 ? Gmax : 1, Gmax + 1};
 
-    CUtensorMap tms[4];
+    CUtensorMap tms[6];
     if (!make_map(&tms[0], H_t, (uint64_t)Mt, (uint64_t)d_t, kLmBM) || !make_map(&tms[1], W_t, (uint64_t)d_t, (uint64_t)V, kLmBK))
         return BS_ERR_CUDA;
     if (need_draft) {
@@ -569,6 +614,12 @@ extern "C" bs_status bs_lmhead_verify(const void* H_t, const void* W_t, int d_t,
     } else {
         tms[2] = tms[0];
         tms[3] = tms[1];
+    }
+    if (!make_out_map(&tms[4], logits_t_out, (uint64_t)Mt, (uint64_t)V)) return BS_ERR_CUDA;
+    if (need_draft) {
+        if (!make_out_map(&tms[5], logits_d_out, (uint64_t)Md, (uint64_t)V)) return BS_ERR_CUDA;
+    } else {
+        tms[5] = tms[4];
     }
 
     VerifyParams vp;

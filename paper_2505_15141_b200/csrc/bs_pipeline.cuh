@@ -53,6 +53,10 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 __device__ __forceinline__ void fence_reads_before_refill() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
+// The other direction: ordinary shared stores that a bulk copy shared -> global is about to read.
+__device__ __forceinline__ void fence_writes_before_bulk_store() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
