@@ -21,7 +21,8 @@ static_assert(kRsVecPerLane * 32 * 16 * kRsWarps == kResSegBytes, "pieces must t
 
 struct RsMeta {
     int b, sg;
-    int nvec;        // valid 16-byte vectors of this segment (per row)
+    int nvec;        // valid 16-byte vectors in the first half of the slot
+    int nvec2;       // ... in the second half: the draft row's segment, or segment sg + 1 of a row sampled alone
     int flags;       // bit 0: bonus (target row only), bit 1: last item of this sequence in the CTA's range
     float kt, kd;    // p_v = 2^(x_t c + kt), q_v = 2^(x_d c + kd)
 };
@@ -45,12 +46,18 @@ __device__ __forceinline__ RsSeq rs_seq(const ResidParams& p, int b) {
     s.wgt = s.bonus ? 1 : 2;
     return s;
 }
-// Items [i0, i1) of sequence b whose first weight unit lies in [lo, hi); pre = first unit of b.
-__device__ __forceinline__ void rs_items(int pre, int wgt, int nseg, int lo, int hi, int& i0, int& i1) {
-    if (wgt <= 0) { i0 = i1 = 0; return; }
-    const int a = max(lo, pre) - pre, e = min(hi, pre + wgt * nseg) - pre;
-    i0 = (a + wgt - 1) / wgt;
-    i1 = e > 0 ? (e + wgt - 1) / wgt : 0;
+// Items of a sequence in the pipelined kernel.  A slot has two 16 KB halves: for a row pair they hold
+// the same segment of the target and of the draft row, for a row sampled alone two consecutive
+// segments of it, so that every item keeps up to 32 KB in flight (with one segment per item the
+// CTAs whose sequences were all accepted moved half the bytes per item and finished last).
+__device__ __forceinline__ int rs_nitems(const RsSeq& s, int nseg) {
+    return s.wgt <= 0 ? 0 : (s.bonus ? (nseg + 1) >> 1 : nseg);
+}
+__device__ __forceinline__ int rs_first_seg(const RsSeq& s, int item) { return s.bonus ? 2 * item : item; }
+// Items [i0, i1) of a sequence with `nitems` items that lie in the CTA's range [lo, hi); pre = index of its first item.
+__device__ __forceinline__ void rs_items(int pre, int nitems, int lo, int hi, int& i0, int& i1) {
+    i0 = max(lo, pre) - pre;
+    i1 = min(hi, pre + nitems) - pre;
     if (i1 < i0) i1 = i0;
 }
 

@@ -2,9 +2,9 @@
 // the else-branch of Algorithm 6 (one token from Norm([P - Q]_+) at the first rejected position)
 // and the line after its loop (the bonus token from P), by inverse CDF in vocabulary order.
 //
-// A work item is one 16 KB segment of the row pair (target row tau_b, draft row tau_b) of one
-// sequence; a fully accepted sequence has only the target row, so its items weigh half.  The
-// weighted item list is cut into gridDim.x contiguous ranges, one per CTA.
+// A work item fills one 32 KB slot: one 16 KB segment of the row pair (target row tau_b, draft row
+// tau_b) of a sequence, or two consecutive segments of the target row of a fully accepted
+// sequence.  The item list is cut into gridDim.x contiguous ranges, one per CTA.
 //
 //   warp 16 (one lane)  producer: for each item of its range, one or two bulk async copies
 //                       (TMA, no multicast) global -> shared into a ring of 2 x 16 KB slots,
@@ -56,14 +56,14 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
 
     pdl_enter();                                              // accept_len and the row statistics come from the kernel before
 
-    // ---- prefix sum of item weights over the batch (all threads, redundantly per CTA) ----
+    // ---- prefix sum of item counts over the batch (all threads, redundantly per CTA) ----
     {
         const int per = div_up(p.B, kRsThreads);
         const int b0 = tid * per;
         int local = 0;
         for (int k = 0; k < per; ++k) {
             const int b = b0 + k;
-            if (b < p.B) local += rs_seq(p, b).wgt * p.nseg;
+            if (b < p.B) local += rs_nitems(rs_seq(p, b), p.nseg);
         }
         int incl = local;
 #pragma unroll
@@ -80,7 +80,7 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
             const int b = b0 + k;
             if (b < p.B) {
                 s_prefix[b] = run;
-                run += rs_seq(p, b).wgt * p.nseg;
+                run += rs_nitems(rs_seq(p, b), p.nseg);
             }
         }
         if (tid == kRsThreads - 1) s_prefix[p.B] = run;
@@ -110,7 +110,7 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
         int mine = 0;
         for (int b = bfirst + tid; b <= blast; b += kRsThreads) {
             int i0, i1;
-            rs_items(s_prefix[b], (s_prefix[b + 1] - s_prefix[b]) / p.nseg, p.nseg, lo, hi, i0, i1);
+            rs_items(s_prefix[b], s_prefix[b + 1] - s_prefix[b], lo, hi, i0, i1);
             mine += i1 - i0;
         }
         if (mine) atomicAdd(&s_count, mine);
@@ -127,7 +127,7 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
         for (int b = bfirst; b <= blast; ++b) {
             const RsSeq sq = rs_seq(p, b);
             int i0, i1;
-            rs_items(s_prefix[b], sq.wgt, p.nseg, lo, hi, i0, i1);
+            rs_items(s_prefix[b], rs_nitems(sq, p.nseg), lo, hi, i0, i1);
             if (i1 <= i0) continue;
             const float2 ts = p.row_stats[(size_t)b * p.R + rs_tslot(p, sq)];
             float kt = -(ts.x * p.c + log2f(ts.y)), kd = 0.f;
@@ -138,21 +138,25 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
                 kd = -(ds.x * p.c + log2f(ds.y));
                 dp = row_ptr(static_cast<const T*>(p.draft), b, p.Gmax, sq.tau, p.V);
             }
-            for (int sg = i0; sg < i1; ++sg) {
+            for (int it = i0; it < i1; ++it) {
                 if (!mbar_wait(smem_u32(&s_empty[slot]), ph ^ 1u)) { atomicExch(p.abort_flag, 1); return; }
+                const int sg = rs_first_seg(sq, it);
                 const int e0 = sg * p.seg;
                 const int n = min(p.seg, p.V - e0);
+                // second half of the slot: the draft row's segment, or the next segment of a row sampled alone
+                const int n2 = !sq.bonus ? n : (sg + 1 < p.nseg ? min(p.seg, p.V - e0 - p.seg) : 0);
                 const uint32_t bytes = (uint32_t)n * (uint32_t)sizeof(T);
+                const uint32_t bytes2 = (uint32_t)n2 * (uint32_t)sizeof(T);
                 RsMeta m;
-                m.b = b; m.sg = sg; m.nvec = n / kVec;
-                m.flags = (sq.bonus ? 1 : 0) | (sg == i1 - 1 ? 2 : 0);
+                m.b = b; m.sg = sg; m.nvec = n / kVec; m.nvec2 = n2 / kVec;
+                m.flags = (sq.bonus ? 1 : 0) | (it == i1 - 1 ? 2 : 0);
                 m.kt = kt; m.kd = kd;
                 s_meta[slot] = m;
                 const uint32_t bar = smem_u32(&s_full[slot]);
                 const uint32_t dst = smem_u32(ring + (size_t)slot * kRsStageBytes);
-                mbar_arrive_expect_tx(bar, sq.bonus ? bytes : 2u * bytes);   // releases the record to the waiters
+                mbar_arrive_expect_tx(bar, bytes + bytes2);    // releases the record to the waiters
                 bulk_load(dst, tp + e0, bytes, bar);
-                if (!sq.bonus) bulk_load(dst + kResSegBytes, dp + e0, bytes, bar);
+                if (n2) bulk_load(dst + kResSegBytes, (sq.bonus ? tp + p.seg : dp) + e0, bytes2, bar);
                 if (++slot == nstages) { slot = 0; ph ^= 1u; }
             }
         }
@@ -165,7 +169,7 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
         for (int b = bfirst; b <= blast; ++b) {
             const RsSeq sq = rs_seq(p, b);
             int i0, i1;
-            rs_items(s_prefix[b], sq.wgt, p.nseg, lo, hi, i0, i1);
+            rs_items(s_prefix[b], rs_nitems(sq, p.nseg), lo, hi, i0, i1);
             if (i1 <= i0) continue;
             ++shares;
             // wait until all consumer warps have written their masses of this share
@@ -183,10 +187,12 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
                 }
             }
             __threadfence();
+            // the ticket counts segments: an item of a row sampled alone covers two (the last one maybe one)
+            const unsigned segs = sq.bonus ? (unsigned)(min(2 * i1, p.nseg) - 2 * i0) : (unsigned)(i1 - i0);
             unsigned old = 0;
-            if (lane == 0) old = atomicAdd(p.ticket + b, (unsigned)(i1 - i0));
+            if (lane == 0) old = atomicAdd(p.ticket + b, segs);
             old = __shfl_sync(0xffffffffu, old, 0);
-            if (old + (unsigned)(i1 - i0) == (unsigned)p.nseg) {
+            if (old + segs == (unsigned)p.nseg) {
                 __threadfence();
                 MassFn f;
                 f.c = p.c;
@@ -214,33 +220,44 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
         f.c = p.c; f.kt = m.kt; f.kd = m.kd; f.bonus = (m.flags & 1) != 0;
         const uint32_t base = smem_u32(ring + (size_t)slot * kRsStageBytes) + (uint32_t)(warp * kRsPieceBytes + lane * 16);
         uint4 a[kRsVecPerLane], d[kRsVecPerLane];
-        bool valid[kRsVecPerLane];
+        bool valid[kRsVecPerLane], valid2[kRsVecPerLane];
 #pragma unroll
         for (int q = 0; q < kRsVecPerLane; ++q) {
-            valid[q] = warp * kRsPieceVecs + q * 32 + lane < m.nvec;
-            if (valid[q]) {
-                a[q] = lds128(base + (uint32_t)(q * 512));
-                d[q] = f.bonus ? a[q] : lds128(base + (uint32_t)(kResSegBytes + q * 512));
-            }
+            const int vi = warp * kRsPieceVecs + q * 32 + lane;
+            valid[q] = vi < m.nvec;
+            valid2[q] = vi < m.nvec2;
+            if (valid[q]) a[q] = lds128(base + (uint32_t)(q * 512));
+            if (valid2[q]) d[q] = lds128(base + (uint32_t)(kResSegBytes + q * 512));
         }
         fence_reads_before_refill();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&s_empty[slot]));  // the slot's data is in registers now
-        float acc = 0.f;
+        // row pair: one mass per piece from both halves; row alone: one mass per half
+        float acc = 0.f, acc2 = 0.f;
 #pragma unroll
         for (int q = 0; q < kRsVecPerLane; ++q) {
+            float r[kVec];
             if (valid[q]) {
-                float r[kVec];
-                RsElems<T>::masses(a[q], d[q], f, r);
+                RsElems<T>::masses(a[q], f.bonus ? a[q] : d[q], f, r);
                 float vs = 0.f;
 #pragma unroll
                 for (int i = 0; i < kVec; ++i) vs += r[i];
                 acc += vs;
             }
+            if (f.bonus && valid2[q]) {
+                RsElems<T>::masses(d[q], d[q], f, r);
+                float vs = 0.f;
+#pragma unroll
+                for (int i = 0; i < kVec; ++i) vs += r[i];
+                acc2 += vs;
+            }
         }
         acc = warp_sum(acc);
+        if (f.bonus) acc2 = warp_sum(acc2);
         if (lane == 0) {
-            p.resid_partial[(size_t)m.b * p.S + m.sg * kRsWarps + warp] = acc;
+            float* out = p.resid_partial + (size_t)m.b * p.S + m.sg * kRsWarps + warp;
+            out[0] = acc;
+            if (f.bonus && m.nvec2 > 0) out[kRsWarps] = acc2;
             if (m.flags & 2) {                                // this CTA's share of the sequence ends here
                 __threadfence();
                 atomicAdd(&s_done, 1u);
