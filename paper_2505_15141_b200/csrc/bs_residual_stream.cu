@@ -38,7 +38,6 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
     __shared__ __align__(8) unsigned long long s_empty[kRsMaxStages];
     __shared__ RsMeta s_meta[kRsMaxStages];
     __shared__ int s_scan[kRsThreads / 32];
-    __shared__ int s_count;                                   // items of this CTA
     __shared__ unsigned int s_done;                           // consumer warps that finished a sequence share
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -49,7 +48,6 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
             mbar_init(smem_u32(&s_full[s]), 1);
             mbar_init(smem_u32(&s_empty[s]), kRsWarps);
         }
-        s_count = 0;
         s_done = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -105,19 +103,8 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
         }
         blast = l;
     }
-    // number of items of this CTA (every thread needs it to know when to stop)
-    {
-        int mine = 0;
-        for (int b = bfirst + tid; b <= blast; b += kRsThreads) {
-            int i0, i1;
-            rs_items(s_prefix[b], s_prefix[b + 1] - s_prefix[b], lo, hi, i0, i1);
-            mine += i1 - i0;
-        }
-        if (mine) atomicAdd(&s_count, mine);
-        __syncthreads();
-    }
-    const int count = s_count;
-    if (count <= 0 || hi <= lo) return;
+    const int count = hi - lo;                                // items of this CTA: the list has unit weights
+    if (count <= 0) return;
 
     if (warp == kRsWarps) {
         // =============================== producer ===============================
