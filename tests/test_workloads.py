@@ -1,5 +1,6 @@
 """Input generators: Philox known answers, uniform mapping, shapes and determinism."""
 import numpy as np
+import pytest
 import torch
 
 from conftest import golden_lines
@@ -76,3 +77,20 @@ def test_sigma_schedules():
     s = wl.round_sigma(w3, 1, None)
     assert s.shape == (64,) and s.min() >= 0.3 and s.max() <= 2.0
     assert (s == wl.round_sigma(w3, 99, None)).all()
+
+
+def test_throughput_workloads_reward_range_and_step_duration():
+    for name in ("llama3_tput", "tiny_tput"):
+        w = wl.WORKLOADS[name]
+        assert w.alg == "ucb_reward" and w.arm_gamma[0] == 0                 # canonical decoding is an arm
+        # the stand-in for the measured step duration grows with the longest speculation length in the batch
+        d = [wl.step_seconds(w, np.full(w.B, g)) for g in range(w.Gmax + 1)]
+        assert d[0] == w.step_target_s and all(a < b for a, b in zip(d, d[1:]))
+        mixed = np.zeros(w.B, dtype=np.int64); mixed[-1] = w.Gmax
+        assert wl.step_seconds(w, mixed) == d[-1]
+        # no round can earn more than the declared width: every sequence emits Gmax + 1 tokens in the shortest step
+        best = (w.Gmax + 1) / d[0] * (w.B if w.whole_batch else 1)
+        assert w.reward_width == pytest.approx(best) and w.reward_width > 0
+        # gamma = 0 rounds have one target row per sequence and emit exactly one token
+        rnd = wl.make_round(w, 1, np.zeros(w.B, dtype=np.int32), B=min(w.B, 3))
+        assert (rnd.gamma == 0).all() and rnd.target.shape[1] == w.Gmax + 1
