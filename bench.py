@@ -75,6 +75,9 @@ def parse_args():
                          "rejection + resampling in one launch) -> update")
     ap.add_argument("--no-others", action="store_true",
                     help="skip the short runs of the other workloads that the default invocation adds to its line")
+    ap.add_argument("--bandit-step", action="store_true",
+                    help="one bs_bandit_step per round (update + next round's select) instead of bs_bandit_select "
+                         "and bs_bandit_update; measured: no faster, the two small launches already overlap")
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="budget of the CPU-oracle sample")
@@ -281,6 +284,16 @@ def run_cuda(args, w):
         else:
             bs.bs_bandit_update(state, alg, B, K, arm_d, out_len)
 
+    fused_bandit = args.bandit_step
+
+    def step_bandit_call(s_next):
+        """History step of this round and select step of the next (whose uniforms are s_next's) in one launch."""
+        if reward:
+            bs.bs_throughput_reward(out_len, None, B, step_s, w.whole_batch, reward_d)
+            bs.bs_bandit_step(state, alg, B, K, reward_d, None, None, arm_d, gamma_d)
+        else:
+            bs.bs_bandit_step(state, alg, B, K, out_len, s_next["u_arm"], None, arm_d, gamma_d)
+
     def init_call():
         if reward:
             bs.bs_bandit_init_reward(state, B, K, w.arm_gamma, w.delta, w.reward_width)
@@ -317,42 +330,52 @@ def run_cuda(args, w):
         fn(s["target"], s["draft"], tok_d if drafted else s["tokens"], gamma_d, s["u_accept"], s["u_resample"],
            w.temperature, accept_len, p_tok, q_tok, out_tokens, out_len, ws)
 
-    def step_calls(s):
-        bs.bs_bandit_select(state, alg, B, K, s["u_arm"], None, arm_d, gamma_d)
+    def step_calls(s, s_next):
+        # the arms of this round: chosen here, or by the step call that ended the round before
+        if not fused_bandit:
+            bs.bs_bandit_select(state, alg, B, K, s["u_arm"], None, arm_d, gamma_d)
         if walk:
             if drafted:
                 draft_calls(s)
             walk_call(s)
+        else:
+            if drafted:
+                draft_calls(s)
+                s = dict(s, tokens=tok_d)
+            verify_call(s)
+            bs.bs_residual_sample(s["target"], s["draft"], s["tokens"], gamma_d, accept_len, s["u_resample"],
+                                  w.temperature, out_tokens, out_len, ws)
+        if fused_bandit:
+            step_bandit_call(s_next)
+        else:
             update_call()
-            return
-        if drafted:
-            draft_calls(s)
-            s = dict(s, tokens=tok_d)
-        verify_call(s)
-        bs.bs_residual_sample(s["target"], s["draft"], s["tokens"], gamma_d, accept_len, s["u_resample"],
-                              w.temperature, out_tokens, out_len, ws)
-        update_call()
+
+    def first_select():
+        if fused_bandit:
+            bs.bs_bandit_select(state, alg, B, K, sets[0]["u_arm"], None, arm_d, gamma_d)
 
     side = torch.cuda.Stream(device=dev)
     graphs = []
     if not args.no_graph:
         with torch.cuda.stream(side):
-            step_calls(sets[0])                                # first launch outside capture
+            first_select()
+            step_calls(sets[0], sets[1 % ring])                # first launch outside capture
             side.synchronize()
-            for s in sets:
+            for i, s in enumerate(sets):
                 g = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(g, stream=side):
-                    step_calls(s)
+                    step_calls(s, sets[(i + 1) % ring])
                 graphs.append(g)
         torch.cuda.synchronize()
         # start from a clean bandit: the capture warm-up above played one round
         init_call()
+    first_select()
 
     def run_step(i):
         if graphs:
             graphs[i % ring].replay()
         else:
-            step_calls(sets[i % ring])
+            step_calls(sets[i % ring], sets[(i + 1) % ring])
 
     def pulls():
         return bs.bs_bandit_read(state, alg, B, K)["n"].copy()
@@ -529,6 +552,8 @@ def run_cuda(args, w):
                                 "select, verify with early exit + resample in one launch, update" if walk else
                                 "select, draft x Gmax, verify on drafted statistics, resample, update"
                                 if drafted else "select, verify, resample, update"),
+                       "bandit_calls": ("bs_bandit_step: the update and the next round's select in one launch"
+                                        if fused_bandit else "bs_bandit_select and bs_bandit_update, two launches"),
                        "multi_gpu": "one independent batch per rank, no collective on the data path"},
             "tokens_per_s": mean_y * B * value,
             "mean_accepted_len": mean_y,
@@ -540,7 +565,8 @@ def run_cuda(args, w):
                          "ms_per_launch": verify_ms, "residual_ms_per_launch": resid_ms},
             "e2e": e2e, "cpu_baseline": cpu, "clocks": clocks, "variants": variants,
             "other_workloads": getattr(args, "others", None),
-            "gpu_launches": ((3 if walk else 4) + (2 * G if drafted else 0) + (1 if reward else 0)) * args.steps,
+            "gpu_launches": ((3 if walk else 4) - (1 if fused_bandit else 0) + (2 * G if drafted else 0)
+                             + (1 if reward else 0)) * args.steps,
         }
         if walk:
             line["roofline"]["kernel"] = "verify_walk_kernel (bs_verify_walk)"

@@ -310,6 +310,21 @@ bs_status bs_bandit_update(void* state, size_t state_bytes, bs_alg alg, int B, i
                            const int32_t* arm, const int32_t* reward_y, const uint8_t* active,
                            void* stream);
 
+/* bs_bandit_update of this round and bs_bandit_select of the next in one launch (Algorithm 3: the
+ * history line of round t, then the select line of round t + 1), with the same results as the
+ * two calls.
+ *  reward_y [B] int32 (UCBSpec, EXP3Spec) or reward_r [B] fp64 (BS_UCB_REWARD): the other may be NULL
+ *  u_arm_next [B] fp32: the uniforms of the next round's draw (EXP3Spec; else may be NULL)
+ *  active: one mask for both steps (NULL = all active)
+ *  arm [B] int32 in/out: the arms played this round on entry, the next round's arms on return
+ *  gamma [B] int32 out: the next round's speculation lengths.  It must not be the array a kernel
+ *  still in flight on another stream reads; on one stream the call is ordered like any other.
+ *  index_out as in bs_bandit_select. */
+bs_status bs_bandit_step(void* state, size_t state_bytes, bs_alg alg, int B, int K,
+                         const int32_t* reward_y, const double* reward_r, const float* u_arm_next,
+                         const uint8_t* active, int32_t* arm, int32_t* gamma, double* index_out,
+                         void* stream);
+
 /* Reads the sufficient statistics back to host arrays (any may be NULL).  Synchronises.
  *  UCBSpec: n_host [B,K] int64, sumY_host [B,K] int64, t_host [B] int64; S_host unused.
  *  EXP3Spec: S_host [B,K] fp64, n_host [B,K] int64 (pulls per arm, not used by the algorithm),

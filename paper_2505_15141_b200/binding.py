@@ -54,6 +54,7 @@ SIGNATURES = {
     "bs_bandit_select": (_i, [_vp, _sz, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
     "bs_bandit_update": (_i, [_vp, _sz, _i, _i, _i, _vp, _vp, _vp, _vp]),
     "bs_bandit_read": (_i, [_vp, _sz, _i, _i, _i, _vp, _vp, _vp, _vp, _vp]),
+    "bs_bandit_step": (_i, [_vp, _sz, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "bs_bandit_init_reward": (_i, [_vp, _sz, _i, _i, _vp, _d, _d, _vp]),
     "bs_bandit_update_reward": (_i, [_vp, _sz, _i, _i, _vp, _vp, _vp, _vp]),
     "bs_throughput_reward": (_i, [_vp, _vp, _i, _d, _i, _vp, _vp]),
@@ -308,6 +309,17 @@ def bs_bandit_select(state, alg: int, B: int, K: int, u_arm, active, arm, gamma,
 def bs_bandit_update(state, alg: int, B: int, K: int, arm, reward_y, active=None, stream=None) -> None:
     _check(_lib.bs_bandit_update(_ptr(state), state.numel(), alg, B, K, _ptr(arm), _ptr(reward_y),
                                  _ptr(active), _stream(stream)), "bs_bandit_update")
+
+
+def bs_bandit_step(state, alg: int, B: int, K: int, reward, u_arm_next, active, arm, gamma, index_out=None,
+                   stream=None) -> None:
+    """Update with this round's reward (int32 accepted lengths, or fp64 rewards for BS_UCB_REWARD) and
+    select the next round's arms, in one launch; `arm` is read and overwritten."""
+    ry, rr = (None, reward) if alg == BS_UCB_REWARD else (reward, None)
+    assert (rr.dtype == torch.float64) if rr is not None else (ry.dtype == torch.int32)
+    _check(_lib.bs_bandit_step(_ptr(state), state.numel(), alg, B, K, _ptr(ry), _ptr(rr), _ptr(u_arm_next),
+                               _ptr(active), _ptr(arm), _ptr(gamma), _ptr(index_out), _stream(stream)),
+           "bs_bandit_step")
 
 
 def bs_bandit_read(state, alg: int, B: int, K: int, stream=None) -> dict:

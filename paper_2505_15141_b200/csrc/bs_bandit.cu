@@ -63,15 +63,11 @@ __device__ inline double confidence_radius(double half_width, int K, long long t
     return __dmul_rn(half_width, sqrt(__dmul_rn(frac, inner)));
 }
 
-// One warp per sequence, lane i = arm i.
-__global__ void __launch_bounds__(128) bandit_select_kernel(void* state, int alg, int B, int K,
-                                                           const float* u_arm, const uint8_t* active,
-                                                           int32_t* arm_out, int32_t* gamma_out, double* index_out) {
-    pdl_enter();
-    const int b = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+// The select step for sequence b by one warp, lane i = arm i.
+__device__ __forceinline__ void bandit_select_warp(const BanditState& s, int alg, int b, int K, const float* u_arm,
+                                                   const uint8_t* active, int32_t* arm_out, int32_t* gamma_out,
+                                                   double* index_out) {
     const int lane = threadIdx.x & 31;
-    if (b >= B) return;
-    const BanditState s = bandit_view(state, B, K);
     if (active && !active[b]) {
         if (lane == 0) { arm_out[b] = -1; gamma_out[b] = 0; }
         if (index_out && lane < K) index_out[(size_t)b * K + lane] = nan("");
@@ -132,44 +128,65 @@ __global__ void __launch_bounds__(128) bandit_select_kernel(void* state, int alg
     if (index_out && lane < K) index_out[(size_t)b * K + lane] = shown;
 }
 
-__global__ void bandit_update_kernel(void* state, int alg, int B, int K, const int32_t* arm,
-                                     const int32_t* reward_y, const uint8_t* active) {
+// One warp per sequence.
+__global__ void __launch_bounds__(128) bandit_select_kernel(void* state, int alg, int B, int K,
+                                                           const float* u_arm, const uint8_t* active,
+                                                           int32_t* arm_out, int32_t* gamma_out, double* index_out) {
     pdl_enter();
-    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    const int b = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (b >= B) return;
+    bandit_select_warp(bandit_view(state, B, K), alg, b, K, u_arm, active, arm_out, gamma_out, index_out);
+}
+
+// The history step for sequence b by one thread: accepted length y (UCBSpec, EXP3Spec) or real reward r.
+__device__ __forceinline__ void bandit_update_one(const BanditState& s, int alg, int b, int K, const int32_t* arm,
+                                                  const int32_t* reward_y, const double* reward_r,
+                                                  const uint8_t* active) {
     if (active && !active[b]) return;
-    const BanditState s = bandit_view(state, B, K);
     const int a = arm[b];
     if (a < 0 || a >= K) return;
-    const int L = s.hdr->L;
-    const int y = max(1, min(reward_y[b], L + 1));          // accepted length, bonus included
-    if (alg == BS_UCB) {
+    if (alg == BS_UCB_REWARD) {
+        double r = reward_r[b];
+        r = isnan(r) ? 0.0 : fmin(fmax(r, 0.0), s.hdr->width);
         s.A_i[(size_t)b * K + a] += 1;
-        s.Bm[(size_t)b * K + a] += y;
+        s.Bm_d[(size_t)b * K + a] = __dadd_rn(s.Bm_d[(size_t)b * K + a], r);
     } else {
-        // loss estimate (L + 1 - y) / (L p_{t, I_t}); the other arms' estimates are zero
-        const double z = __ddiv_rn((double)(L + 1 - y), __dmul_rn((double)L, s.ps[b]));
-        s.A_d[(size_t)b * K + a] = __dadd_rn(s.A_d[(size_t)b * K + a], z);
-        s.Bm[(size_t)b * K + a] += 1;
+        const int L = s.hdr->L;
+        const int y = max(1, min(reward_y[b], L + 1));      // accepted length, bonus included
+        if (alg == BS_UCB) {
+            s.A_i[(size_t)b * K + a] += 1;
+            s.Bm[(size_t)b * K + a] += y;
+        } else {
+            // loss estimate (L + 1 - y) / (L p_{t, I_t}); the other arms' estimates are zero
+            const double z = __ddiv_rn((double)(L + 1 - y), __dmul_rn((double)L, s.ps[b]));
+            s.A_d[(size_t)b * K + a] = __dadd_rn(s.A_d[(size_t)b * K + a], z);
+            s.Bm[(size_t)b * K + a] += 1;
+        }
     }
     s.t[b] += 1;
 }
 
-// Real-reward UCBSpec: n += 1, sumR += clamp(r, 0, W), t += 1.
-__global__ void bandit_update_reward_kernel(void* state, int B, int K, const int32_t* arm, const double* reward,
-                                            const uint8_t* active) {
+__global__ void bandit_update_kernel(void* state, int alg, int B, int K, const int32_t* arm,
+                                     const int32_t* reward_y, const double* reward_r, const uint8_t* active) {
     pdl_enter();
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= B) return;
-    if (active && !active[b]) return;
+    bandit_update_one(bandit_view(state, B, K), alg, b, K, arm, reward_y, reward_r, active);
+}
+
+// History step of this round and select step of the next in one launch: one warp per sequence, lane 0
+// records the outcome, then the warp chooses the next arm from the updated statistics.
+__global__ void __launch_bounds__(128) bandit_step_kernel(void* state, int alg, int B, int K, const int32_t* reward_y,
+                                                         const double* reward_r, const float* u_arm_next,
+                                                         const uint8_t* active, int32_t* arm, int32_t* gamma,
+                                                         double* index_out) {
+    pdl_enter();
+    const int b = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (b >= B) return;
     const BanditState s = bandit_view(state, B, K);
-    const int a = arm[b];
-    if (a < 0 || a >= K) return;
-    double r = reward[b];
-    r = isnan(r) ? 0.0 : fmin(fmax(r, 0.0), s.hdr->width);
-    s.A_i[(size_t)b * K + a] += 1;
-    s.Bm_d[(size_t)b * K + a] = __dadd_rn(s.Bm_d[(size_t)b * K + a], r);
-    s.t[b] += 1;
+    if ((threadIdx.x & 31) == 0) bandit_update_one(s, alg, b, K, arm, reward_y, reward_r, active);
+    __syncwarp();                                             // the lanes read what lane 0 wrote
+    bandit_select_warp(s, alg, b, K, u_arm_next, active, arm, gamma, index_out);
 }
 
 // Tokens per second of the round: per sequence, or the batch total for every active sequence.
@@ -262,15 +279,29 @@ extern "C" bs_status bs_bandit_update(void* state, size_t state_bytes, bs_alg al
     if (!bandit_args_ok(state, state_bytes, alg, B, K) || !arm || !reward_y) return BS_ERR_INVALID_ARG;
     if (alg == BS_UCB_REWARD) return BS_ERR_INVALID_ARG;    // real rewards: bs_bandit_update_reward
     return cuda_status(launch_pdl(bandit_update_kernel, div_up(B, 128), 128, 0, static_cast<cudaStream_t>(stream),
-                                  state, (int)alg, B, K, arm, reward_y, active));
+                                  state, (int)alg, B, K, arm, reward_y, static_cast<const double*>(nullptr), active));
 }
 
 extern "C" bs_status bs_bandit_update_reward(void* state, size_t state_bytes, int B, int K,
                                              const int32_t* arm, const double* reward, const uint8_t* active,
                                              void* stream) {
     if (!bandit_args_ok(state, state_bytes, BS_UCB_REWARD, B, K) || !arm || !reward) return BS_ERR_INVALID_ARG;
-    return cuda_status(launch_pdl(bandit_update_reward_kernel, div_up(B, 128), 128, 0,
-                                  static_cast<cudaStream_t>(stream), state, B, K, arm, reward, active));
+    return cuda_status(launch_pdl(bandit_update_kernel, div_up(B, 128), 128, 0, static_cast<cudaStream_t>(stream),
+                                  state, (int)BS_UCB_REWARD, B, K, arm, static_cast<const int32_t*>(nullptr), reward,
+                                  active));
+}
+
+extern "C" bs_status bs_bandit_step(void* state, size_t state_bytes, bs_alg alg, int B, int K,
+                                    const int32_t* reward_y, const double* reward_r, const float* u_arm_next,
+                                    const uint8_t* active, int32_t* arm, int32_t* gamma, double* index_out,
+                                    void* stream) {
+    if (!bandit_args_ok(state, state_bytes, alg, B, K) || !arm || !gamma) return BS_ERR_INVALID_ARG;
+    if (alg == BS_UCB_REWARD ? !reward_r : !reward_y) return BS_ERR_INVALID_ARG;
+    if (alg == BS_EXP3 && !u_arm_next) return BS_ERR_INVALID_ARG;
+    const int warps_per_cta = 4;
+    return cuda_status(launch_pdl(bandit_step_kernel, div_up(B, warps_per_cta), warps_per_cta * 32, 0,
+                                  static_cast<cudaStream_t>(stream), state, (int)alg, B, K, reward_y, reward_r, u_arm_next,
+                                  active, arm, gamma, index_out));
 }
 
 extern "C" bs_status bs_throughput_reward(const int32_t* out_len, const uint8_t* active, int B, double seconds,

@@ -134,10 +134,12 @@ def gpu_round(bs, rnd: wl.RoundInputs, temperature: float, workspace=None):
 
 
 def closed_loop(bs, w: wl.Workload, rounds: int, device, sample: Optional[Sequence[int]] = None,
-                first_round: int = 1, state=None, oracle_bandit=None, carry: Optional[dict] = None) -> Tally:
+                first_round: int = 1, state=None, oracle_bandit=None, carry: Optional[dict] = None,
+                fused_step: bool = False) -> Tally:
     """select -> make inputs for the chosen arms -> verify -> resample -> update, on the GPU and in
     the oracle side by side.  `sample`: sequences whose verification the oracle replays (default
-    all); the oracle bandit of the others is fed the CUDA reward (teacher forcing)."""
+    all); the oracle bandit of the others is fed the CUDA reward (teacher forcing).  fused_step: the
+    update of a round and the select of the next go through bs_bandit_step (one launch)."""
     B, K, G, V = w.B, w.K, w.Gmax, w.V
     alg = {None: None, "ucb": bs.BS_UCB, "exp3": bs.BS_EXP3, "ucb_reward": bs.BS_UCB_REWARD}[w.alg]
     tally = Tally()
@@ -159,7 +161,8 @@ def closed_loop(bs, w: wl.Workload, rounds: int, device, sample: Optional[Sequen
         un = wl.round_uniforms(w.seed, rnd_i, B, G)
         if alg is not None:
             u_arm_d = torch.as_tensor(un.u_arm, device=device)
-            bs.bs_bandit_select(state, alg, B, K, u_arm_d, None, arm_d, gamma_d)
+            if not fused_step or rnd_i == first_round:       # later rounds: chosen by the step call of the round before
+                bs.bs_bandit_select(state, alg, B, K, u_arm_d, None, arm_d, gamma_d)
             arm_gpu = to_np(arm_d).astype(np.int64)
             if w.alg in ("ucb", "ucb_reward"):
                 arm_ref, _, flagged = oracle_bandit.select()
@@ -194,10 +197,17 @@ def closed_loop(bs, w: wl.Workload, rounds: int, device, sample: Optional[Sequen
             rew = ob.throughput_reward(y, seconds, w.whole_batch)
             assert np.array_equal(rew_d.cpu().numpy(), rew), f"round {rnd_i}: throughput reward differs"
             assert rew.max() <= w.reward_width
-            bs.bs_bandit_update_reward(state, B, K, arm_d, rew_d)
+            if fused_step and rnd_i + 1 < first_round + rounds:
+                bs.bs_bandit_step(state, alg, B, K, rew_d, None, None, arm_d, gamma_d)
+            else:
+                bs.bs_bandit_update_reward(state, B, K, arm_d, rew_d)
             oracle_bandit.update(arm, rew)
         elif alg is not None:
-            bs.bs_bandit_update(state, alg, B, K, arm_d, out.out_len)
+            if fused_step and rnd_i + 1 < first_round + rounds:
+                u_next = torch.as_tensor(wl.round_uniforms(w.seed, rnd_i + 1, B, G).u_arm, device=device)
+                bs.bs_bandit_step(state, alg, B, K, out.out_len, u_next, None, arm_d, gamma_d)
+            else:
+                bs.bs_bandit_update(state, alg, B, K, arm_d, out.out_len)
             oracle_bandit.update(arm, y)
     if alg is not None:
         st = bs.bs_bandit_read(state, alg, B, K)

@@ -95,3 +95,37 @@ def test_reward_calls_reject_what_they_cannot_use(lib):
             lib.bs_throughput_reward(y, None, B, seconds, True, r)
     lib.bs_bandit_init_reward(state, B, K, [0, 0, 0], 0.5, 3.0)                     # canonical decoding only: allowed
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("name,rounds", [("tiny_ucb", 64), ("tiny_tput", 120), ("llama3_ucb", 30), ("qwen_exp3", 30)])
+def test_closed_loop_with_the_fused_bandit_step(lib, name, rounds):
+    """bs_bandit_step (update of round t + select of round t + 1 in one launch) against the oracle's two
+    steps: same arms, same statistics."""
+    w = wl.WORKLOADS[name]
+    sample = None if w.B <= 8 else [0, w.B // 2, w.B - 1]
+    t = parity.closed_loop(lib, w, rounds, DEV, sample=sample, fused_step=True)
+    assert t.flagged_arm <= 2
+
+
+def test_bandit_step_equals_update_then_select(lib):
+    rng = np.random.default_rng(5)
+    B, gam = 70, [1, 2, 4, 7, 3]
+    K = len(gam)
+    for alg in (lib.BS_UCB, lib.BS_EXP3):
+        sa = lib.new_bandit(alg, B, gam, 0.5, DEV); sb = lib.new_bandit(alg, B, gam, 0.5, DEV)
+        arm_a = torch.zeros(B, dtype=torch.int32, device=DEV); arm_b = torch.zeros(B, dtype=torch.int32, device=DEV)
+        g_a = torch.zeros(B, dtype=torch.int32, device=DEV); g_b = torch.zeros(B, dtype=torch.int32, device=DEV)
+        ia = torch.zeros(B, K, dtype=torch.float64, device=DEV); ib = torch.zeros(B, K, dtype=torch.float64, device=DEV)
+        u = torch.as_tensor(rng.random(B).astype(np.float32), device=DEV)
+        act = torch.as_tensor((rng.random(B) < 0.85).astype(np.uint8), device=DEV)
+        lib.bs_bandit_select(sa, alg, B, K, u, act, arm_a, g_a)
+        lib.bs_bandit_select(sb, alg, B, K, u, act, arm_b, g_b)
+        for t in range(60):
+            y = torch.as_tensor(rng.integers(1, 9, size=B).astype(np.int32), device=DEV)
+            u = torch.as_tensor(rng.random(B).astype(np.float32), device=DEV)
+            lib.bs_bandit_update(sa, alg, B, K, arm_a, y, act)
+            lib.bs_bandit_select(sa, alg, B, K, u, act, arm_a, g_a, ia)
+            lib.bs_bandit_step(sb, alg, B, K, y, u, act, arm_b, g_b, ib)
+            assert torch.equal(arm_a, arm_b) and torch.equal(g_a, g_b)
+            assert torch.equal(torch.nan_to_num(ia, nan=-1.0), torch.nan_to_num(ib, nan=-1.0))
+        assert torch.equal(sa, sb)                                        # the whole state blob, bit for bit
