@@ -92,3 +92,38 @@ def test_lmhead_round_repeats_bit_for_bit(lib, name, reps):
     assert int(bad) == 0, f"{int(bad)} of {reps} repetitions differ from the first"
     st = lib.bs_get_device_status(ws, B, G, V)
     assert (st & ~lib.BS_DEV_RESIDUAL_FALLBACK == 0).all()
+
+
+def test_drafted_round_repeats_bit_for_bit(lib):
+    """Drafting on the device (one call per position), verification on the drafting statistics, resampling:
+    the drafted tokens, the outputs and the workspace repeat."""
+    w = wl.WORKLOADS["llama3_ucb"]
+    B, G, V, T = w.B, w.Gmax, w.V, w.temperature
+    _, rnd, gam, ua, ur = _inputs("llama3_ucb", 63)
+    ud = torch.as_tensor(rnd.uniforms.u_draft, device=DEV)
+    ws = lib.new_workspace(B, G, V, DEV)
+
+    def run():
+        tok = torch.full((B, G), -1, dtype=torch.int32, device=DEV)
+        for j in range(G):
+            lib.bs_draft_sample(rnd.draft, j, gam, ud, T, tok, ws)
+        acc = torch.empty(B, dtype=torch.int32, device=DEV)
+        p = torch.empty(B, G, dtype=torch.float32, device=DEV); q = torch.empty(B, G, dtype=torch.float32, device=DEV)
+        ot = torch.empty(B, G + 1, dtype=torch.int32, device=DEV); ol = torch.empty(B, dtype=torch.int32, device=DEV)
+        lib.bs_softmax_verify_drafted(rnd.target, rnd.draft, tok, gam, ua, T, acc, p, q, ws)
+        lib.bs_residual_sample(rnd.target, rnd.draft, tok, gam, acc, ur, T, ot, ol, ws)
+        return tok, acc, p, q, ot, ol
+
+    ref = run()
+    ref_ws = ws.clone()
+    bad = torch.zeros((), dtype=torch.int64, device=DEV)
+    reps = 300
+    for i in range(reps):
+        o = run()
+        same = (ws == ref_ws).all()
+        for a, b in zip(o, ref):
+            same = same & (a == b).all()
+        bad += (~same).to(torch.int64)
+    assert int(bad) == 0, f"{int(bad)} of {reps} repetitions differ from the first"
+    st = lib.bs_get_device_status(ws, B, G, V)
+    assert (st & ~lib.BS_DEV_RESIDUAL_FALLBACK == 0).all()
