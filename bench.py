@@ -421,6 +421,7 @@ def run_cuda(args, w):
     rsd = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(ksteps)]
     dft = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(ksteps)]
     walk_rows = torch.zeros((), dtype=torch.int64, device=dev)
+    resid_rows = torch.zeros((), dtype=torch.int64, device=dev)   # rows bs_residual_sample must read
     nk0 = pulls()
     for i in range(ksteps):
         s = sets[(args.warmup + args.steps + i) % ring]
@@ -441,6 +442,8 @@ def run_cuda(args, w):
             bs.bs_residual_sample(s["target"], s["draft"], s["tokens"], gamma_d, accept_len, s["u_resample"],
                                   w.temperature, out_tokens, out_len, ws)
         rsd[i][1].record(stream)
+        if not walk and w.temperature > 0.0:                   # the row pair of a rejected position, or the bonus row alone
+            resid_rows += torch.where(accept_len < gamma_d, 2, 1).sum()
         if walk:                                               # rows the walk had to read: up to the stop position
             tau = accept_len.to(torch.int64); gm = gamma_d.to(torch.int64)
             walk_rows += (tau + 1).sum() if drafted else torch.where(tau < gm, 2 * (tau + 1), 2 * gm + 1).sum()
@@ -454,6 +457,7 @@ def run_cuda(args, w):
     full_bytes = verify_bytes
     if walk:
         verify_bytes = float(walk_rows.item()) * V * es / ksteps
+    resid_bytes = float(resid_rows.item()) * V * es / ksteps
     draft_ms = sum(a.elapsed_time(b) for a, b in dft) / ksteps if drafted else None
     draft_bytes = float((dk * arm_gamma[None, :]).sum()) * V * es / ksteps if drafted else None
     mean_y = float(y_sum.item()) / (B * ksteps)
@@ -562,7 +566,12 @@ def run_cuda(args, w):
                          "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": ncu_traffic(w.name, verify_bytes), "bytes_per_launch": verify_bytes,
                          "nominal_peak": 8000.0, "frac_of_nominal": achieved / 8000.0,
-                         "ms_per_launch": verify_ms, "residual_ms_per_launch": resid_ms},
+                         "ms_per_launch": verify_ms, "residual_ms_per_launch": resid_ms,
+                         # the second kernel of the round, same units and peak: rows it must read / its event time
+                         "residual": (None if walk or resid_bytes <= 0 else
+                                      {"kernel": "residual_stream_kernel (bs_residual_sample)", "bytes_per_launch": resid_bytes,
+                                       "achieved": resid_bytes / (resid_ms * 1e-3) / 1e9,
+                                       "frac": resid_bytes / (resid_ms * 1e-3) / 1e9 / peak})},
             "e2e": e2e, "cpu_baseline": cpu, "clocks": clocks, "variants": variants,
             "other_workloads": getattr(args, "others", None),
             "gpu_launches": ((3 if walk else 4) - (1 if fused_bandit else 0) + (2 * G if drafted else 0)
