@@ -127,3 +127,27 @@ def test_drafted_round_repeats_bit_for_bit(lib):
     assert int(bad) == 0, f"{int(bad)} of {reps} repetitions differ from the first"
     st = lib.bs_get_device_status(ws, B, G, V)
     assert (st & ~lib.BS_DEV_RESIDUAL_FALLBACK == 0).all()
+
+
+def test_two_streams_with_their_own_workspaces_do_not_disturb_each_other(lib):
+    """Two batches in flight at once (two-call path, two streams, a workspace each) give what each gives alone."""
+    wa, rnda, gama, uaa, ura = _inputs("llama3_ucb", 64)
+    wb, rndb, gamb, uab, urb = _inputs("llama2_fixed", 65)
+    wsa = lib.new_workspace(wa.B, wa.Gmax, wa.V, DEV); wsb = lib.new_workspace(wb.B, wb.Gmax, wb.V, DEV)
+    refa = lib.verify_round(rnda.target, rnda.draft, rnda.tokens, gama, uaa, ura, wa.temperature, wsa)
+    refb = lib.verify_round(rndb.target, rndb.draft, rndb.tokens, gamb, uab, urb, wb.temperature, wsb)
+    torch.cuda.synchronize()
+    ref_wsa, ref_wsb = wsa.clone(), wsb.clone()
+    sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+    for i in range(200):
+        with torch.cuda.stream(sa):
+            oa = lib.verify_round(rnda.target, rnda.draft, rnda.tokens, gama, uaa, ura, wa.temperature, wsa)
+        with torch.cuda.stream(sb):
+            ob = lib.verify_round(rndb.target, rndb.draft, rndb.tokens, gamb, uab, urb, wb.temperature, wsb)
+            if i % 2:                                           # the shorter round twice: the overlap shifts
+                ob = lib.verify_round(rndb.target, rndb.draft, rndb.tokens, gamb, uab, urb, wb.temperature, wsb)
+        sa.synchronize(); sb.synchronize()
+        assert torch.equal(oa.out_tokens, refa.out_tokens) and torch.equal(oa.accept_len, refa.accept_len)
+        assert torch.equal(oa.p_tok, refa.p_tok) and torch.equal(wsa, ref_wsa), f"iteration {i}: first batch differs"
+        assert torch.equal(ob.out_tokens, refb.out_tokens) and torch.equal(ob.accept_len, refb.accept_len)
+        assert torch.equal(ob.p_tok, refb.p_tok) and torch.equal(wsb, ref_wsb), f"iteration {i}: second batch differs"
