@@ -508,7 +508,7 @@ def run_cuda(args, w):
         def e2e_step():
             for k in host:
                 devb[k].copy_(host[k], non_blocking=True)
-            step_calls(devb)
+            step_calls(devb, devb)                             # the uniforms of the next round arrive with it
             h_tokens.copy_(out_tokens, non_blocking=True)
             h_len.copy_(out_len, non_blocking=True)
             torch.cuda.current_stream().synchronize()          # the caller reads the tokens every round
