@@ -328,3 +328,42 @@ def test_largest_supported_sizes(lib, B, G, V, dtype):
     assert ((y == tau + 1) & (tau >= 0) & (tau <= rnd.gamma)).all()
     # one more than the limits is refused on the host
     assert lib.bs_workspace_bytes(B, G, (1 << 20) + 8) == 0 and lib.bs_workspace_bytes(4097, G, V) == 0
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("V", [3000, 40000, 20011])
+def test_masked_logits(lib, dtype, V):
+    """Logits filtered the way a sampler's top-k does it: everything outside a model's k best entries is
+    -inf, with a different set for the two models.  P or Q is exactly zero on most of the vocabulary; a
+    drafted token the target has masked must be rejected, whole segments hold no mass at all.  Both the
+    two-call path and the early-exit walk (aligned V only)."""
+    rng = np.random.default_rng(V + 1)
+    tally = parity.Tally()
+    B, G, T = 6, 5, 0.9
+    rnd = _random_round(rng, B, G, V, dtype, T, sigma=1.5)
+    for x, k in ((rnd.target, 40), (rnd.draft, 25)):
+        kth = x.float().topk(k, dim=-1).values[..., -1:]
+        x.masked_fill_(x.float() < kth, float("-inf"))
+    rnd.target[0, :, : V // 2] = float("-inf")                # the first half of the vocabulary carries nothing
+    rnd.tokens = wl.draw_draft_tokens(rnd.draft, T, rnd.uniforms.u_draft).contiguous()
+    rnd.gamma = np.array([G, G, G, 3, 1, 0], np.int32)
+    out = parity.gpu_round(lib, rnd, T)
+    st = lib.bs_get_device_status(out.workspace, B, G, V)
+    assert (st & ~lib.BS_DEV_RESIDUAL_FALLBACK == 0).all(), st
+    refs = parity.check_round(out, rnd, T, tally, where=f"masked V={V}")
+    assert tally.sequences == B
+    # a drafted token outside the target's kept set has p = 0: never accepted
+    p = out.p_tok.cpu().numpy(); tau = out.accept_len.cpu().numpy()
+    for b in range(B):
+        for j in range(int(rnd.gamma[b])):
+            if p[b, j] == 0.0:
+                assert tau[b] <= j
+    if V % 8 == 0:
+        ow = lib.verify_round_walk(rnd.target, rnd.draft, rnd.tokens, torch.as_tensor(rnd.gamma, device=DEV),
+                                   torch.as_tensor(rnd.uniforms.u_accept, device=DEV),
+                                   torch.as_tensor(rnd.uniforms.u_resample, device=DEV), T)
+        torch.cuda.synchronize()
+        assert torch.equal(ow.accept_len, out.accept_len) and torch.equal(ow.out_tokens, out.out_tokens)
+    # greedy on masked rows: the arg-max is a kept entry
+    outg = parity.gpu_round(lib, rnd, 0.0)
+    parity.check_round(outg, rnd, 0.0, tally, where=f"masked greedy V={V}")
