@@ -367,7 +367,8 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tm_h0, const __grid_const
                                             a1 += ex2(fmaf(__uint_as_float(v[i + 1]), p.c, nm));
                                         }
                                     }
-                                    on.s += a0 + a1;
+                                    const float dl = fmaf(on.m, p.c, nm);      // rounding error of nm, undone to first order
+                                    on.s = fmaf(a0 + a1, fmaf(-dl, 0.69314718f, 1.f), on.s);
                                 }
                             }
                         }

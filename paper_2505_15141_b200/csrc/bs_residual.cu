@@ -151,13 +151,13 @@ __global__ void __launch_bounds__(kThreads, 2) residual_kernel(const ResidParams
         f.c = p.c;
         f.bonus = tau >= g;
         const float2 ts = p.row_stats[(size_t)b * p.R + tau];
-        f.kt = -(ts.x * p.c + log2f(ts.y));
-        f.kd = 0.f;
+        MassFn::fold(ts.x, ts.y, p.c, f.kt, f.at);
+        f.kd = 0.f; f.ad = 1.f;
         const T* tp = row_ptr(static_cast<const T*>(p.target), b, p.Gmax + 1, tau, p.V);
         const T* dp = tp;
         if (!f.bonus) {
             const float2 ds = p.row_stats[(size_t)b * p.R + p.Gmax + 1 + tau];
-            f.kd = -(ds.x * p.c + log2f(ds.y));
+            MassFn::fold(ds.x, ds.y, p.c, f.kd, f.ad);
             dp = row_ptr(static_cast<const T*>(p.draft), b, p.Gmax, tau, p.V);
         }
         // ---- level 1: segment masses, no CTA-wide synchronisation between segments ----

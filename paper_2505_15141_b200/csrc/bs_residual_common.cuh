@@ -33,15 +33,30 @@ struct ResidParams {
 };
 constexpr int kResidVerify = 0, kResidDraft = 1;
 
-// Mass of one element.  kt / kd fold the row max and normaliser: p = 2^(x*c + kt).
+// Mass of one element.  kt / kd fold the row max and normaliser into the exponent, p = at * 2^(x*c + kt):
+// kt is the rounded -(m c + log2 Z); at = 2^(what the two roundings lost) to first order, so that P and Q
+// are not scaled apart by an error that grows with |m| / temperature.
 struct MassFn {
     float c, kt, kd;
+    float at, ad;
     bool bonus;
     __device__ __forceinline__ float operator()(float xt, float xd) const {
-        float pv = ex2(fmaf(xt, c, kt));
+        const float pv = at * ex2(fmaf(xt, c, kt));
         if (bonus) return pv;
-        float qv = ex2(fmaf(xd, c, kd));
-        return fmaxf(0.f, pv - qv);
+        const float qv = ex2(fmaf(xd, c, kd));
+        return fmaxf(0.f, fmaf(-ad, qv, pv));
+    }
+    // row statistics (raw max m, sum Z relative to m) -> (k, a)
+    __device__ static __forceinline__ void fold(float m, float Z, float c, float& k, float& a) {
+        const float p1 = m * c;
+        const float d1 = fmaf(m, c, -p1);                     // m c = p1 + d1 exactly
+        const float l = log2f(Z);
+        const float sum = p1 + l;
+        const float bb = sum - p1;
+        const float d2 = (p1 - (sum - bb)) + (l - bb);        // p1 + l = sum + d2 exactly
+        k = -sum;
+        a = fmaf(-(d1 + d2), 0.69314718f, 1.f);               // 2^-(d1 + d2), |d1 + d2| < 1e-4
+        if (!(fabsf(d1 + d2) < 1.f)) a = 1.f;                 // non-finite statistics: reported elsewhere
     }
 };
 

@@ -24,7 +24,8 @@ struct RsMeta {
     int nvec;        // valid 16-byte vectors in the first half of the slot
     int nvec2;       // ... in the second half: the draft row's segment, or segment sg + 1 of a row sampled alone
     int flags;       // bit 0: bonus (target row only), bit 1: last item of this sequence in the CTA's range
-    float kt, kd;    // p_v = 2^(x_t c + kt), q_v = 2^(x_d c + kd)
+    float kt, kd;    // p_v = at 2^(x_t c + kt), q_v = ad 2^(x_d c + kd)
+    float at, ad;
 };
 
 // Per-sequence facts every role derives the same way.

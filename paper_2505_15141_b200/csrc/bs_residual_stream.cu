@@ -117,12 +117,13 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
             rs_items(s_prefix[b], rs_nitems(sq, p.nseg), lo, hi, i0, i1);
             if (i1 <= i0) continue;
             const float2 ts = p.row_stats[(size_t)b * p.R + rs_tslot(p, sq)];
-            float kt = -(ts.x * p.c + log2f(ts.y)), kd = 0.f;
+            float kt, at, kd = 0.f, ad = 1.f;
+            MassFn::fold(ts.x, ts.y, p.c, kt, at);
             const T* tp = rs_trow<T>(p, b, sq);
             const T* dp = tp;
             if (!sq.bonus) {
                 const float2 ds = p.row_stats[(size_t)b * p.R + p.Gmax + 1 + sq.tau];
-                kd = -(ds.x * p.c + log2f(ds.y));
+                MassFn::fold(ds.x, ds.y, p.c, kd, ad);
                 dp = row_ptr(static_cast<const T*>(p.draft), b, p.Gmax, sq.tau, p.V);
             }
             for (int it = i0; it < i1; ++it) {
@@ -137,7 +138,7 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
                 RsMeta m;
                 m.b = b; m.sg = sg; m.nvec = n / kVec; m.nvec2 = n2 / kVec;
                 m.flags = (sq.bonus ? 1 : 0) | (it == i1 - 1 ? 2 : 0);
-                m.kt = kt; m.kd = kd;
+                m.kt = kt; m.kd = kd; m.at = at; m.ad = ad;
                 s_meta[slot] = m;
                 const uint32_t bar = smem_u32(&s_full[slot]);
                 const uint32_t dst = smem_u32(ring + (size_t)slot * kRsStageBytes);
@@ -185,11 +186,11 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
                 f.c = p.c;
                 f.bonus = sq.bonus;
                 const float2 ts = p.row_stats[(size_t)b * p.R + rs_tslot(p, sq)];
-                f.kt = -(ts.x * p.c + log2f(ts.y));
-                f.kd = 0.f;
+                MassFn::fold(ts.x, ts.y, p.c, f.kt, f.at);
+                f.kd = 0.f; f.ad = 1.f;
                 if (!sq.bonus) {
                     const float2 ds = p.row_stats[(size_t)b * p.R + p.Gmax + 1 + sq.tau];
-                    f.kd = -(ds.x * p.c + log2f(ds.y));
+                    MassFn::fold(ds.x, ds.y, p.c, f.kd, f.ad);
                 }
                 rs_level2<T>(p, b, sq, f);
             }
@@ -204,7 +205,7 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
         if (!mbar_wait_warp(smem_u32(&s_full[slot]), ph)) { atomicExch(p.abort_flag, 1); return; }
         const RsMeta m = s_meta[slot];
         MassFn f;
-        f.c = p.c; f.kt = m.kt; f.kd = m.kd; f.bonus = (m.flags & 1) != 0;
+        f.c = p.c; f.kt = m.kt; f.kd = m.kd; f.at = m.at; f.ad = m.ad; f.bonus = (m.flags & 1) != 0;
         const uint32_t base = smem_u32(ring + (size_t)slot * kRsStageBytes) + (uint32_t)(warp * kRsPieceBytes + lane * 16);
         uint4 a[kRsVecPerLane], d[kRsVecPerLane];
         bool valid[kRsVecPerLane], valid2[kRsVecPerLane];

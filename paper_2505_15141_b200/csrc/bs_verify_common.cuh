@@ -130,7 +130,11 @@ __device__ __forceinline__ void online_add(Online& on, const uint4 (&v)[N], floa
                 acc1 += ex2(fmaf(f[q + 1], c, nm));
             }
         }
-        on.s += acc0 + acc1;
+        // nm is the rounded product: the terms above are 2^((x - m) c) times 2^dl with dl = m c + nm, the
+        // rounding error of the product, which one FMA gives exactly.  Undone to first order (dl^2 < 1e-9),
+        // so that the sum does not carry an error that grows with |m| / temperature.
+        const float dl = fmaf(on.m, c, nm);
+        on.s = fmaf(acc0 + acc1, fmaf(-dl, 0.69314718f, 1.f), on.s);
     }
 }
 

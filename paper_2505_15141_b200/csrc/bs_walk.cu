@@ -48,7 +48,7 @@ struct WkMeta {
     int type, b, k;
     int row;               // stats: 0 = target row k, 1 = draft row k;  mass: 1 = target row only (bonus)
     int sg, nvec, flags;   // flags bit 0: first stage of a row piece, bit 1: last stage of a piece / of the CTA's share
-    float kt, kd;
+    float kt, kd, at, ad;
 };
 // Per event handed to the finisher (written by consumer warp 0).
 struct WkEvent {
@@ -156,7 +156,7 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                             // reports that it has seen the decision, so that the words can be cleared
                             WkMeta m;
                             m.type = kItemAck; m.b = b; m.k = sq.k; m.row = 0; m.sg = 0; m.nvec = 0; m.flags = 3;
-                            m.kt = m.kd = 0.f;
+                            m.kt = m.kd = 0.f; m.at = m.ad = 1.f;
                             ok = issue(m, nullptr, nullptr, 0);
                             sq.stage = 2;
                             --alive;
@@ -169,10 +169,11 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                         const T* tp = row_ptr(static_cast<const T*>(v.target), b, v.Gmax + 1, k, v.V);
                         const T* dp = bonus ? nullptr : row_ptr(static_cast<const T*>(v.draft), b, v.Gmax, k, v.V);
                         const float2 ts = __ldcg(v.row_stats + (size_t)b * v.R + k);
-                        float kt = -(ts.x * v.c + log2f(ts.y)), kd = 0.f;
+                        float kt, at, kd = 0.f, ad = 1.f;
+                        MassFn::fold(ts.x, ts.y, v.c, kt, at);
                         if (!bonus) {
                             const float2 ds = __ldcg(v.row_stats + (size_t)b * v.R + v.Gmax + 1 + k);
-                            kd = -(ds.x * v.c + log2f(ds.y));
+                            MassFn::fold(ds.x, ds.y, v.c, kd, ad);
                         }
                         const int rseg = p.r.seg, rnseg = p.r.nseg;
                         const int j0 = (int)((long long)rnseg * part / p.nG), j1 = (int)((long long)rnseg * (part + 1) / p.nG);
@@ -182,7 +183,7 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                             WkMeta m;
                             m.type = kItemMass; m.b = b; m.k = k; m.row = bonus ? 1 : 0; m.sg = sg; m.nvec = n / kVec;
                             m.flags = (sg == j0 ? 1 : 0) | (sg == j1 - 1 ? 2 : 0);
-                            m.kt = kt; m.kd = kd;
+                            m.kt = kt; m.kd = kd; m.at = at; m.ad = ad;
                             ok = issue(m, tp + e0, bonus ? nullptr : dp + e0, (uint32_t)n * (uint32_t)sizeof(T));
                         }
                         sq.stage = 2;                          // this sequence is done for the producer
@@ -206,7 +207,7 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                         WkMeta m;
                         m.type = kItemStats; m.b = b; m.k = k; m.row = row; m.sg = sg; m.nvec = n / kVec;
                         m.flags = ((sg == 0 || i == i0) ? 1 : 0) | ((sg == v.nseg - 1 || i == i1 - 1) ? 2 : 0);
-                        m.kt = m.kd = 0.f;
+                        m.kt = m.kd = 0.f; m.at = m.ad = 1.f;
                         ok = issue(m, rowp + e0, nullptr, (uint32_t)n * (uint32_t)sizeof(T));
                     }
                     sq.stage = 1;
@@ -224,7 +225,7 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
         if (!ok) atomicExch(v.abort_flag, 1);
         // the end marker lets the consumers and the finisher leave (also after a failed wait, if a slot frees up)
         WkMeta e;
-        e.type = kItemEnd; e.b = 0; e.k = 0; e.row = 0; e.sg = 0; e.nvec = 0; e.flags = 2; e.kt = e.kd = 0.f;
+        e.type = kItemEnd; e.b = 0; e.k = 0; e.row = 0; e.sg = 0; e.nvec = 0; e.flags = 2; e.kt = e.kd = 0.f; e.at = e.ad = 1.f;
         issue(e, nullptr, nullptr, 0);
         return;
     }
@@ -421,11 +422,11 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                 MassFn f;
                 f.c = v.c; f.bonus = sq.bonus != 0;
                 const float2 ts = __ldcg(v.row_stats + (size_t)b * v.R + k);
-                f.kt = -(ts.x * v.c + log2f(ts.y));
-                f.kd = 0.f;
+                MassFn::fold(ts.x, ts.y, v.c, f.kt, f.at);
+                f.kd = 0.f; f.ad = 1.f;
                 if (!f.bonus) {
                     const float2 ds = __ldcg(v.row_stats + (size_t)b * v.R + v.Gmax + 1 + k);
-                    f.kd = -(ds.x * v.c + log2f(ds.y));
+                    MassFn::fold(ds.x, ds.y, v.c, f.kd, f.ad);
                 }
                 rs_level2<T>(p.r, b, sq, f);                   // token, out_tokens, out_len; clears the mass ticket
                 if (lane == 0) {                               // leave the workspace clean for the next call
@@ -477,7 +478,7 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
         } else if (m.type == kItemMass) {
             // a 16 KB segment of the row pair: warp w owns the w-th 1 KB piece and writes its mass
             MassFn f;
-            f.c = v.c; f.kt = m.kt; f.kd = m.kd; f.bonus = m.row != 0;
+            f.c = v.c; f.kt = m.kt; f.kd = m.kd; f.at = m.at; f.ad = m.ad; f.bonus = m.row != 0;
             const uint32_t pb = base + (uint32_t)(warp * kRsPieceBytes + lane * 16);
             uint4 a[kRsVecPerLane], d[kRsVecPerLane];
             bool valid[kRsVecPerLane];
