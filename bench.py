@@ -43,9 +43,9 @@ FALLBACK_HBM_GBS = 6650.0
 # bytes, the writes (workspace partials, write-backs) do not.  None = not captured.
 NCU_TRAFFIC = {
     "qwen_exp3": (1.0003, 4.0e6),          # profiles/verify_stream_kernel.md, fp32 column
-    "llama3_ucb": (1.0005, 4.0e6),         # profiles/verify_stream_kernel.md, bf16 column
-    "lmhead_llama3": (1.0000, 27.7e6),     # profiles/lmhead_gemm_kernel.md, B=16 (logits still dirty in L2 not counted)
-    "lmhead_llama3_b128": (1.0180, 568.0e6),
+    "llama3_ucb": (1.0005, 4.2e6),         # profiles/verify_stream_kernel.md, bf16 column
+    "lmhead_llama3": (1.0000, 30.6e6),     # profiles/lmhead_gemm_kernel.md, B=16 (logits still dirty in L2 not counted)
+    "lmhead_llama3_b128": (1.0180, 568.1e6),
 }
 
 
