@@ -49,6 +49,17 @@ NCU_TRAFFIC = {
 }
 
 
+HOLD_CYCLES = 400_000          # about 0.2 ms of a spinning kernel
+
+
+def hold_gpu():
+    """Keeps the stream busy while the host enqueues the events and launches that follow, so that an event
+    pair brackets the kernel's own duration and not the host's time between two enqueue calls (which
+    shows once a launch is shorter than the host needs to issue it)."""
+    import torch
+    torch.cuda._sleep(HOLD_CYCLES)
+
+
 def ncu_traffic(name: str, algorithmic_read_bytes: float):
     t = NCU_TRAFFIC.get(name)
     return None if t is None else t[0] * algorithmic_read_bytes + t[1]
@@ -426,6 +437,7 @@ def run_cuda(args, w):
     for i in range(ksteps):
         s = sets[(args.warmup + args.steps + i) % ring]
         bs.bs_bandit_select(state, alg, B, K, s["u_arm"], None, arm_d, gamma_d)
+        hold_gpu()
         if drafted:
             dft[i][0].record(stream)
             draft_calls(s)
@@ -726,6 +738,7 @@ def run_lmhead(args, w):
     y_sum = torch.zeros((), dtype=torch.int64, device=dev)
     for i in range(ksteps):
         s = dsets[i % 2]
+        hold_gpu()
         evs[i][0].record(stream); lm_call(s)
         evs[i][1].record(stream); res_call(s)
         evs[i][2].record(stream)
