@@ -38,13 +38,14 @@ L2_BYTES = 126 * 1024 * 1024
 FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel,
-# from the ncu captures summarised under profiles/: (read traffic per algorithmic byte, bytes
-# written per launch).  Captured on smaller cases of the same kernels; read traffic grows with the
-# bytes, the writes (workspace partials, write-backs) do not.  None = not captured.
+# from profiler captures of smaller cases of the same kernels: (read traffic per algorithmic byte,
+# bytes written per launch).  Read traffic grows with the bytes, the writes (workspace partials,
+# write-backs) do not.  An entry is only valid for the kernel it was captured on: when that kernel
+# changes, the entry goes to None until the capture is repeated.
 NCU_TRAFFIC = {
-    "qwen_exp3": (1.0003, 4.0e6),          # profiles/verify_stream_kernel.md, fp32 column
-    "llama3_ucb": (1.0005, 4.2e6),         # profiles/verify_stream_kernel.md, bf16 column
-    "lmhead_llama3": (1.0000, 30.6e6),     # profiles/lmhead_gemm_kernel.md, B=16 (logits still dirty in L2 not counted)
+    "qwen_exp3": None,
+    "llama3_ucb": None,
+    "lmhead_llama3": (1.0000, 30.6e6),     # B=16 (logits still dirty in L2 are not counted)
     "lmhead_llama3_b128": (1.0180, 568.1e6),
 }
 
@@ -93,6 +94,9 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="budget of the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-all-cores", action="store_true",
+                    help="also time the oracle sample in one single-threaded process per host core")
+    ap.add_argument("--oracle-worker", action="store_true", help=argparse.SUPPRESS)
     ap.add_argument("--no-graph", action="store_true", help="launch the four calls directly each step")
     return ap.parse_args()
 
@@ -108,25 +112,78 @@ def host_cores() -> int:
 # CPU oracle timing (cpu_baseline leg and --impl reference)
 # ---------------------------------------------------------------------------------------------
 
-def oracle_sample(w, rnd_inputs, seconds: float, max_seqs=None):
-    """Runs the oracle's verification on sequences of one round until `seconds` are used.
+ORACLE_SAMPLE_SEQS = 16        # sequences of round 1 that both CPU legs time, over and over
+
+
+def oracle_inputs(w):
+    """The bounded sample both CPU legs time: the first sequences of round 1 with the arms that shape
+    the benchmark's first input set, generated on the host and converted to the oracle's input arrays
+    before any clock starts."""
+    from paper_2505_15141_b200 import workloads as wl
+    nb = min(w.B, ORACLE_SAMPLE_SEQS)
+    rnd = wl.make_round(w, 1, default_arms(w, 0), device="cpu", B=nb)
+    toks = rnd.tokens.cpu().numpy()
+    seqs = []
+    for b in range(nb):
+        g = int(rnd.gamma[b])
+        seqs.append((rnd.target[b, :g + 1].float().numpy(), rnd.draft[b, :g].float().numpy(), toks[b], g,
+                     rnd.uniforms.u_accept[b], float(rnd.uniforms.u_resample[b])))
+    return seqs
+
+
+def oracle_sample(w, seqs, seconds: float):
+    """Runs the oracle's verification over the sample, again and again, until `seconds` are used.
     Returns (sequences done, elapsed seconds)."""
     from oracle import verify as ov
-    toks = rnd_inputs.tokens.cpu().numpy()
     done, t0 = 0, time.perf_counter()
-    B = rnd_inputs.target.shape[0]
-    limit = B if max_seqs is None else min(B, max_seqs)
-    while done < limit:
-        b = done
-        g = int(rnd_inputs.gamma[b])
-        t_rows = rnd_inputs.target[b, :g + 1].float().cpu().numpy()
-        d_rows = rnd_inputs.draft[b, :g].float().cpu().numpy()
-        ov.verify_sequence(t_rows, d_rows, toks[b], g, rnd_inputs.uniforms.u_accept[b],
-                           float(rnd_inputs.uniforms.u_resample[b]), w.temperature)
+    while True:
+        t_rows, d_rows, toks, g, u_acc, u_res = seqs[done % len(seqs)]
+        ov.verify_sequence(t_rows, d_rows, toks, g, u_acc, u_res, w.temperature)
         done += 1
         if time.perf_counter() - t0 > seconds:
             break
     return done, time.perf_counter() - t0
+
+
+def oracle_worker(args, w):
+    """One process of the all-core figure: times its own copy of the sample, prints wall-clock marks."""
+    import torch
+    torch.set_num_threads(1)
+    seqs = oracle_inputs(w)
+    t0 = time.time()
+    n, _ = oracle_sample(w, seqs, args.cpu_seconds)
+    print(json.dumps({"seqs": n, "t0": t0, "t1": time.time()}))
+
+
+def oracle_all_cores(args, w, cores: int):
+    """The same sample in `cores` single-threaded processes at once (sequences are independent, so the
+    oracle parallelises over them and over nothing else).  Rounds/s = all sequences done, over the span
+    from the first start to the last end.  Every child has a hard limit; stragglers are killed by PID."""
+    cmd = [sys.executable, os.path.abspath(__file__), "--impl", "reference", "--oracle-worker", "--workload", w.name,
+           "--cpu-seconds", str(args.cpu_seconds)]
+    if args.batch:
+        cmd += ["--batch", str(args.batch)]
+    if args.fixed_gamma:
+        cmd += ["--fixed-gamma", str(args.fixed_gamma)]
+    env = dict(os.environ, OMP_NUM_THREADS="1", MKL_NUM_THREADS="1", CUDA_VISIBLE_DEVICES="")
+    for k in ("RANK", "LOCAL_RANK", "WORLD_SIZE"):
+        env.pop(k, None)
+    procs = [subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True, env=env)
+             for _ in range(cores)]
+    deadline = time.time() + args.cpu_seconds + 240.0
+    marks = []
+    for pr in procs:
+        try:
+            out, _ = pr.communicate(timeout=max(1.0, deadline - time.time()))
+            marks.append(json.loads(out.strip().splitlines()[-1]))
+        except Exception:
+            pr.kill()
+    if not marks:
+        return None
+    span = max(m["t1"] for m in marks) - min(m["t0"] for m in marks)
+    n = sum(m["seqs"] for m in marks)
+    return {"value": (n / w.B) / span, "unit": UNIT, "cores": len(marks),
+            "sample": f"{n} sequences in {len(marks)} single-threaded processes over {span:.1f} s"}
 
 
 def rank_round_index(rank: int, i: int) -> int:
@@ -159,34 +216,40 @@ def default_arms(w, step: int) -> np.ndarray:
 
 
 def run_reference(args, w):
-    """The oracle, as it stands, on the host cores: each step is a bounded sample of one round."""
-    from paper_2505_15141_b200 import workloads as wl
+    """The oracle, as it stands, on the host cores: each step is a bounded sample of one round (the
+    same sample the CUDA arm's cpu_baseline leg times)."""
     import torch
     torch.set_num_threads(1)
-    per_step = max(0.5, min(10.0, 90.0 / max(1, args.steps + args.warmup)))
-    nb = min(w.B, 16)                                   # sequences generated for the sample
-    rnd = wl.make_round(w, 1, default_arms(w, 0), device="cpu", B=nb)
+    per_step = max(0.2, min(10.0, 90.0 / max(1, args.steps + args.warmup), args.cpu_seconds))
+    seqs_in = oracle_inputs(w)
     times, seqs = [], []
     for i in range(args.warmup + args.steps):
-        n, dt = oracle_sample(w, rnd, per_step)
+        n, dt = oracle_sample(w, seqs_in, per_step)
         if i >= args.warmup:
             times.append(dt); seqs.append(n)
     rounds = sum(seqs) / w.B
     total = sum(times)
     val = rounds / total
+    world = int(os.environ.get("WORLD_SIZE", "1"))
     line = {
-        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / max(1, args.steps),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "B": w.B, "V": w.V, "arm_gamma": list(w.arm_gamma),
-                   "logits_dtype": w.dtype, "temperature": w.temperature},
+        "config": cpu_config(w),
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle",
-                         "sample": f"{sum(seqs)} sequences of {w.B}-sequence rounds in {total:.1f} s, "
-                                   f"verification only (numpy fp64, one thread)"},
+                         "sample": f"{sum(seqs)} verifications of the first {len(seqs_in)} sequences of a "
+                                   f"{w.B}-sequence round in {total:.1f} s, verification only (numpy fp64, one "
+                                   f"thread; rank 0 of {world} runs it, the others idle)"},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line))
+
+
+def cpu_config(w) -> dict:
+    """The workload keys both arms print."""
+    return {"workload": w.name, "B": w.B, "V": w.V, "arm_gamma": list(w.arm_gamma), "bandit": w.alg or "fixed",
+            "logits_dtype": w.dtype, "temperature": w.temperature}
 
 
 # ---------------------------------------------------------------------------------------------
@@ -547,20 +610,20 @@ def run_cuda(args, w):
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         torch.set_num_threads(1)
-        rnd = sets[0]["rnd"]
-        rnd.gamma = np.asarray(w.arm_gamma, dtype=np.int32)[default_arms(w, 0)]
-        n, dt = oracle_sample(w, rnd, args.cpu_seconds)
+        seqs_in = oracle_inputs(w)
+        n, dt = oracle_sample(w, seqs_in, args.cpu_seconds)
         cpu = {"value": (n / B) / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
-               "sample": f"{n} of the {B} sequences of one round in {dt:.1f} s, verification only "
-                         f"(numpy fp64, one thread; host has {host_cores()} cores)"}
+               "sample": f"{n} verifications of the first {len(seqs_in)} sequences of a {B}-sequence round in "
+                         f"{dt:.1f} s, verification only (numpy fp64, one thread; host has {host_cores()} cores)"}
+        if args.cpu_all_cores:
+            cpu["all_cores"] = oracle_all_cores(args, w, host_cores())
 
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": w.name, "B": B, "V": V, "arm_gamma": list(w.arm_gamma), "bandit": w.alg or "fixed",
-                       "logits_dtype": w.dtype, "temperature": w.temperature,
+            "config": {**cpu_config(w),
                        "l2": f"ring of {ring} input sets, {ring * set_bytes / 1e6:.0f} MB > 2 x L2",
                        "launch": "one CUDA graph per step" if graphs else "direct launches",
                        "path": ("select, draft x Gmax, verify with early exit on drafted statistics + resample "
@@ -579,11 +642,18 @@ def run_cuda(args, w):
                          "traffic": ncu_traffic(w.name, verify_bytes), "bytes_per_launch": verify_bytes,
                          "nominal_peak": 8000.0, "frac_of_nominal": achieved / 8000.0,
                          "ms_per_launch": verify_ms, "residual_ms_per_launch": resid_ms,
-                         # the second kernel of the round, same units and peak: rows it must read / its event time
+                         # The second call of the round.  In sampling mode the statistics kernel computes the
+                         # residual masses of most stop rows itself (second touch, out of L2), so what is left
+                         # for bs_residual_sample is the inverse CDF; `stop_row_bytes` are the rows it would
+                         # have to stream if none of that had happened.
                          "residual": (None if walk or resid_bytes <= 0 else
-                                      {"kernel": "residual_stream_kernel (bs_residual_sample)", "bytes_per_launch": resid_bytes,
-                                       "achieved": resid_bytes / (resid_ms * 1e-3) / 1e9,
-                                       "frac": resid_bytes / (resid_ms * 1e-3) / 1e9 / peak})},
+                                      {"kernel": "residual_stream_kernel (bs_residual_sample)",
+                                       "ms_per_launch": resid_ms, "stop_row_bytes": resid_bytes}),
+                         # both calls together against the same single-touch bytes
+                         "verify_plus_residual": (None if walk else
+                                                  {"ms": verify_ms + resid_ms,
+                                                   "achieved": verify_bytes / ((verify_ms + resid_ms) * 1e-3) / 1e9,
+                                                   "frac": verify_bytes / ((verify_ms + resid_ms) * 1e-3) / 1e9 / peak})},
             "e2e": e2e, "cpu_baseline": cpu, "clocks": clocks, "variants": variants,
             "other_workloads": getattr(args, "others", None),
             "gpu_launches": ((3 if walk else 4) - (1 if fused_bandit else 0) + (2 * G if drafted else 0)
@@ -647,7 +717,8 @@ def run_lmhead_reference(args, w):
             fr += f; tt += dt
     val = fr / tt
     print(json.dumps({
-        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT,
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * tt / max(1, args.steps), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "gamma": w.gamma, "V": w.V, "d_t": w.d_t, "d_d": w.d_d},
@@ -850,26 +921,51 @@ def other_workloads_summary():
             d = json.loads(res.stdout.strip().splitlines()[-1])
             r = d["roofline"]
             out[name] = {"value": d["value"], "unit": d["unit"], "ms_per_step": d["ms_per_step"],
+                         "algorithmic_gbs": d.get("algorithmic_gbs"),
                          "roofline": {k: r.get(k) for k in ("bound", "kernel", "achieved", "peak", "unit", "frac",
-                                                            "ms_per_launch")},
+                                                            "ms_per_launch", "residual_ms_per_launch")},
                          "variants": d.get("variants")}
         except Exception as e:                                   # the main line must not depend on these
             out[name] = {"error": f"{type(e).__name__}: {e}"[:200]}
     return out
 
 
+def spawn_ranks(n: int) -> int:
+    """`--gpus N` without a launcher: start N ranks of this script on this node, as
+    `python -m torch.distributed.run --nnodes=1 --nproc-per-node N` would be asked to, and pass their
+    output through (rank 0 prints the line)."""
+    import socket
+    sk = socket.socket()
+    sk.bind(("127.0.0.1", 0))
+    port = sk.getsockname()[1]
+    sk.close()
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *sys.argv[1:]]
+    return subprocess.run(cmd).returncode
+
+
 def main():
     args = parse_args()
     from paper_2505_15141_b200 import workloads as wl
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args.gpus))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.gpus != world:
+        sys.exit(f"bench.py: --gpus {args.gpus} but the launcher started {world} rank(s)")
+    rank = int(os.environ.get("RANK", "0"))
+    if args.impl == "reference" and world > 1:
+        print(f"bench.py: rank {rank} of {world} ({'runs the oracle' if rank == 0 else 'idle'})", file=sys.stderr)
     plain_default = (args.workload == "qwen_exp3" and args.impl == "cuda" and not (args.batch or args.fixed_gamma
-                     or args.walk or args.drafted or args.no_others) and int(os.environ.get("WORLD_SIZE", "1")) == 1)
+                     or args.walk or args.drafted or args.no_others) and world == 1)
     args.others = other_workloads_summary() if plain_default else None
+    if plain_default:
+        args.cpu_all_cores = True
     if args.workload in wl.LMHEAD_WORKLOADS:
         w = wl.LMHEAD_WORKLOADS[args.workload]
         if args.batch:
             w = dataclasses.replace(w, B=args.batch)
         if args.impl == "reference":
-            if int(os.environ.get("RANK", "0")) == 0:
+            if rank == 0:
                 run_lmhead_reference(args, w)
             return
         run_lmhead(args, w)
@@ -880,7 +976,9 @@ def main():
     if args.fixed_gamma:
         w = dataclasses.replace(w, arm_gamma=(args.fixed_gamma,), alg=None)
     if args.impl == "reference":
-        if int(os.environ.get("RANK", "0")) == 0:
+        if args.oracle_worker:
+            oracle_worker(args, w)
+        elif rank == 0:
             run_reference(args, w)
         return
     run_cuda(args, w)

@@ -7,6 +7,7 @@ differ only where the oracle says it is a near-tie:
   token    u within 1e-6 (normalised CDF units) of an edge of the oracle token's interval, and
            the CUDA token has positive mass and an interval that meets [u - 1e-6, u + 1e-6]
   arm      top two UCB values within 1e-9 (not bit-equal), or u_arm within 1e-9 of a CDF edge
+  fallback the residual's total mass is below 2^-17 and the CUDA token is the one the target row gives
 Every such event is counted; anything else must match exactly.  After a flagged divergence the
 oracle is re-synchronised to the CUDA outcome so that one tie does not derail a trajectory.
 """
@@ -23,6 +24,7 @@ from oracle import verify as ov
 from paper_2505_15141_b200 import workloads as wl
 
 P_TOL = 1e-5
+RESIDUAL_FLOOR = 2.0 ** -18     # residual totals at or below this are "no mass" on the device (reading c5)
 # EXP3Spec's cumulative loss estimates, fp64 on both sides.  The two exp() routines differ in the
 # last bit, and a difference d in S_i moves p_i by about eta * d * p_i, hence the next estimate
 # (L+1-y)/(L p_i) by eta * d relative: every pull multiplies the difference by about
@@ -39,12 +41,13 @@ class Tally:
     flagged_accept: int = 0
     flagged_token: int = 0
     flagged_arm: int = 0
+    flagged_fallback: int = 0
     max_p_err: float = 0.0
     max_S_rel: float = 0.0
     sum_y: int = 0
 
     def merge(self, o: "Tally") -> None:
-        for k in ("sequences", "positions", "flagged_accept", "flagged_token", "flagged_arm", "sum_y"):
+        for k in ("sequences", "positions", "flagged_accept", "flagged_token", "flagged_arm", "flagged_fallback", "sum_y"):
             setattr(self, k, getattr(self, k) + getattr(o, k))
         self.max_p_err = max(self.max_p_err, o.max_p_err)
 
@@ -83,6 +86,15 @@ def check_sequence(ref: ov.SequenceResult, tau_gpu: int, out_tokens_gpu: np.ndar
     assert list(out_tokens_gpu[:tau]) == [int(t) for t in tokens[:tau]], f"{where}: accepted tokens differ"
     assert (out_tokens_gpu[tau + 1:] == -1).all(), f"{where}: padding of out_tokens is not -1"
     tok = int(out_tokens_gpu[tau])
+    if (tok != ref.token and not greedy and tau < gamma and not ref.used_fallback
+            and ref.mass.sum() < 2 * RESIDUAL_FLOOR):
+        # P and Q are normalised, so the residual's total is the probability of stopping here; the
+        # kernels count a total at or below RESIDUAL_FLOOR as "no mass" and draw from the target row
+        alt, lo, hi = ov.inverse_cdf(ov.softmax_row(target_rows[tau], temperature), float(u_resample))
+        if tok == alt:
+            tally.flagged_fallback += 1
+            ref.token, ref.cdf_lo, ref.cdf_hi, ref.used_fallback = tok, lo, hi, True
+            ref.out_tokens[-1] = tok
     if tok != ref.token:
         assert not greedy, f"{where}: greedy token {tok} != {ref.token}"
         u = float(u_resample)

@@ -73,13 +73,21 @@ def test_entry_points_agree_on_random_shapes(lib, B, G, V, bf16, T):
     ref = outs["plain"]
     tau = ref.accept_len.cpu().numpy()
     assert ((tau >= 0) & (tau <= gamma)).all() and (ref.out_len.cpu().numpy() == tau + 1).all()
+    # Two paths may only differ on a sequence where the oracle sees a near-tie: every differing sequence
+    # goes to the oracle on both sides, which accepts a deviation only if it is a flagged accept or
+    # CDF-edge tie, and counts it.
+    ties = parity.Tally()
     for k in ("drafted", "walk", "walk_drafted"):
         o = outs[k]
-        same = (o.accept_len == ref.accept_len)
-        assert same.float().mean() >= 0.97 or int((~same).sum()) <= 1, k       # near-ties only
         assert torch.equal(o.out_len, o.accept_len + 1), k
-        agree = same & (o.out_tokens == ref.out_tokens).all(dim=1)
-        assert agree.float().mean() >= 0.95 or int((~agree).sum()) <= 1, k
+        agree = (o.accept_len == ref.accept_len) & (o.out_tokens == ref.out_tokens).all(dim=1)
+        differ = [int(b) for b in torch.nonzero(~agree).flatten().cpu().numpy()]
+        if differ:
+            before = ties.flagged_accept + ties.flagged_token + ties.flagged_fallback
+            parity.check_round(ref, rnd, T, ties, seqs=differ, where=f"fuzz plain vs {k}")
+            parity.check_round(o, rnd, T, ties, seqs=differ, where=f"fuzz {k} vs plain", walk=k.startswith("walk"))
+            assert ties.flagged_accept + ties.flagged_token + ties.flagged_fallback > before, (k, differ)
+    assert ties.flagged_accept + ties.flagged_token + ties.flagged_fallback <= max(4, B // 50), vars(ties)
     assert torch.equal(outs["drafted"].accept_len, ref.accept_len)              # same statistics kernels, same pieces
     # a few sequences of every path against the oracle
     seqs = sorted(set(int(x) for x in rng.integers(0, B, size=min(B, 3))))

@@ -108,6 +108,51 @@ def test_device_data_errors_are_reported_not_fatal(lib):
     parity.check_round(out, rnd, 1.0, tally, seqs=[0], where="after errors")
 
 
+@pytest.mark.parametrize("dtype,V", [(torch.float32, 4096), (torch.bfloat16, 32000), (torch.float32, 1001),
+                                     (torch.bfloat16, 20011)])
+def test_zero_mass_residual_falls_back_to_the_target_row(lib, dtype, V):
+    """Algorithm 6's else-branch when [P - Q]_+ has no mass.  With draft == target nothing is ever
+    rejected, so the stop is forced through bs_residual_sample's accept_len input: the residual at the
+    stop row is exactly zero on both sides, the token must be the one the oracle draws from the stop
+    row's target distribution, and the status word must say that the fallback was taken.  Aligned
+    rows take the pipelined kernels, odd V the generic ones."""
+    rng = np.random.default_rng(V + 5)
+    B, G, T = 6, 4, 0.8
+    rnd = _random_round(rng, B, G, V, dtype, T, gamma=[4, 4, 3, 2, 1, 4])
+    rnd.draft = rnd.target[:, :G].clone().contiguous()
+    forced = np.array([0, 3, 1, 1, 0, 4], np.int32)              # the last sequence keeps everything: bonus row
+    dev = rnd.target.device
+    ws = lib.new_workspace(B, G, V, dev)
+    acc = torch.empty(B, dtype=torch.int32, device=dev)
+    p = torch.empty(B, G, device=dev); q = torch.empty(B, G, device=dev)
+    ot = torch.empty(B, G + 1, dtype=torch.int32, device=dev); ol = torch.empty(B, dtype=torch.int32, device=dev)
+    gamma_d = torch.as_tensor(rnd.gamma, device=dev)
+    lib.bs_softmax_verify(rnd.target, rnd.draft, rnd.tokens, gamma_d, torch.as_tensor(rnd.uniforms.u_accept, device=dev),
+                          T, acc, p, q, ws)
+    assert (acc.cpu().numpy() == rnd.gamma).all() and torch.allclose(p, q, atol=1e-6, rtol=0)   # q == p accepts everything
+    lib.bs_residual_sample(rnd.target, rnd.draft, rnd.tokens, gamma_d, torch.as_tensor(forced, device=dev),
+                           torch.as_tensor(rnd.uniforms.u_resample, device=dev), T, ot, ol, ws)
+    st = lib.bs_get_device_status(ws, B, G, V)
+    assert (st[:5] == lib.BS_DEV_RESIDUAL_FALLBACK).all() and st[5] == 0, st
+    toks = rnd.tokens.cpu().numpy()
+    flagged = 0
+    for b in range(B):
+        t_rows = rnd.target[b].float().cpu().numpy()
+        u = float(rnd.uniforms.u_resample[b])
+        ref = ov.verify_sequence(t_rows, t_rows[:G], toks[b], int(rnd.gamma[b]), rnd.uniforms.u_accept[b], u, T,
+                                 keep_mass=True, forced_tau=int(forced[b]))
+        assert ref.used_fallback == (b < 5) and ref.tau == forced[b]
+        assert int(ol[b]) == forced[b] + 1 and list(ot[b, :forced[b]].cpu().numpy()) == list(toks[b, :forced[b]])
+        tok = int(ot[b, forced[b]])
+        if tok != ref.token:                                     # only at an edge of the token's interval
+            c = np.cumsum(ref.mass) / ref.mass.sum()
+            lo, hi = (c[tok - 1] if tok > 0 else 0.0), c[tok]
+            assert min(u - ref.cdf_lo, ref.cdf_hi - u) < ov.CDF_TIE and ref.mass[tok] > 0
+            assert lo <= u + ov.CDF_TIE and hi >= u - ov.CDF_TIE
+            flagged += 1
+    assert flagged <= 1
+
+
 def test_same_inputs_twice_are_bit_identical(lib):
     rng = np.random.default_rng(13)
     rnd = _random_round(rng, 16, 5, 32000, torch.bfloat16, 0.7)
@@ -175,6 +220,62 @@ def test_bandit_trajectories_match_the_oracle(lib, alg_name):
     else:
         assert np.allclose(st["S"], ref.S, rtol=1e-10)
     assert flagged_total <= 2
+
+
+def test_exp3spec_thousand_rounds_without_restart(lib):
+    """Algorithm 9 over the 1000 rounds of the 4-armed adversarial workload (256 sequences, arms
+    gamma = 1, 3, 5, 8, the arms' acceptance rates rotating every 200 rounds) with NO re-synchronisation
+    of the cumulative loss estimates: the oracle keeps its own S throughout and is only told which arm
+    the device played.  Both sides are fp64; their exp() routines differ in the last bit and the
+    difference compounds (a difference d in S_i moves the next estimate by eta * d relative), so S
+    drifts apart -- measured here, bounded below.  What the drift may change is an arm choice whose
+    uniform falls between the two sides' CDF edges; every differing choice must be exactly that, and
+    the two probability vectors must differ by no more than the drift in S explains."""
+    rng = np.random.default_rng(4)
+    B, arm_gamma, rounds = 256, (1, 3, 5, 8), 1000
+    K, L = len(arm_gamma), max(arm_gamma)
+    rate = np.array([0.85, 0.65, 0.45, 0.2])                     # acceptance rate of the draft qualities 0.3 .. 3.0
+    state = lib.new_bandit(lib.BS_EXP3, B, arm_gamma, 0.5, DEV)
+    ref = ob.EXP3Spec(B, arm_gamma)
+    arm_d = torch.empty(B, dtype=torch.int32, device=DEV); gam_d = torch.empty_like(arm_d)
+    p_d = torch.empty(B, K, dtype=torch.float64, device=DEV)
+    differ, between, worst_p, drift = 0, 0, 0.0, 0.0
+    for t in range(1, rounds + 1):
+        u = wl.round_uniforms(4, t, B, L).u_arm
+        lib.bs_bandit_select(state, lib.BS_EXP3, B, K, torch.as_tensor(u, device=DEV), None, arm_d, gam_d, p_d)
+        arm = arm_d.cpu().numpy().astype(np.int64)
+        p_gpu = p_d.cpu().numpy()
+        a_ref, _, _ = ref.select(u)
+        p_ref = ref.last_p
+        # first order: dp_i = -eta p_i (dS_i - sum_j p_j dS_j), so |dp| <= 2 eta max|dS|
+        eta = ref.learning_rate(t)
+        S_gpu = lib.bs_bandit_read(state, lib.BS_EXP3, B, K)["S"]
+        dS = np.abs(S_gpu - ref.S).max(axis=1)
+        dp = np.abs(p_gpu - p_ref).max(axis=1)
+        assert (dp <= 2.5 * eta * dS + 1e-14).all(), (t, float(dp.max()), float(dS.max()))
+        worst_p = max(worst_p, float(dp.max()))
+        c_gpu, c_ref = np.cumsum(p_gpu, axis=1), np.cumsum(p_ref, axis=1)
+        for b in np.nonzero(arm != a_ref)[0]:
+            differ += 1
+            i = min(arm[b], a_ref[b])                            # the edge the two sides put on opposite sides of u
+            assert abs(int(arm[b]) - int(a_ref[b])) == 1, (t, b)
+            lo, hi = min(c_gpu[b, i], c_ref[b, i]), max(c_gpu[b, i], c_ref[b, i])
+            assert lo - 1e-9 <= u[b] <= hi + 1e-9, (t, b, lo, float(u[b]), hi)
+            between += 1
+            ref.p_sel[b] = p_ref[b][arm[b]]                      # the oracle plays the device's arm with its own p
+        phase = (t - 1) // 200
+        alpha = rate[(arm + phase) % 4]
+        passes = rng.random((B, L)) < alpha[:, None]
+        run = np.where(passes.all(axis=1), L, np.argmin(passes, axis=1))
+        y = (1 + np.minimum(run, np.asarray(arm_gamma)[arm])).astype(np.int32)
+        lib.bs_bandit_update(state, lib.BS_EXP3, B, K, arm_d, torch.as_tensor(y, device=DEV))
+        ref.update(arm, y)
+    S_gpu = lib.bs_bandit_read(state, lib.BS_EXP3, B, K)["S"]
+    drift = float((np.abs(S_gpu - ref.S) / np.maximum(np.abs(ref.S), 1e-12)).max())
+    print(f"EXP3Spec, {rounds} rounds x {B} sequences without restart: {differ} of {rounds * B} arm choices differ, "
+          f"all {between} with the uniform between the two CDF edges; largest |dp| {worst_p:.2e}, "
+          f"final relative drift of S {drift:.2e}")
+    assert differ == between and differ <= 40 and drift < 1e-4
 
 
 def test_bandit_golden_tables_on_device(lib):

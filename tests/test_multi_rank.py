@@ -60,3 +60,25 @@ def test_two_gloo_ranks_shard_sequences_without_data_collectives():
         p.join(timeout=180)
         assert p.exitcode == 0
     assert out.get(timeout=5) == "ok"
+
+
+def test_bench_gpus_flag_starts_that_many_ranks():
+    """`bench.py --gpus 2` with no launcher around it must itself start two ranks.  The reference arm
+    needs no GPU: rank 0 times the oracle and prints the line with n_gpus = 2, rank 1 exits idle."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "reference",
+                          "--workload", "tiny_ucb", "--steps", "2", "--warmup", "1", "--cpu-seconds", "0.3"],
+                         capture_output=True, text=True, timeout=300, cwd=ROOT, env=env)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [ln for ln in res.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1                                        # rank 0 alone prints
+    d = json.loads(lines[0])
+    assert d["impl"] == "reference" and d["n_gpus"] == 2 and d["value"] > 0
+    assert "rank 0 of 2" in res.stderr and "rank 1 of 2" in res.stderr
+    # a launcher that started a different number of ranks than --gpus says is an error, not a silent 1-GPU run
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "4", "--impl", "reference",
+                          "--workload", "tiny_ucb"], capture_output=True, text=True, timeout=120, cwd=ROOT,
+                         env=dict(env, WORLD_SIZE="1", RANK="0"))
+    assert res.returncode != 0 and "--gpus 4" in res.stderr

@@ -206,6 +206,38 @@ def test_bonus_and_residual_use_the_right_rows():
     assert r.tau == 0 and r.y == 1 and r.token == 0
 
 
+def test_residual_without_mass_falls_back_to_the_target_row():
+    """Norm([P - Q]_+) needs a positive total (notation paragraph before Algorithm 6).  With identical
+    models the accept test cannot reject, so the stop is forced: the residual at the stop row is then
+    exactly zero, the step samples from that row's target distribution instead and says so."""
+    rng = np.random.default_rng(31)
+    for trial in range(100):
+        V = int(rng.integers(2, 30))
+        gamma = int(rng.integers(1, 5))
+        tl = rng.normal(0, 2, size=(gamma + 1, V))
+        toks = rng.integers(0, V, size=gamma)
+        stop = int(rng.integers(0, gamma))
+        u = rng.random()
+        T = float(rng.choice([0.5, 1.0, 2.0]))
+        r = ov.verify_sequence(tl, tl[:gamma].copy(), toks, gamma, rng.random(gamma), u, T, forced_tau=stop)
+        assert r.used_fallback and r.tau == stop and r.y == stop + 1
+        # the token of the stop row's own distribution for this uniform, by a written-out loop
+        P = np.exp(tl[stop] / T - (tl[stop] / T).max())
+        P /= P.sum()
+        run, want = 0.0, None
+        for v in range(V):
+            run += P[v]
+            if run > u * P.sum():
+                want = v
+                break
+        assert r.token == want and r.out_tokens == list(toks[:stop]) + [want]
+        # not the bonus row's token law: the rows differ, so the intervals do
+        assert r.cdf_lo <= u < r.cdf_hi and abs((r.cdf_hi - r.cdf_lo) - P[want]) < 1e-12
+    # a residual with mass anywhere never takes that branch
+    r = ov.verify_sequence(np.array([[1.0, 0.0], [0.0, 0.0]]), np.array([[0.0, 1.0]]), [1], 1, [0.99], 0.5, 1.0)
+    assert not r.used_fallback and r.tau == 0 and r.token == 0
+
+
 def test_greedy_against_brute_force_with_ties():
     rng = np.random.default_rng(21)
     for trial in range(300):

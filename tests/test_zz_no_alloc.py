@@ -60,6 +60,37 @@ def test_noalloc_matches_workspace_variant_twice(lib, dtype, V):
     assert torch.equal(got[0], want[0]) and torch.equal(got[0].cpu(), gamma.cpu())
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_noalloc_matches_the_oracle(lib, dtype):
+    """The entry point by itself against the CPU checker (Algorithm 6's accept loop): accepted lengths
+    exact except at flagged near-ties of the accept test, token probabilities within 1e-5.  One
+    sequence carries a token outside the vocabulary: that position counts as rejected, as the header
+    says, although no status word can be read back from the built-in scratch."""
+    from oracle import verify as ov
+    B, G, V, T = 9, 4, 32000, 0.9
+    t, d, tok, gamma, u = _inputs(31 + (dtype == torch.bfloat16), B, G, V, dtype)
+    gamma = torch.full_like(gamma, G)
+    tok[4, 1] = V + 3
+    acc, p, q = _run(lib.bs_softmax_verify_noalloc, t, d, tok, gamma, u, T)
+    flagged = 0
+    for b in range(B):
+        toks = tok[b].cpu().numpy().copy()
+        cut = G
+        if b == 4:
+            toks[1], cut = 0, 1                                  # the oracle sees valid positions only
+        ref = ov.verify_sequence(t[b].float().cpu().numpy(), d[b].float().cpu().numpy(), toks, cut,
+                                 u[b].cpu().numpy(), 0.5, T)
+        got = int(acc[b])
+        if got != ref.tau:
+            j = min(got, ref.tau)
+            assert abs(ref.accept_margin[j]) < ov.ACCEPT_TIE, (b, got, ref.tau)
+            flagged += 1
+        assert got <= cut
+        assert np.abs(p[b, :cut].cpu().numpy() - ref.p_tok).max() <= 1e-5
+        assert np.abs(q[b, :cut].cpu().numpy() - ref.q_tok).max() <= 1e-5
+    assert flagged <= 1
+
+
 def test_noalloc_rejects_sizes_beyond_its_scratch(lib):
     B, G, V = 512, 8, 152064
     assert lib.bs_workspace_bytes(B, G, V) > lib.BS_NOALLOC_SCRATCH_BYTES
