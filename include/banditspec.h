@@ -16,12 +16,7 @@
  *
  * Conventions that hold for every entry point
  *  - Every array pointer is a DEVICE pointer owned by the caller unless the comment says
- *    "host".  The library allocates no device memory.  Its only process-wide state is a set of
- *    per-device values looked up on first use and never changed afterwards (the opt-in shared
- *    memory limit, kernel attributes, resident-CTA counts, the device address of the built-in
- *    scratch array of bs_softmax_verify_noalloc) and that scratch array itself; the look-ups are
- *    not locked, so the very first calls on a device should not come from several host threads
- *    at once.
+ *    "host".  The library allocates no device memory and keeps no global state.
  *  - `stream` is a cudaStream_t passed as void*.  Calls are asynchronous on that stream,
  *    never synchronise, and may be captured in a CUDA graph.
  *  - The return value covers host-side argument checks and launch errors only.  Problems
@@ -90,14 +85,6 @@ size_t bs_workspace_bytes(int B, int Gmax, int V);
 /* Clears the workspace (arrival counters must start at zero; the kernels leave them at zero
  * again after every call).  Call once after allocating, 256-byte aligned. */
 bs_status bs_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
-
-/* The byte range [*offset, *offset + *bytes) of a workspace that holds book-keeping whose VALUES depend
- * on the launch and on timing -- the counters through which the statistics kernel hands its work out,
- * a launch counter, and per-sequence words saying which of the residual masses that kernel computed
- * itself.  Everything outside the range (arrival counters, status words, row statistics, segment
- * partials, piece masses) is a function of the inputs alone, so two runs on the same inputs can be
- * compared byte for byte outside it.  Host pointers; BS_ERR_INVALID_ARG for sizes outside the limits. */
-bs_status bs_workspace_bookkeeping_range(int B, int Gmax, int V, size_t* offset, size_t* bytes);
 
 /* Copies the per-sequence status words of the LAST verify/residual call to host memory.
  * Synchronises the stream.  host_status: host array [B].  Returns BS_ERR_DEVICE_DATA if any
@@ -172,13 +159,7 @@ bs_status bs_residual_sample(const void* target_logits, const void* draft_logits
  *    every call.  Calls that overlap on the same GPU (different streams, different threads) race
  *    on it and give wrong results: serialise them.
  *  - The row statistics stay inside the library, so bs_residual_sample cannot follow this call;
- *    it serves callers that need accept_len and the token probabilities only.
- *  - The per-sequence status words and the abort word live in the array too, and
- *    bs_get_device_status cannot be pointed at it: device-detected data problems are handled as
- *    in bs_softmax_verify (an out-of-range token counts as rejected, an out-of-range gamma as
- *    gamma = 0, nothing traps) but are not reported, and a pipeline wait that gave up leaves
- *    accept_len / p_tok / q_tok of the unfinished sequences unwritten without a way to learn of
- *    it.  Callers that need the report use bs_softmax_verify with a workspace. */
+ *    it serves callers that need accept_len and the token probabilities only. */
 #define BS_NOALLOC_SCRATCH_BYTES (2 << 20)
 bs_status bs_softmax_verify_noalloc(const void* target_logits, const void* draft_logits, bs_dtype dtype,
                                     const int32_t* draft_tokens, const int32_t* gamma, const float* u_accept,

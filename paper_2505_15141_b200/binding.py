@@ -37,7 +37,6 @@ SIGNATURES = {
     "bs_last_cuda_error": (C.c_char_p, []),
     "bs_workspace_bytes": (_sz, [_i, _i, _i]),
     "bs_workspace_init": (_i, [_vp, _sz, _vp]),
-    "bs_workspace_bookkeeping_range": (_i, [_i, _i, _i, _vp, _vp]),
     "bs_get_device_status": (_i, [_vp, _sz, _i, _i, _i, _vp, _vp]),
     "bs_softmax_verify": (_i, [_vp, _vp, _i, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bs_residual_sample": (_i, [_vp, _vp, _i, _vp, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _sz, _vp]),
@@ -116,19 +115,6 @@ def new_workspace(B: int, Gmax: int, V: int, device="cuda") -> torch.Tensor:
     ws = torch.empty(n, dtype=torch.uint8, device=device)
     bs_workspace_init(ws)
     return ws
-
-
-def bs_workspace_bookkeeping_range(B: int, Gmax: int, V: int):
-    """(offset, bytes) of the part of a workspace whose values depend on the launch and on timing."""
-    off, n = C.c_size_t(0), C.c_size_t(0)
-    _check(_lib.bs_workspace_bookkeeping_range(B, Gmax, V, C.byref(off), C.byref(n)), "bs_workspace_bookkeeping_range")
-    return int(off.value), int(n.value)
-
-
-def workspace_results(workspace: torch.Tensor, B: int, Gmax: int, V: int) -> torch.Tensor:
-    """A copy of the workspace without its book-keeping range: a function of the inputs alone."""
-    off, n = bs_workspace_bookkeeping_range(B, Gmax, V)
-    return torch.cat([workspace[:off], workspace[off + n:]])
 
 
 def bs_get_device_status(workspace: torch.Tensor, B: int, Gmax: int, V: int, stream=None) -> np.ndarray:

@@ -29,38 +29,20 @@ __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a -
 //   ticket_verify [B] u32     per-sequence arrival counters of the statistics kernel (zero between calls)
 //   ticket_resid  [B] u32     per-sequence arrival counters of the resampling kernel (zero between calls)
 //   ticket_row    [B, R] u32  first B words: bit j set = the statistics of draft row j were left by a
-//                             drafting call (bs_draft_sample) and not yet consumed, bit 31 = a drafting
-//                             pass met a row without a finite normaliser; second B words: decision
+//                             drafting call (bs_draft_sample) and not yet consumed; second B words: decision
 //                             words of bs_verify_walk (zero between calls); rest unused
 //   status        [B] i32     device-data status bits of the last call pair
 //   abort         [1] i32     set when a bounded pipeline wait gave up (reported as BS_ERR_TIMEOUT)
-//   sched         [64] u32    work hand-out of the pipelined statistics kernel, see kSched*
-//   mass_tau      [B] u32     (tag << 8) | (tau + 1): the statistics call `tag` found tau accepted drafts for
-//                             the sequence and the residual masses of that stop row may be taken from
-//                             resid_partial once mass_done says they are complete
-//   mass_done     [B] u32     (tag << 8) | number of mass chunks of the sequence that are written
 //   row_stats     [B, R, 2] f32, R = 2*Gmax+1: (raw max logit, Z) per row; greedy: (max, arg-max bits)
 //                 rows 0..Gmax are target rows, rows Gmax+1..2*Gmax are draft rows
 //   partial       [B, R, S, 2] f32, S = ceil(V / 8192): per-segment (max, Z) / (max, arg-max)
 //   resid_partial [B, Sr] f32, Sr = 16 * ceil(V / 4096): residual mass of every 1 KB piece of a row pair
 //                 (the generic kernel uses one entry per 16 KB segment)
 struct Workspace {
-    size_t off_ticket_verify, off_ticket_resid, off_ticket_row, off_status, off_abort, off_sched, off_mass_tau,
-        off_mass_done, off_row_stats, off_partial, off_resid_partial, total;
+    size_t off_ticket_verify, off_ticket_resid, off_ticket_row, off_status, off_abort, off_row_stats, off_partial,
+        off_resid_partial, total;
     int R, S, Sr;
 };
-
-// Words of the `sched` region.  The first three are zero between launches of the pipelined statistics
-// kernel (its last CTA to leave clears them); the epoch only ever grows.
-//   cursor     chunks of the item list handed out beyond the one every CTA starts with
-//   mass_head  mass chunks handed out: chunk h belongs to sequence h / C, part h % C
-//   exit       CTAs that have left
-//   epoch      bumped by every launch that writes row statistics or piece masses.  A pipelined statistics
-//              launch that starts at epoch E tags the mass words it writes with epoch_tag(E) and leaves
-//              E + 1 behind, so the resampling call that follows accepts exactly the words tagged
-//              epoch_tag(epoch - 1); any other launch in between bumps the epoch and thereby voids them.
-constexpr int kSchedCursor = 0, kSchedMassHead = 1, kSchedExit = 2, kSchedEpoch = 3, kSchedWords = 64;
-__host__ __device__ inline uint32_t epoch_tag(uint32_t epoch) { return epoch % 0xffffffu + 1u; }   // 1 .. 2^24 - 1
 
 __host__ __device__ inline Workspace workspace_layout(int B, int Gmax, int V) {
     Workspace w;
@@ -73,20 +55,12 @@ __host__ __device__ inline Workspace workspace_layout(int B, int Gmax, int V) {
     w.off_ticket_row = o;    o = align_up(o + sizeof(uint32_t) * (size_t)B * (w.R < 2 ? 2 : w.R), 256);
     w.off_status = o;        o = align_up(o + sizeof(int32_t) * (size_t)B, 256);
     w.off_abort = o;         o = align_up(o + sizeof(int32_t), 256);
-    w.off_sched = o;         o = align_up(o + sizeof(uint32_t) * kSchedWords, 256);
-    w.off_mass_tau = o;      o = align_up(o + sizeof(uint32_t) * (size_t)B, 256);
-    w.off_mass_done = o;     o = align_up(o + sizeof(uint32_t) * (size_t)B, 256);
     w.off_row_stats = o;     o = align_up(o + sizeof(float) * 2 * (size_t)B * w.R, 256);
     w.off_partial = o;       o = align_up(o + sizeof(float) * 2 * (size_t)B * w.R * w.S, 256);
     w.off_resid_partial = o; o = align_up(o + sizeof(float) * (size_t)B * w.Sr, 256);
     w.total = o;
     return w;
 }
-
-// Any kernel other than the pipelined statistics kernel that writes row statistics or piece masses
-// calls this once (one thread of the grid): mass words left by an earlier statistics call no longer
-// describe the workspace.
-__device__ __forceinline__ void void_mass_words(uint32_t* sched) { atomicAdd(sched + kSchedEpoch, 1u); }
 
 // ---- small device helpers -----------------------------------------------------------
 

@@ -422,7 +422,6 @@ __global__ void __launch_bounds__(kThreads) lmhead_finalize_kernel(const VerifyP
                                                                    const int NT) {
     __shared__ float2 s_w[kWarps];
     pdl_enter();
-    if (blockIdx.x == 0 && threadIdx.x == 0) void_mass_words(p.sched);   // new row statistics: older mass words are void
     const int b = blockIdx.x / p.R, lr = blockIdx.x - b * p.R;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = clamp_gamma(p.gamma[b], p.Gmax);
@@ -637,7 +636,6 @@ extern "C" bs_status bs_lmhead_verify(const void* H_t, const void* W_t, int d_t,
     vp.seg = seg_elems(BS_F32); vp.nseg = div_up(V, vp.seg);
     vp.c = lp.c;
     vp.mode = kModeVerify; vp.position = 0; vp.draft_ready = vp.ticket_row; vp.draft_out = nullptr;
-    set_mass_fields(vp, ws, w, BS_F32);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (mh == 1)
         return greedy ? launch_lmhead<1, 4, true>(tms, lp, vp, partial, st)

@@ -139,7 +139,6 @@ __global__ void __launch_bounds__(kThreads, 2) residual_kernel(const ResidParams
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     pdl_enter();
-    if (blockIdx.x == 0 && tid == 0) void_mass_words(p.sched);       // this launch overwrites piece masses
     // CTA (b, part) owns a contiguous range of the segments of sequence b
     {
         const int b = blockIdx.x / nsplit, part = blockIdx.x - b * nsplit;
@@ -188,7 +187,7 @@ __global__ void __launch_bounds__(kThreads, 2) residual_kernel(const ResidParams
             s_mass[tid] = tid < p.nseg ? __ldcg(p.resid_partial + (size_t)b * p.S + tid) : 0.f;
             double excl, Rtot;
             double incl = block_scan((double)s_mass[tid], s_w, excl, Rtot);
-            if (!(Rtot > (f.bonus ? 0.0 : kResidualFloor)) || !isfinite(Rtot)) {
+            if (!(Rtot > 0.0) || !isfinite(Rtot)) {
                 // [P - Q]_+ has no mass (P == Q up to rounding) or the row is not finite:
                 // fall back to the target distribution of the same row
                 bits |= f.bonus ? BS_DEV_NONFINITE : BS_DEV_RESIDUAL_FALLBACK;
@@ -323,7 +322,6 @@ extern "C" bs_status bs_residual_sample(const void* target_logits, const void* d
     p.nseg = div_up(V, p.seg);
     p.c = greedy ? 1.f : kLog2e / temperature;
     p.mode = kResidVerify; p.position = 0; p.draft_out = nullptr;
-    set_mass_fields(p, ws, w);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (greedy) {
         return cuda_status(launch_pdl(greedy_emit_kernel, div_up(B, 128), 128, 0, st, p));
@@ -358,7 +356,6 @@ bs_status bs::run_draft_resample(const void* draft_logits, bs_dtype dtype, int p
     p.nseg = div_up(V, p.seg);
     p.c = kLog2e / temperature;
     p.mode = kResidDraft; p.position = position; p.draft_out = draft_tokens;
-    set_mass_fields(p, ws, w);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     return dtype == BS_F32 ? launch_residual_stream<float>(p, st) : launch_residual_stream<__nv_bfloat16>(p, st);
 }

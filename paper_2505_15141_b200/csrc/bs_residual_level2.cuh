@@ -28,24 +28,14 @@ struct RsMeta {
     float at, ad;
 };
 
-// Mass chunks of a sequence: the items of its stop row (pair) are handed out in this many contiguous
-// parts when the statistics kernel computes the piece masses itself.
-__host__ __device__ inline int mass_chunks(int rnseg) {
-    const int c = (rnseg + 1) >> 1;                          // never more parts than the shorter item list has items
-    return c > 8 ? 8 : (c < 1 ? 1 : c);
-}
-
 // Per-sequence facts every role derives the same way.
 struct RsSeq {
     int tau, bonus, wgt;     // weight of one item: 2 (row pair) or 1 (target row only)
-    int done;                // the piece masses of this stop row are already in resid_partial
 };
-// tag: epoch_tag of the statistics call whose mass words are acceptable, 0 = none.
-__device__ __forceinline__ RsSeq rs_seq(const ResidParams& p, int b, uint32_t tag = 0u) {
+__device__ __forceinline__ RsSeq rs_seq(const ResidParams& p, int b) {
     int g = p.gamma[b];
     if (g < 0 || g > p.Gmax) g = 0;
     RsSeq s;
-    s.done = 0;
     if (p.mode == kResidDraft) {          // drafting: sample from the draft row `position` alone, if the sequence drafts it
         s.tau = p.position;
         s.bonus = 1;
@@ -55,9 +45,6 @@ __device__ __forceinline__ RsSeq rs_seq(const ResidParams& p, int b, uint32_t ta
     s.tau = max(0, min(p.accept_len[b], g));
     s.bonus = s.tau >= g;
     s.wgt = s.bonus ? 1 : 2;
-    if (tag)
-        s.done = __ldcg(p.mass_tau + b) == ((tag << 8) | (uint32_t)(s.tau + 1)) &&
-                 __ldcg(p.mass_done + b) == ((tag << 8) | (uint32_t)mass_chunks(p.nseg));
     return s;
 }
 // Items of a sequence in the pipelined kernel.  A slot has two 16 KB halves: for a row pair they hold
@@ -65,10 +52,8 @@ __device__ __forceinline__ RsSeq rs_seq(const ResidParams& p, int b, uint32_t ta
 // segments of it, so that every item keeps up to 32 KB in flight (with one segment per item the
 // CTAs whose sequences were all accepted moved half the bytes per item and finished last).
 __device__ __forceinline__ int rs_nitems(const RsSeq& s, int nseg) {
-    return (s.wgt <= 0 || s.done) ? 0 : (s.bonus ? (nseg + 1) >> 1 : nseg);
+    return s.wgt <= 0 ? 0 : (s.bonus ? (nseg + 1) >> 1 : nseg);
 }
-// The same for a stop row whose masses are still to be computed, whoever computes them.
-__device__ __forceinline__ int rs_row_items(int bonus, int nseg) { return bonus ? (nseg + 1) >> 1 : nseg; }
 __device__ __forceinline__ int rs_first_seg(const RsSeq& s, int item) { return s.bonus ? 2 * item : item; }
 // Items [i0, i1) of a sequence with `nitems` items that lie in the CTA's range [lo, hi); pre = index of its first item.
 __device__ __forceinline__ void rs_items(int pre, int nitems, int lo, int hi, int& i0, int& i1) {
@@ -136,7 +121,7 @@ __device__ void rs_level2(const ResidParams& p, int b, const RsSeq sq, MassFn f)
     const float u = p.mode == kResidDraft ? p.u_resample[(size_t)b * p.Gmax + p.position] : p.u_resample[b];
     int tok = -1;
 
-    if (Rtot > (f.bonus ? 0.0 : kResidualFloor) && isfinite(Rtot)) {
+    if (Rtot > 0.0 && isfinite(Rtot)) {
         const double target = (double)u * Rtot;
         double excl = __shfl_up_sync(0xffffffffu, incl, 1);
         if (lane == 0) excl = 0.0;
@@ -303,9 +288,7 @@ __device__ void rs_level2(const ResidParams& p, int b, const RsSeq sq, MassFn f)
     if (p.mode == kResidDraft) {                              // drafting: the token is the whole output
         if (lane == 0) {
             p.draft_out[(size_t)b * p.Gmax + p.position] = tok;
-            // the status word belongs to the verification call that follows (it assigns it): what the
-            // drafting pass found travels in the spare bit of the word of drafted positions
-            if (bits) atomicOr(p.draft_ready + b, 0x80000000u);
+            if (bits) atomicOr(p.status + b, bits);
             p.ticket[b] = 0u;
         }
         return;

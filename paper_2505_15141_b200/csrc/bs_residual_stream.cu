@@ -20,12 +20,6 @@
 //                       u * R, the piece (2 x 1 KB, an L2 hit) is read again, scanned in fp64 and
 //                       the crossing element is the token.  The same r_v feed both levels.
 //
-// The statistics call that came before may have computed the piece masses of a sequence's stop row
-// itself (while the row pair was still in L2); its words in the workspace say for which stop row and
-// whether all of them are written.  Such a sequence contributes no items here: a warp runs its level 2
-// straight away.  A sequence whose words do not match (another accept_len was passed in, the masses were
-// left unfinished, the rows are not the pipelined kernel's) is streamed as before.
-//
 // Every wait (mbarriers, the finisher's poll of the consumers' progress) is bounded; a wait that
 // gives up sets the abort word and the thread leaves.
 #include "bs_residual_level2.cuh"
@@ -60,10 +54,6 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
 
     pdl_enter();                                              // accept_len and the row statistics come from the kernel before
 
-    // mass words of the statistics call that bumped the epoch last are the ones that count
-    const uint32_t tag = p.mode == kResidVerify ? epoch_tag(__ldcg(p.sched + kSchedEpoch) - 1u) : 0u;
-    if (p.mode == kResidDraft && blockIdx.x == 0 && tid == 0) void_mass_words(p.sched);   // this launch overwrites piece masses
-
     // ---- prefix sum of item counts over the batch (all threads, redundantly per CTA) ----
     {
         const int per = div_up(p.B, kRsThreads);
@@ -71,7 +61,7 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
         int local = 0;
         for (int k = 0; k < per; ++k) {
             const int b = b0 + k;
-            if (b < p.B) local += rs_nitems(rs_seq(p, b, tag), p.nseg);
+            if (b < p.B) local += rs_nitems(rs_seq(p, b), p.nseg);
         }
         int incl = local;
 #pragma unroll
@@ -88,7 +78,7 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
             const int b = b0 + k;
             if (b < p.B) {
                 s_prefix[b] = run;
-                run += rs_nitems(rs_seq(p, b, tag), p.nseg);
+                run += rs_nitems(rs_seq(p, b), p.nseg);
             }
         }
         if (tid == kRsThreads - 1) s_prefix[p.B] = run;
@@ -114,30 +104,6 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
         blast = l;
     }
     const int count = hi - lo;                                // items of this CTA: the list has unit weights
-
-    // ---- sequences whose piece masses are in place: level 2 at once ----
-    // Sequence b goes to CTA b % grid; the finisher warp takes the CTA's first one, consumer warps
-    // (from the last one down) any further ones, so that up to 296 sequences cost no consumer any time.
-    if (tag && warp != kRsWarps) {
-        const int helper = warp == kRsWarps + 1 ? 0 : kRsWarps - warp;       // 0, then 1 .. 16
-        const long long bl = (long long)helper * gridDim.x + blockIdx.x;
-        for (long long bb = bl; bb < p.B; bb += 17LL * gridDim.x) {
-            const int b = (int)bb;
-            const RsSeq sq = rs_seq(p, b, tag);
-            if (!sq.done) continue;
-            MassFn f;
-            f.c = p.c;
-            f.bonus = sq.bonus;
-            const float2 ts = p.row_stats[(size_t)b * p.R + sq.tau];
-            MassFn::fold(ts.x, ts.y, p.c, f.kt, f.at);
-            f.kd = 0.f; f.ad = 1.f;
-            if (!sq.bonus) {
-                const float2 ds = p.row_stats[(size_t)b * p.R + p.Gmax + 1 + sq.tau];
-                MassFn::fold(ds.x, ds.y, p.c, f.kd, f.ad);
-            }
-            rs_level2<T>(p, b, sq, f);
-        }
-    }
     if (count <= 0) return;
 
     if (warp == kRsWarps) {
@@ -146,7 +112,7 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
         int slot = 0;
         uint32_t ph = 0;
         for (int b = bfirst; b <= blast; ++b) {
-            const RsSeq sq = rs_seq(p, b, tag);
+            const RsSeq sq = rs_seq(p, b);
             int i0, i1;
             rs_items(s_prefix[b], rs_nitems(sq, p.nseg), lo, hi, i0, i1);
             if (i1 <= i0) continue;
@@ -189,7 +155,7 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
         // =============================== finisher ===============================
         unsigned shares = 0;                                  // sequence shares of this CTA seen so far
         for (int b = bfirst; b <= blast; ++b) {
-            const RsSeq sq = rs_seq(p, b, tag);
+            const RsSeq sq = rs_seq(p, b);
             int i0, i1;
             rs_items(s_prefix[b], rs_nitems(sq, p.nseg), lo, hi, i0, i1);
             if (i1 <= i0) continue;
@@ -226,9 +192,6 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
                     const float2 ds = p.row_stats[(size_t)b * p.R + p.Gmax + 1 + sq.tau];
                     MassFn::fold(ds.x, ds.y, p.c, f.kd, f.ad);
                 }
-                // the masses in the workspace are now those of this call's stop row: words left by the
-                // statistics call for another stop row (or an unfinished set) no longer describe them
-                if (p.mode == kResidVerify && lane == 0) p.mass_tau[b] = 0u;
                 rs_level2<T>(p, b, sq, f);
             }
         }

@@ -27,7 +27,6 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const VerifyParams p) 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int kVec = Elem<T>::kVec;
     pdl_enter();
-    if (blockIdx.x == 0 && tid == 0) void_mass_words(p.sched);       // new row statistics: older mass words are void
 
     // ---- prefix sum of work items over the batch (every CTA, redundantly) ----
     {
@@ -233,14 +232,6 @@ extern "C" bs_status bs_workspace_init(void* workspace, size_t workspace_bytes, 
     return cuda_status(cudaMemsetAsync(workspace, 0, workspace_bytes, static_cast<cudaStream_t>(stream)));
 }
 
-extern "C" bs_status bs_workspace_bookkeeping_range(int B, int Gmax, int V, size_t* offset, size_t* bytes) {
-    if (!offset || !bytes || !sizes_ok(B, Gmax, V)) return BS_ERR_INVALID_ARG;
-    const Workspace w = workspace_layout(B, Gmax, V);
-    *offset = w.off_sched;
-    *bytes = w.off_row_stats - w.off_sched;                  // sched, mass_tau, mass_done
-    return BS_OK;
-}
-
 extern "C" bs_status bs_get_device_status(const void* workspace, size_t workspace_bytes, int B, int Gmax, int V,
                                           int32_t* host_status, void* stream) {
     if (!workspace || !host_status || !sizes_ok(B, Gmax, V)) return BS_ERR_INVALID_ARG;
@@ -303,7 +294,6 @@ bs_status bs::run_verify(const void* target_logits, const void* draft_logits, bs
     p.c = greedy ? 1.f : kLog2e / temperature;
     p.mode = mode; p.position = position; p.draft_out = draft_out;
     p.draft_ready = p.ticket_row;          // the per-row counters' slot: the pipelined kernel counts per sequence
-    set_mass_fields(p, ws, w, dtype);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // rows start on 16-byte boundaries: bulk-copy pipeline; otherwise the generic kernel
     const bool aligned = ((size_t)V * es) % 16 == 0 && (reinterpret_cast<uintptr_t>(target_logits) & 15) == 0 &&

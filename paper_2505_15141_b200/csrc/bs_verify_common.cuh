@@ -35,12 +35,6 @@ struct VerifyParams {
     int mode, position;
     uint32_t* draft_ready;   // [B] bit j set: the statistics of draft row j are in row_stats
     int32_t* draft_out;      // kModeDraft, greedy: [B, Gmax] drafted tokens (entry [b, position] written)
-    // Hand-out of work and the residual masses the pipelined kernel leaves for bs_residual_sample:
-    uint32_t* sched;         // [kSchedWords]
-    uint32_t* mass_tau;      // [B]
-    uint32_t* mass_done;     // [B]
-    float* resid_partial;    // [B, Sr] piece masses of the stop row (pair)
-    int Sr, rseg, rnseg;     // resampling geometry: entries per sequence, elements per 16 KB segment, segments per row
 };
 constexpr int kModeVerify = 0, kModeDraft = 1, kModeDrafted = 2;
 
@@ -236,11 +230,10 @@ __device__ __forceinline__ AcceptLoads accept_prefetch(const VerifyParams& p, in
 }
 
 // accept_finish: stats(r) returns the (max, Z) / (max, arg-max) pair of row slot r.  Writes
-// accept_len, p_tok, q_tok and the status word and returns tau.  graw = gamma[b] as read,
-// g = clamp_gamma(graw).
+// accept_len, p_tok, q_tok and the status word.  graw = gamma[b] as read, g = clamp_gamma(graw).
 template <typename T, bool GREEDY, typename StatsFn>
-__device__ __forceinline__ int accept_finish(const VerifyParams& p, int b, int graw, int g, const AcceptLoads& a,
-                                             StatsFn stats, int extra_bits = 0) {
+__device__ __forceinline__ void accept_finish(const VerifyParams& p, int b, int graw, int g, const AcceptLoads& a,
+                                              StatsFn stats, int extra_bits = 0) {
     const int lane = threadIdx.x & 31;
     const int j = lane;
     const bool valid = j < g;
@@ -287,7 +280,6 @@ __device__ __forceinline__ int accept_finish(const VerifyParams& p, int b, int g
         p.accept_len[b] = tau;
         p.status[b] = st_bits;
     }
-    return tau;                                              // the same in every lane
 }
 
 template <typename T, bool GREEDY, typename StatsFn>
@@ -296,18 +288,6 @@ __device__ __forceinline__ void accept_scan_warp(const VerifyParams& p, int b, S
     const int g = clamp_gamma(graw, p.Gmax);
     const AcceptLoads a = accept_prefetch<T, GREEDY>(p, b, g);
     accept_finish<T, GREEDY>(p, b, graw, g, a, stats);
-}
-
-// The words of the workspace through which the pipelined statistics kernel hands work out and leaves
-// the residual masses (every launcher of a kernel that takes VerifyParams fills them the same way).
-inline void set_mass_fields(VerifyParams& p, char* ws, const Workspace& w, int dtype) {
-    p.sched = reinterpret_cast<uint32_t*>(ws + w.off_sched);
-    p.mass_tau = reinterpret_cast<uint32_t*>(ws + w.off_mass_tau);
-    p.mass_done = reinterpret_cast<uint32_t*>(ws + w.off_mass_done);
-    p.resid_partial = reinterpret_cast<float*>(ws + w.off_resid_partial);
-    p.Sr = w.Sr;
-    p.rseg = res_seg_elems(dtype);
-    p.rnseg = div_up(p.V, p.rseg);
 }
 
 template <typename T, bool GREEDY>

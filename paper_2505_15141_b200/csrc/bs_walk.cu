@@ -101,7 +101,6 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
     }
     __syncthreads();
     pdl_enter();                                              // gamma comes from the kernel before this one
-    if (blockIdx.x == 0 && tid == 0) void_mass_words(v.sched);   // new statistics and masses: older mass words are void
 
     if (warp == kWkWarps) {
         // =============================== producer ===============================
@@ -371,10 +370,8 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                 bool missing = false;                          // drafted mode: position k was never drafted
                 if (p.drafted && k < g) {
                     if (lane == 0) s_fin[1] = __ldcg(v.row_stats + (size_t)b * v.R + v.Gmax + 1 + k);
-                    const unsigned ready = __ldcg(v.draft_ready + b);
-                    missing = ((ready >> k) & 1u) == 0u;
+                    missing = ((__ldcg(v.draft_ready + b) >> k) & 1u) == 0u;
                     if (missing) bits |= BS_DEV_DRAFT_MISSING;
-                    if (ready >> 31) bits |= BS_DEV_NONFINITE;   // a drafting pass could not sample its row
                     __syncwarp();
                 }
                 if (!(ts.y > 0.f) || !isfinite(ts.y) || !isfinite(ts.x)) bits |= BS_DEV_NONFINITE;
@@ -421,7 +418,7 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                 if (old + (unsigned)len != (unsigned)p.r.nseg) continue;
                 __threadfence();
                 RsSeq sq;
-                sq.tau = k; sq.bonus = k >= g; sq.wgt = sq.bonus ? 1 : 2; sq.done = 0;
+                sq.tau = k; sq.bonus = k >= g; sq.wgt = sq.bonus ? 1 : 2;
                 MassFn f;
                 f.c = v.c; f.bonus = sq.bonus != 0;
                 const float2 ts = __ldcg(v.row_stats + (size_t)b * v.R + k);
@@ -625,7 +622,6 @@ static bs_status run_walk(const void* target_logits, const void* draft_logits, b
     v.nseg = div_up(V, v.seg);
     v.c = greedy ? 1.f : kLog2e / temperature;
     v.mode = kModeVerify; v.position = 0; v.draft_ready = v.ticket_row; v.draft_out = nullptr;
-    set_mass_fields(v, ws, w, dtype);
     ResidParams& r = p.r;
     r.target = target_logits; r.draft = draft_logits; r.tokens = draft_tokens; r.gamma = gamma;
     r.accept_len = accept_len; r.u_resample = u_resample; r.out_tokens = out_tokens; r.out_len = out_len;
@@ -639,7 +635,6 @@ static bs_status run_walk(const void* target_logits, const void* draft_logits, b
     r.nseg = div_up(V, r.seg);
     r.c = v.c;
     r.mode = kResidVerify; r.position = 0; r.draft_out = nullptr;
-    set_mass_fields(r, ws, w);
     // decision words: the second B words of the per-row counter slot (the first B mark drafted positions)
     p.dec = v.ticket_row + B;
     p.nG = 1;

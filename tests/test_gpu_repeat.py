@@ -27,9 +27,8 @@ def _inputs(name, round_index):
 def test_two_call_round_repeats_bit_for_bit(lib, name, reps):
     w, rnd, gam, ua, ur = _inputs(name, 61)
     ws = lib.new_workspace(w.B, w.Gmax, w.V, DEV)
-    res = lambda t: lib.workspace_results(t, w.B, w.Gmax, w.V)     # all but the hand-out and launch counters
     ref = lib.verify_round(rnd.target, rnd.draft, rnd.tokens, gam, ua, ur, w.temperature, ws)
-    ref_ws = res(ws)
+    ref_ws = ws.clone()
     flush = torch.empty(48 << 20, dtype=torch.float32, device=DEV)
     bad = torch.zeros((), dtype=torch.int64, device=DEV)
     for i in range(reps):
@@ -37,7 +36,7 @@ def test_two_call_round_repeats_bit_for_bit(lib, name, reps):
             flush.zero_()                                   # vary what the round finds in L2
         o = lib.verify_round(rnd.target, rnd.draft, rnd.tokens, gam, ua, ur, w.temperature, ws)
         # the workspace holds the row statistics, the segment partials and every residual piece mass
-        same = ((res(ws) == ref_ws).all() & (o.accept_len == ref.accept_len).all() & (o.out_tokens == ref.out_tokens).all()
+        same = ((ws == ref_ws).all() & (o.accept_len == ref.accept_len).all() & (o.out_tokens == ref.out_tokens).all()
                 & (o.p_tok == ref.p_tok).all() & (o.q_tok == ref.q_tok).all() & (o.out_len == ref.out_len).all())
         bad += (~same).to(torch.int64)
     assert int(bad) == 0, f"{int(bad)} of {reps} repetitions differ from the first"
@@ -46,14 +45,13 @@ def test_two_call_round_repeats_bit_for_bit(lib, name, reps):
 def test_walk_round_repeats_bit_for_bit(lib):
     w, rnd, gam, ua, ur = _inputs("qwen_exp3", 62)
     ws = lib.new_workspace(w.B, w.Gmax, w.V, DEV)
-    res = lambda t: lib.workspace_results(t, w.B, w.Gmax, w.V)
     ref = lib.verify_round_walk(rnd.target, rnd.draft, rnd.tokens, gam, ua, ur, w.temperature, ws)
-    ref_ws = res(ws)                                        # positions are examined in order: what is written is fixed too
+    ref_ws = ws.clone()                                     # positions are examined in order: what is written is fixed too
     bad = torch.zeros((), dtype=torch.int64, device=DEV)
     reps = 1500
     for i in range(reps):
         o = lib.verify_round_walk(rnd.target, rnd.draft, rnd.tokens, gam, ua, ur, w.temperature, ws)
-        same = ((res(ws) == ref_ws).all() & (o.accept_len == ref.accept_len).all() & (o.out_tokens == ref.out_tokens).all()
+        same = ((ws == ref_ws).all() & (o.accept_len == ref.accept_len).all() & (o.out_tokens == ref.out_tokens).all()
                 & (o.p_tok == ref.p_tok).all() & (o.q_tok == ref.q_tok).all() & (o.out_len == ref.out_len).all())
         bad += (~same).to(torch.int64)
     assert int(bad) == 0, f"{int(bad)} of {reps} repetitions differ from the first"
@@ -82,11 +80,11 @@ def test_lmhead_round_repeats_bit_for_bit(lib, name, reps):
         return lt, ld, acc, p, q, ot, ol
 
     ref = run()
-    ref_ws = lib.workspace_results(ws, B, G, V)
+    ref_ws = ws.clone()
     bad = torch.zeros((), dtype=torch.int64, device=DEV)
     for i in range(reps):
         o = run()
-        same = (lib.workspace_results(ws, B, G, V) == ref_ws).all()
+        same = (ws == ref_ws).all()
         for a, b in zip(o, ref):
             same = same & (a == b).all()
         bad += (~same).to(torch.int64)
@@ -117,12 +115,12 @@ def test_drafted_round_repeats_bit_for_bit(lib):
         return tok, acc, p, q, ot, ol
 
     ref = run()
-    ref_ws = lib.workspace_results(ws, B, G, V)
+    ref_ws = ws.clone()
     bad = torch.zeros((), dtype=torch.int64, device=DEV)
     reps = 300
     for i in range(reps):
         o = run()
-        same = (lib.workspace_results(ws, B, G, V) == ref_ws).all()
+        same = (ws == ref_ws).all()
         for a, b in zip(o, ref):
             same = same & (a == b).all()
         bad += (~same).to(torch.int64)
@@ -139,9 +137,7 @@ def test_two_streams_with_their_own_workspaces_do_not_disturb_each_other(lib):
     refa = lib.verify_round(rnda.target, rnda.draft, rnda.tokens, gama, uaa, ura, wa.temperature, wsa)
     refb = lib.verify_round(rndb.target, rndb.draft, rndb.tokens, gamb, uab, urb, wb.temperature, wsb)
     torch.cuda.synchronize()
-    resa = lambda: lib.workspace_results(wsa, wa.B, wa.Gmax, wa.V)
-    resb = lambda: lib.workspace_results(wsb, wb.B, wb.Gmax, wb.V)
-    ref_wsa, ref_wsb = resa(), resb()
+    ref_wsa, ref_wsb = wsa.clone(), wsb.clone()
     sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
     for i in range(200):
         with torch.cuda.stream(sa):
@@ -152,6 +148,6 @@ def test_two_streams_with_their_own_workspaces_do_not_disturb_each_other(lib):
                 ob = lib.verify_round(rndb.target, rndb.draft, rndb.tokens, gamb, uab, urb, wb.temperature, wsb)
         sa.synchronize(); sb.synchronize()
         assert torch.equal(oa.out_tokens, refa.out_tokens) and torch.equal(oa.accept_len, refa.accept_len)
-        assert torch.equal(oa.p_tok, refa.p_tok) and torch.equal(resa(), ref_wsa), f"iteration {i}: first batch differs"
+        assert torch.equal(oa.p_tok, refa.p_tok) and torch.equal(wsa, ref_wsa), f"iteration {i}: first batch differs"
         assert torch.equal(ob.out_tokens, refb.out_tokens) and torch.equal(ob.accept_len, refb.accept_len)
-        assert torch.equal(ob.p_tok, refb.p_tok) and torch.equal(resb(), ref_wsb), f"iteration {i}: second batch differs"
+        assert torch.equal(ob.p_tok, refb.p_tok) and torch.equal(wsb, ref_wsb), f"iteration {i}: second batch differs"
