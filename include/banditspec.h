@@ -16,7 +16,12 @@
  *
  * Conventions that hold for every entry point
  *  - Every array pointer is a DEVICE pointer owned by the caller unless the comment says
- *    "host".  The library allocates no device memory and keeps no global state.
+ *    "host".  The library allocates no device memory.  Its only process-wide state is a set of
+ *    per-device values looked up on first use and never changed afterwards (the opt-in shared
+ *    memory limit, kernel attributes, resident-CTA counts, the device address of the built-in
+ *    scratch array of bs_softmax_verify_noalloc) and that scratch array itself; the look-ups are
+ *    not locked, so the very first calls on a device should not come from several host threads
+ *    at once.
  *  - `stream` is a cudaStream_t passed as void*.  Calls are asynchronous on that stream,
  *    never synchronise, and may be captured in a CUDA graph.
  *  - The return value covers host-side argument checks and launch errors only.  Problems
@@ -62,6 +67,8 @@ typedef enum { BS_UCB = 0, BS_EXP3 = 1, BS_UCB_REWARD = 2 } bs_alg;
 #define BS_DEV_RESIDUAL_FALLBACK 8 /* [P-Q]_+ had zero mass at the rejected position; sampled from P instead */
 #define BS_DEV_DRAFT_MISSING 16    /* bs_softmax_verify_drafted: a draft row below gamma_b was not produced by
                                       bs_draft_sample on this workspace; every draft of the sequence was rejected */
+#define BS_DEV_BAD_TREE      32    /* bs_tree_verify_greedy: a node's parent is not an earlier node; the node counts as
+                                      hanging under the prompt and never passes */
 
 /* Limits of this implementation. */
 #define BS_MAX_GAMMA   31      /* Gmax <= 31 (one warp scans the accept flags) */
@@ -159,7 +166,13 @@ bs_status bs_residual_sample(const void* target_logits, const void* draft_logits
  *    every call.  Calls that overlap on the same GPU (different streams, different threads) race
  *    on it and give wrong results: serialise them.
  *  - The row statistics stay inside the library, so bs_residual_sample cannot follow this call;
- *    it serves callers that need accept_len and the token probabilities only. */
+ *    it serves callers that need accept_len and the token probabilities only.
+ *  - The per-sequence status words and the abort word live in the array too, and
+ *    bs_get_device_status cannot be pointed at it: device-detected data problems are handled as
+ *    in bs_softmax_verify (an out-of-range token counts as rejected, an out-of-range gamma as
+ *    gamma = 0, nothing traps) but are not reported, and a pipeline wait that gave up leaves
+ *    accept_len / p_tok / q_tok of the unfinished sequences unwritten without a way to learn of
+ *    it.  Callers that need the report use bs_softmax_verify with a workspace. */
 #define BS_NOALLOC_SCRATCH_BYTES (2 << 20)
 bs_status bs_softmax_verify_noalloc(const void* target_logits, const void* draft_logits, bs_dtype dtype,
                                     const int32_t* draft_tokens, const int32_t* gamma, const float* u_accept,
@@ -239,6 +252,44 @@ bs_status bs_verify_walk_drafted(const void* target_logits, const void* draft_lo
                                  const float* u_resample, float temperature, int B, int Gmax, int V,
                                  int32_t* accept_len, float* p_tok, float* q_tok, int32_t* out_tokens,
                                  int32_t* out_len, void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---- greedy verification of a tree of drafted tokens (Section 3, example (2): the tree structure of
+ *      the draft is the hyperparameter an arm stands for; Section 2: greedy decoding) -------------- */
+
+/* The paper prints no verification rule for trees; at temperature -> 0 it is determined by Section 2
+ * alone.  The target is a point mass on its arg-max, so the accept rule of Algorithm 6 accepts a drafted
+ * token iff it IS the target's arg-max at its parent.  Node 0 is the prompt; node n = 1..n_b carries the
+ * drafted token node_tokens[b, n-1] and hangs under node_parent[b, n-1], an earlier node (0..n-1).
+ * Row n of target_logits[b] is the target's next-token distribution after the path to node n (what
+ * a forward pass with tree attention returns), row 0 the one after the prompt.  A node passes iff its
+ * parent passes (the prompt does) and its token is the arg-max of its parent's row (lowest index
+ * among equal maxima).  The accepted path ends at the deepest passing node (the lowest-numbered one
+ * among equally deep ones, which only matters if the draft repeated a token among siblings); the
+ * arg-max of that node's own row is emitted after it.  Sampling mode is not offered for trees.
+ *
+ *  target_logits [B, Nmax+1, V] dtype; rows above n_b are never read
+ *  node_parent   [B, Nmax] int32; node_tokens [B, Nmax] int32; n_nodes [B] int32, 0 <= n_b <= Nmax
+ *  accept_len    [B] out: tau_b = depth of the node the accepted path ends at
+ *  out_nodes     [B, Nmax] out or NULL: the nodes of the accepted path in order (the caller keeps
+ *                their key/value entries), -1 behind it
+ *  out_tokens    [B, Nmax+1] out: the accepted tokens, then the emitted arg-max, -1 behind it
+ *  out_len       [B] out: y_b = tau_b + 1, the reward of the arm (Section 3)
+ *  workspace     bs_workspace_bytes(B, Nmax, V) bytes; Nmax <= BS_MAX_GAMMA
+ * Device-detected problems: n_b outside [0, Nmax] (BS_DEV_BAD_GAMMA, processed as the empty tree), a
+ * token outside [0, V) (BS_DEV_BAD_TOKEN, the node never passes), a parent that is not an earlier
+ * node (BS_DEV_BAD_TREE).  Two launches: the row-statistics kernel of bs_softmax_verify in greedy
+ * mode (one arg-max per row, every valid logit read once) and a walk over the nodes. */
+bs_status bs_tree_verify_greedy(const void* target_logits, bs_dtype dtype, const int32_t* node_parent,
+                                const int32_t* node_tokens, const int32_t* n_nodes, int B, int Nmax, int V,
+                                int32_t* accept_len, int32_t* out_nodes, int32_t* out_tokens, int32_t* out_len,
+                                void* workspace, size_t workspace_bytes, void* stream);
+
+/* Per-sequence trees from a table of K tree shapes (the arms): sequence b gets the parents and the node
+ * count of shape arm[b], as bs_bandit_select chose it (arm[b] < 0, an inactive sequence: the empty tree).
+ *  shape_parent [K, Nmax] int32, shape_nodes [K] int32, arm [B] int32 (all device)
+ *  node_parent  [B, Nmax] out, n_nodes [B] out */
+bs_status bs_tree_expand_shapes(const int32_t* shape_parent, const int32_t* shape_nodes, const int32_t* arm, int K,
+                                int B, int Nmax, int32_t* node_parent, int32_t* n_nodes, void* stream);
 
 /* ---- fused LM head (Algorithm 6, second line: the models are evaluated on all drafted positions
  *      in parallel; the last step of that evaluation is logits = H W) -------------------------- */

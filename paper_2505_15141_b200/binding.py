@@ -27,6 +27,7 @@ BS_ERR_INVALID_ARG, BS_ERR_CUDA, BS_ERR_UNSUPPORTED, BS_ERR_WORKSPACE, BS_ERR_TI
 BS_F32, BS_BF16 = 0, 1
 BS_UCB, BS_EXP3, BS_UCB_REWARD = 0, 1, 2
 BS_DEV_BAD_GAMMA, BS_DEV_BAD_TOKEN, BS_DEV_NONFINITE, BS_DEV_RESIDUAL_FALLBACK, BS_DEV_DRAFT_MISSING = 1, 2, 4, 8, 16
+BS_DEV_BAD_TREE = 32
 BS_MAX_GAMMA, BS_MAX_ARMS, BS_MAX_BATCH = 31, 32, 4096
 
 _vp, _i, _f, _d, _sz = C.c_void_p, C.c_int, C.c_float, C.c_double, C.c_size_t
@@ -46,6 +47,8 @@ SIGNATURES = {
                                     _vp]),
     "bs_draft_sample": (_i, [_vp, _i, _i, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _sz, _vp]),
     "bs_softmax_verify_drafted": (_i, [_vp, _vp, _i, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "bs_tree_verify_greedy": (_i, [_vp, _i, _vp, _vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "bs_tree_expand_shapes": (_i, [_vp, _vp, _vp, _i, _i, _i, _vp, _vp, _vp]),
     "bs_lmhead_workspace_bytes": (_sz, [_i, _i, _i]),
     "bs_lmhead_verify": (_i, [_vp, _vp, _i, _vp, _vp, _i, _vp, _vp, _vp, _f, _i, _i, _i, _vp, _vp, _vp, _vp, _vp,
                               _vp, _sz, _vp]),
@@ -252,6 +255,25 @@ def bs_softmax_verify_drafted(target_logits, draft_logits, draft_tokens, gamma, 
                                           B, G1 - 1, V, _ptr(accept_len), _ptr(p_tok), _ptr(q_tok),
                                           _ptr(workspace), workspace.numel(), _stream(stream)),
            "bs_softmax_verify_drafted")
+
+
+# ---- greedy verification of a tree of drafts ---------------------------------------------------
+
+def bs_tree_verify_greedy(target_logits, node_parent, node_tokens, n_nodes, accept_len, out_nodes, out_tokens,
+                          out_len, workspace, stream=None) -> None:
+    """target_logits [B, Nmax+1, V]: row n = the target's logits after the path to node n (row 0: the prompt)."""
+    B, N1, V = target_logits.shape
+    _check(_lib.bs_tree_verify_greedy(_ptr(target_logits), _dtype_code(target_logits), _ptr(node_parent),
+                                      _ptr(node_tokens), _ptr(n_nodes), B, N1 - 1, V, _ptr(accept_len),
+                                      _ptr(out_nodes), _ptr(out_tokens), _ptr(out_len), _ptr(workspace),
+                                      workspace.numel(), _stream(stream)), "bs_tree_verify_greedy")
+
+
+def bs_tree_expand_shapes(shape_parent, shape_nodes, arm, node_parent, n_nodes, stream=None) -> None:
+    K, Nmax = shape_parent.shape
+    B = arm.shape[0]
+    _check(_lib.bs_tree_expand_shapes(_ptr(shape_parent), _ptr(shape_nodes), _ptr(arm), K, B, Nmax,
+                                      _ptr(node_parent), _ptr(n_nodes), _stream(stream)), "bs_tree_expand_shapes")
 
 
 # ---- fused LM head ----------------------------------------------------------------------

@@ -29,7 +29,8 @@ __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a -
 //   ticket_verify [B] u32     per-sequence arrival counters of the statistics kernel (zero between calls)
 //   ticket_resid  [B] u32     per-sequence arrival counters of the resampling kernel (zero between calls)
 //   ticket_row    [B, R] u32  first B words: bit j set = the statistics of draft row j were left by a
-//                             drafting call (bs_draft_sample) and not yet consumed; second B words: decision
+//                             drafting call (bs_draft_sample) and not yet consumed, bit 31 = a drafting pass
+//                             met a row it could not sample; second B words: decision
 //                             words of bs_verify_walk (zero between calls); rest unused
 //   status        [B] i32     device-data status bits of the last call pair
 //   abort         [1] i32     set when a bounded pipeline wait gave up (reported as BS_ERR_TIMEOUT)

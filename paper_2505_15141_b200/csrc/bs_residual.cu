@@ -187,7 +187,7 @@ __global__ void __launch_bounds__(kThreads, 2) residual_kernel(const ResidParams
             s_mass[tid] = tid < p.nseg ? __ldcg(p.resid_partial + (size_t)b * p.S + tid) : 0.f;
             double excl, Rtot;
             double incl = block_scan((double)s_mass[tid], s_w, excl, Rtot);
-            if (!(Rtot > 0.0) || !isfinite(Rtot)) {
+            if (!(Rtot > (f.bonus ? 0.0 : kResidualFloor)) || !isfinite(Rtot)) {
                 // [P - Q]_+ has no mass (P == Q up to rounding) or the row is not finite:
                 // fall back to the target distribution of the same row
                 bits |= f.bonus ? BS_DEV_NONFINITE : BS_DEV_RESIDUAL_FALLBACK;
@@ -321,7 +321,7 @@ extern "C" bs_status bs_residual_sample(const void* target_logits, const void* d
     p.seg = res_seg_elems(dtype);
     p.nseg = div_up(V, p.seg);
     p.c = greedy ? 1.f : kLog2e / temperature;
-    p.mode = kResidVerify; p.position = 0; p.draft_out = nullptr;
+    p.mode = kResidVerify; p.position = 0; p.draft_out = nullptr; p.draft_ready = nullptr;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (greedy) {
         return cuda_status(launch_pdl(greedy_emit_kernel, div_up(B, 128), 128, 0, st, p));
@@ -356,6 +356,7 @@ bs_status bs::run_draft_resample(const void* draft_logits, bs_dtype dtype, int p
     p.nseg = div_up(V, p.seg);
     p.c = kLog2e / temperature;
     p.mode = kResidDraft; p.position = position; p.draft_out = draft_tokens;
+    p.draft_ready = reinterpret_cast<uint32_t*>(ws + w.off_ticket_row);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     return dtype == BS_F32 ? launch_residual_stream<float>(p, st) : launch_residual_stream<__nv_bfloat16>(p, st);
 }

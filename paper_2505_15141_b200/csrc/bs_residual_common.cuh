@@ -30,8 +30,15 @@ struct ResidParams {
     // the row's statistics are read from its draft slot.
     int mode, position;
     int32_t* draft_out;
+    uint32_t* draft_ready;   // kResidDraft: [B] word of the drafted positions; bit 31 reports a row that could not be sampled
 };
 constexpr int kResidVerify = 0, kResidDraft = 1;
+
+// Norm([P - Q]_+) needs a positive total.  The total is the probability of reaching this step at all
+// (1 - sum_v min(P, Q)), and below about 1e-6 what fp32 holds of P - Q is rounding noise of the two
+// normalisers, not a direction: a total at or below this floor counts as "no mass" and the token is
+// drawn from the target row instead (status bit BS_DEV_RESIDUAL_FALLBACK).
+constexpr double kResidualFloor = 1.0 / 262144.0;            // 2^-18
 
 // Mass of one element.  kt / kd fold the row max and normaliser into the exponent, p = at * 2^(x*c + kt):
 // kt is the rounded -(m c + log2 Z); at = 2^(what the two roundings lost) to first order, so that P and Q

@@ -121,7 +121,7 @@ __device__ void rs_level2(const ResidParams& p, int b, const RsSeq sq, MassFn f)
     const float u = p.mode == kResidDraft ? p.u_resample[(size_t)b * p.Gmax + p.position] : p.u_resample[b];
     int tok = -1;
 
-    if (Rtot > 0.0 && isfinite(Rtot)) {
+    if (Rtot > (f.bonus ? 0.0 : kResidualFloor) && isfinite(Rtot)) {
         const double target = (double)u * Rtot;
         double excl = __shfl_up_sync(0xffffffffu, incl, 1);
         if (lane == 0) excl = 0.0;
@@ -288,7 +288,9 @@ __device__ void rs_level2(const ResidParams& p, int b, const RsSeq sq, MassFn f)
     if (p.mode == kResidDraft) {                              // drafting: the token is the whole output
         if (lane == 0) {
             p.draft_out[(size_t)b * p.Gmax + p.position] = tok;
-            if (bits) atomicOr(p.status + b, bits);
+            // the status word belongs to the verification call that follows (it assigns it): what the
+            // drafting pass found travels in the spare bit of the word of drafted positions
+            if (bits) atomicOr(p.draft_ready + b, 0x80000000u);
             p.ticket[b] = 0u;
         }
         return;

@@ -260,13 +260,14 @@ __global__ void __launch_bounds__(kStreamThreads, 2) verify_stream_kernel(const 
                     }
                 } else if (p.mode == kModeDrafted) {
                     // target rows were merged just now, the draft rows' statistics were left by the drafting calls
-                    const unsigned need = gb >= 32 ? 0xffffffffu : ((1u << gb) - 1u);
+                    const unsigned need = (1u << gb) - 1u;        // gamma <= 31
                     const unsigned have = GREEDY ? need : __ldcg(p.draft_ready + m_b);
                     const float2* rsb = p.row_stats + (size_t)m_b * p.R;
                     const int G1 = p.Gmax + 1;
                     accept_finish<T, GREEDY>(p, m_b, graw, gb, al,
                                              [&](int rr) { return rr < G1 ? s_fin[rr] : __ldcg(rsb + rr); },
-                                             (have & need) == need ? 0 : BS_DEV_DRAFT_MISSING);
+                                             ((have & need) == need ? 0 : BS_DEV_DRAFT_MISSING) |
+                                                 ((have >> 31) ? BS_DEV_NONFINITE : 0));   // a drafting pass could not sample its row
                     if (lane == 0) p.draft_ready[m_b] = 0u;       // consumed: a later round must draft again
                 } else {
                     accept_finish<T, GREEDY>(p, m_b, graw, gb, al, [&](int rr) { return s_fin[rr]; });

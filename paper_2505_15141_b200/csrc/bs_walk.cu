@@ -370,8 +370,10 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                 bool missing = false;                          // drafted mode: position k was never drafted
                 if (p.drafted && k < g) {
                     if (lane == 0) s_fin[1] = __ldcg(v.row_stats + (size_t)b * v.R + v.Gmax + 1 + k);
-                    missing = ((__ldcg(v.draft_ready + b) >> k) & 1u) == 0u;
+                    const unsigned ready = __ldcg(v.draft_ready + b);
+                    missing = ((ready >> k) & 1u) == 0u;
                     if (missing) bits |= BS_DEV_DRAFT_MISSING;
+                    if (ready >> 31) bits |= BS_DEV_NONFINITE;   // a drafting pass could not sample its row
                     __syncwarp();
                 }
                 if (!(ts.y > 0.f) || !isfinite(ts.y) || !isfinite(ts.x)) bits |= BS_DEV_NONFINITE;
@@ -634,7 +636,7 @@ static bs_status run_walk(const void* target_logits, const void* draft_logits, b
     r.seg = res_seg_elems(dtype);
     r.nseg = div_up(V, r.seg);
     r.c = v.c;
-    r.mode = kResidVerify; r.position = 0; r.draft_out = nullptr;
+    r.mode = kResidVerify; r.position = 0; r.draft_out = nullptr; r.draft_ready = nullptr;
     // decision words: the second B words of the per-row counter slot (the first B mark drafted positions)
     p.dec = v.ticket_row + B;
     p.nG = 1;
