@@ -85,6 +85,10 @@ def parse_args():
     ap.add_argument("--walk", action="store_true",
                     help="the round with early exit: select -> bs_verify_walk (verification up to the first "
                          "rejection + resampling in one launch) -> update")
+    ap.add_argument("--auto-path", action="store_true",
+                    help="time a few rounds of the two-call path and of the early-exit path first and run the timed "
+                         "region on the faster one (config.path says which); early exit emits the same tokens but forms "
+                         "the token probabilities only up to the first rejection")
     ap.add_argument("--no-others", action="store_true",
                     help="skip the short runs of the other workloads that the default invocation adds to its line")
     ap.add_argument("--bandit-step", action="store_true",
@@ -429,6 +433,33 @@ def run_cuda(args, w):
             bs.bs_bandit_select(state, alg, B, K, sets[0]["u_arm"], None, arm_d, gamma_d)
 
     side = torch.cuda.Stream(device=dev)
+    path_choice = None
+    if args.auto_path and not drafted and w.temperature > 0.0:
+        # one graph per path on the first input set, replayed: the same inputs and the same cache state for both
+        trial = {}
+        with torch.cuda.stream(side):
+            for cand in (False, True):
+                walk = cand
+                first_select()
+                step_calls(sets[0], sets[1 % ring])
+                side.synchronize()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    step_calls(sets[0], sets[1 % ring])
+                for _ in range(5):
+                    g.replay()
+                a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(side)
+                for _ in range(40):
+                    g.replay()
+                b_.record(side)
+                side.synchronize()
+                trial[cand] = a.elapsed_time(b_) / 40
+                del g
+        walk = trial[True] < trial[False]
+        path_choice = {"two_call_ms": trial[False], "early_exit_ms": trial[True], "chosen": "early_exit" if walk else "two_call"}
+        torch.cuda.synchronize()
+        init_call()
     graphs = []
     if not args.no_graph:
         with torch.cuda.stream(side):
@@ -654,7 +685,7 @@ def run_cuda(args, w):
                                                   {"ms": verify_ms + resid_ms,
                                                    "achieved": verify_bytes / ((verify_ms + resid_ms) * 1e-3) / 1e9,
                                                    "frac": verify_bytes / ((verify_ms + resid_ms) * 1e-3) / 1e9 / peak})},
-            "e2e": e2e, "cpu_baseline": cpu, "clocks": clocks, "variants": variants,
+            "e2e": e2e, "cpu_baseline": cpu, "clocks": clocks, "variants": variants, "path_choice": path_choice,
             "other_workloads": getattr(args, "others", None),
             "gpu_launches": ((3 if walk else 4) - (1 if fused_bandit else 0) + (2 * G if drafted else 0)
                              + (1 if reward else 0)) * args.steps,

@@ -19,37 +19,10 @@
 //
 // CTAs of one group wait for one another, so the kernel is launched cooperatively (all CTAs
 // resident).  Every wait is bounded; a wait that gives up sets the abort word and the CTA drains.
-#include "bs_verify_common.cuh"
-#include "bs_residual_level2.cuh"
-#include "bs_pipeline.cuh"
+#include "bs_walk_common.cuh"
 
 namespace bs {
 
-constexpr int kWkWarps = 16;
-constexpr int kWkConsumers = kWkWarps * 32;
-constexpr int kWkThreads = kWkConsumers + 64;                    // + producer warp + finisher warp
-constexpr int kWkStages = 3;
-constexpr int kWkRing = 8;                                       // events the consumers may run ahead of the finisher
-constexpr int kWkVecPerThread = kSegBytes / 16 / kWkConsumers;   // 4
-static_assert(kSegBytes == 2 * kResSegBytes && kWkWarps == kRsWarps, "one stage holds a segment or a pair of half segments");
-
-constexpr int kItemStats = 0, kItemMass = 1, kItemEnd = 2, kItemAck = 3;
-
-struct WalkParams {
-    VerifyParams v;        // logits, tokens, uniforms, outputs of the accept test, statistics and partials
-    ResidParams r;         // the same logits for the residual pass, its outputs, piece masses
-    uint32_t* dec;         // [B] decision word: (positions decided << 1) | last one accepted
-    int nG;                // CTAs per sequence
-    int drafted;           // 1: the draft rows' statistics were left by bs_draft_sample: stream target rows only
-};
-
-// Per-stage record, written by the producer.
-struct WkMeta {
-    int type, b, k;
-    int row;               // stats: 0 = target row k, 1 = draft row k;  mass: 1 = target row only (bonus)
-    int sg, nvec, flags;   // flags bit 0: first stage of a row piece, bit 1: last stage of a piece / of the CTA's share
-    float kt, kd, at, ad;
-};
 // Per event handed to the finisher (written by consumer warp 0).
 struct WkEvent {
     int type, b, k, row, first_sg, last_sg;
@@ -137,13 +110,22 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
         long long t_last = clock64();
         while (alive > 0 && ok) {
             bool progress = false;
+            unsigned dd[8];                                   // decision words of eight shares, asked for together
             for (int si = 0; si < nmine && ok; ++si) {
+                if ((si & 7) == 0) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        dd[i] = (si + i < nmine && s_seq[si + i].stage == 1) ? ld_volatile_u32(p.dec + s_seq[si + i].b) : 0u;
+                }
                 WkSeq sq = s_seq[si];
                 if (sq.stage == 2) continue;
                 const int b = sq.b, g = sq.g, part = sq.part;
                 if (sq.stage == 1) {
                     // ---- has position k been decided (by whichever finisher of the group completed it)? ----
-                    const unsigned d = ld_volatile_u32(p.dec + b);
+                    unsigned d = 0u;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        if ((si & 7) == i) d = dd[i];
                     if ((d >> 1) != (unsigned)(sq.k + 1)) continue;
                     __threadfence();
                     progress = true;
@@ -319,47 +301,59 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                 float2* pp = v.partial + ((size_t)b * v.R + slot_r) * v.S;
                 for (int q = e.first_sg + lane; q <= e.last_sg; q += 32)
                     pp[q] = (q == e.first_sg) ? out : make_float2(-INFINITY, 0.f);
-                // the drafted token, its two logits, the uniform (they do not depend on the statistics:
-                // in flight while the ticket is)
-                int x = 0;
-                float tl = 0.f, dl = 0.f, u = 2.f;
-                bool bad = false;
-                if (k < g) {
-                    x = v.tokens[(size_t)b * v.Gmax + k];
-                    bad = x < 0 || x >= v.V;
-                    if (!bad) {
-                        tl = Elem<T>::load(row_ptr(static_cast<const T*>(v.target), b, v.Gmax + 1, k, v.V) + x);
-                        dl = Elem<T>::load(row_ptr(static_cast<const T*>(v.draft), b, v.Gmax, k, v.V) + x);
-                        u = v.u_accept[(size_t)b * v.Gmax + k];
-                    }
-                }
                 __threadfence();
                 __syncwarp();
                 unsigned old = 0;
                 if (lane == 0) old = atomicAdd(v.ticket + b, (unsigned)len);
                 old = __shfl_sync(0xffffffffu, old, 0);
                 if (old + (unsigned)len != (p.drafted ? wk_cum<true>(k, g, v.nseg) : wk_cum<false>(k, g, v.nseg))) continue;
-                // ---- position k is complete: merge its rows (lane 0: target, lane 1: draft), decide ----
+                // ---- position k is complete: merge its rows (lanes 0..15: target, 16..31: draft), decide ----
+                // Everything the decision needs is asked for in two rounds of independent loads: the drafted
+                // token, the uniform and all partial slots of the two rows, then the two logits at the token
+                // (a load that waits for another costs a full trip through a busy memory system; the fence
+                // above would have waited for any of them issued earlier).
                 __threadfence();
-                // lanes 0..15 merge the partials of target row k, lanes 16..31 those of draft row k
+                int x = 0;
+                float tl = 0.f, dl = 0.f, u = 2.f;
+                bool bad = false;
+                if (k < g) {
+                    x = v.tokens[(size_t)b * v.Gmax + k];
+                    u = v.u_accept[(size_t)b * v.Gmax + k];
+                }
                 {
                     const int half = lane >> 4, hl = lane & 15;
                     const int rr = half == 0 ? k : v.Gmax + 1 + k;
+                    const bool mine_row = half == 0 || (k < g && !p.drafted);
+                    const float2* qq = v.partial + ((size_t)b * v.R + rr) * v.S;
                     Online o{-INFINITY, 0.f};
-                    if (half == 0 || (k < g && !p.drafted)) {
-                        const float2* qq = v.partial + ((size_t)b * v.R + rr) * v.S;
-                        for (int q = hl; q < v.nseg; q += 16) {
-                            const float2 t = __ldcg(qq + q);
-                            o.merge(t.x, t.y, v.c);
+                    for (int q0 = hl; q0 < v.nseg; q0 += 64) {        // four slots per lane in flight
+                        float2 t[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int q = q0 + 16 * i;
+                            t[i] = (mine_row && q < v.nseg) ? __ldcg(qq + q) : make_float2(-INFINITY, 0.f);
                         }
+                        if (q0 == hl && k < g) {                      // the token has arrived by now: its two logits
+                            bad = x < 0 || x >= v.V;
+                            if (!bad) {
+                                tl = Elem<T>::load(row_ptr(static_cast<const T*>(v.target), b, v.Gmax + 1, k, v.V) + x);
+                                dl = Elem<T>::load(row_ptr(static_cast<const T*>(v.draft), b, v.Gmax, k, v.V) + x);
+                            }
+                        }
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) o.merge(t[i].x, t[i].y, v.c);
                     }
+                    // lanes whose first slot lies beyond the row never entered the loop: lane 0 always did
+                    tl = __shfl_sync(0xffffffffu, tl, 0);
+                    dl = __shfl_sync(0xffffffffu, dl, 0);
+                    bad = __shfl_sync(0xffffffffu, (int)bad, 0) != 0;
                     float M = o.m;
 #pragma unroll
                     for (int off = 8; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
                     float Z = o.s * rescale(o.m, M, v.c);
 #pragma unroll
                     for (int off = 8; off > 0; off >>= 1) Z += __shfl_xor_sync(0xffffffffu, Z, off);
-                    if (hl == 0 && (half == 0 || (k < g && !p.drafted))) {
+                    if (hl == 0 && mine_row) {
                         s_fin[half] = make_float2(M, Z);
                         v.row_stats[(size_t)b * v.R + rr] = make_float2(M, Z);
                     }
@@ -411,6 +405,14 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
                 __threadfence();
                 __syncwarp();
                 if (lane == 0) atomicExch(p.dec + b, ((unsigned)(k + 1) << 1) | (acc ? 1u : 0u));
+                if (acc && k + 1 < g && lane == 0) {
+                    // the walk goes on: ask L2 for the two logits the next decision will need (nobody waits for this)
+                    const int xn = v.tokens[(size_t)b * v.Gmax + k + 1];
+                    if (xn >= 0 && xn < v.V) {
+                        asm volatile("prefetch.global.L2 [%0];" ::"l"(row_ptr(static_cast<const T*>(v.target), b, v.Gmax + 1, k + 1, v.V) + xn));
+                        asm volatile("prefetch.global.L2 [%0];" ::"l"(row_ptr(static_cast<const T*>(v.draft), b, v.Gmax, k + 1, v.V) + xn));
+                    }
+                }
             } else {
                 // ---- this CTA's share of the residual masses of the stop position k is written ----
                 __threadfence();
@@ -642,6 +644,12 @@ static bs_status run_walk(const void* target_logits, const void* draft_logits, b
     p.nG = 1;
     p.drafted = (drafted && !greedy) ? 1 : 0;         // greedy rounds never read draft rows anyway
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // groups of 2, 4 or 8 CTAs as thread-block clusters (hand-offs through distributed shared memory); rows of a
+    // single segment and batches too large for that leave one CTA per sequence: the kernel of this file
+    bs_status s;
+    if (greedy) s = dtype == BS_F32 ? launch_walk_cluster<float, true>(p, st) : launch_walk_cluster<__nv_bfloat16, true>(p, st);
+    else s = dtype == BS_F32 ? launch_walk_cluster<float, false>(p, st) : launch_walk_cluster<__nv_bfloat16, false>(p, st);
+    if (s != BS_ERR_UNSUPPORTED) return s;
     if (greedy) return dtype == BS_F32 ? launch_walk<float, true>(p, st) : launch_walk<__nv_bfloat16, true>(p, st);
     return dtype == BS_F32 ? launch_walk<float, false>(p, st) : launch_walk<__nv_bfloat16, false>(p, st);
 }
