@@ -43,8 +43,9 @@ FALLBACK_HBM_GBS = 6650.0
 # write-backs) do not.  An entry is only valid for the kernel it was captured on: when that kernel
 # changes, the entry goes to None until the capture is repeated.
 NCU_TRAFFIC = {
-    "qwen_exp3": None,
-    "llama3_ucb": None,
+    "qwen_exp3": (1.0003, 4.1e6),          # fp32 statistics kernel, captured at B=32
+    "llama3_ucb": (1.0005, 3.9e6),         # bf16 statistics kernel
+    "llama3_tree": (1.0004, 4.5e6),        # the same kernel in greedy mode
     "lmhead_llama3": (1.0000, 30.6e6),     # B=16 (logits still dirty in L2 are not counted)
     "lmhead_llama3_b128": (1.0180, 568.1e6),
 }
@@ -73,7 +74,7 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--workload", default="qwen_exp3",
                     choices=["tiny_ucb", "llama2_fixed", "llama3_ucb", "qwen_exp3", "llama3_tput", "lmhead_llama3",
-                             "lmhead_llama3_b128"])
+                             "lmhead_llama3_b128", "llama3_tree", "tiny_tree"])
     ap.add_argument("--batch", type=int, default=0,
                     help="override the workload's batch size (smaller cases for profiler captures)")
     ap.add_argument("--fixed-gamma", type=int, default=0,
@@ -937,7 +938,242 @@ def run_lmhead(args, w):
         dist.destroy_process_group()
 
 
-OTHER_WORKLOADS = ("llama3_ucb", "llama2_fixed", "llama3_tput", "lmhead_llama3", "lmhead_llama3_b128")
+# ---------------------------------------------------------------------------------------------
+# greedy verification of a tree of drafts, tree shapes as the arms of UCBSpec
+# ---------------------------------------------------------------------------------------------
+
+def tree_oracle_inputs(w):
+    from paper_2505_15141_b200 import workloads as wl
+    import dataclasses as dc
+    inp = wl.make_tree_inputs(dc.replace(w, B=min(w.B, ORACLE_SAMPLE_SEQS)), 1, "cpu")
+    t = inp.target.float().numpy()
+    return [(t[b], [int(x) for x in w.shapes[b % w.K]], inp.tokens[b % w.K, b].numpy(), len(w.shapes[b % w.K]))
+            for b in range(t.shape[0])]
+
+
+def tree_oracle_sample(seqs, seconds: float):
+    from oracle import tree as otree
+    done, t0 = 0, time.perf_counter()
+    while True:
+        rows, parent, tokens, n = seqs[done % len(seqs)]
+        otree.verify_tree_greedy(rows, parent, tokens, n)
+        done += 1
+        if time.perf_counter() - t0 > seconds:
+            break
+    return done, time.perf_counter() - t0
+
+
+def tree_config(w) -> dict:
+    return {"workload": w.name, "B": w.B, "V": w.V, "logits_dtype": w.dtype, "temperature": 0.0,
+            "shapes": {"nodes": [len(x) for x in w.shapes], "depth": list(w.depths)}, "bandit": "ucb over the shapes"}
+
+
+def run_tree_reference(args, w):
+    import torch
+    torch.set_num_threads(1)
+    per_step = max(0.2, min(10.0, 90.0 / max(1, args.steps + args.warmup), args.cpu_seconds))
+    seqs = tree_oracle_inputs(w)
+    n_tot, t_tot = 0, 0.0
+    for i in range(args.warmup + args.steps):
+        n, dt = tree_oracle_sample(seqs, per_step)
+        if i >= args.warmup:
+            n_tot += n; t_tot += dt
+    val = (n_tot / w.B) / t_tot
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * t_tot / max(1, args.steps), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": tree_config(w),
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle",
+                         "sample": f"{n_tot} tree verifications of the first {len(seqs)} sequences in {t_tot:.1f} s "
+                                   f"(numpy, one thread)"},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}, "gpu_launches": 0}))
+
+
+def run_tree(args, w):
+    import torch
+    import torch.distributed as dist
+    import __graft_entry__ as entry
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        dist.init_process_group(backend="nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if rank == 0:
+        entry.build()
+    if world > 1:
+        dist.barrier()
+    from paper_2505_15141_b200 import binding as bs, workloads as wl
+
+    B, K, N, V, es = w.B, w.K, w.Nmax, w.V, w.elem_size
+    set_bytes = es * V * B * (N + 1)
+    ring = max(2, -(-2 * L2_BYTES // set_bytes) + 1)
+    sets = [wl.make_tree_inputs(w, rank_round_index(rank, i), dev) for i in range(ring)]
+    sp_d, sn_d = sets[0].shape_parent, sets[0].shape_nodes
+    state = bs.new_bandit(bs.BS_UCB, B, w.depths, w.delta, dev)
+    ws = bs.new_workspace(B, N, V, dev)
+    arm_d = torch.zeros(B, dtype=torch.int32, device=dev); gam_d = torch.zeros_like(arm_d)
+    parent_d = torch.zeros(B, N, dtype=torch.int32, device=dev); n_d = torch.zeros(B, dtype=torch.int32, device=dev)
+    tok_d = torch.zeros(B, N, dtype=torch.int32, device=dev)
+    acc = torch.zeros(B, dtype=torch.int32, device=dev); on = torch.zeros(B, N, dtype=torch.int32, device=dev)
+    otk = torch.zeros(B, N + 1, dtype=torch.int32, device=dev); ol = torch.zeros(B, dtype=torch.int32, device=dev)
+    rows_b = torch.arange(B, device=dev)
+
+    def step_calls(s):
+        bs.bs_bandit_select(state, bs.BS_UCB, B, K, None, None, arm_d, gam_d)
+        bs.bs_tree_expand_shapes(sp_d, sn_d, arm_d, parent_d, n_d)
+        tok_d.copy_(s.tokens[arm_d.long(), rows_b])           # stands in for the draft model drafting along the chosen shape
+        bs.bs_tree_verify_greedy(s.target, parent_d, tok_d, n_d, acc, on, otk, ol, ws)
+        bs.bs_bandit_update(state, bs.BS_UCB, B, K, arm_d, ol)
+
+    def sync_all():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    side = torch.cuda.Stream(device=dev)
+    graphs = []
+    if not args.no_graph:
+        with torch.cuda.stream(side):
+            step_calls(sets[0])
+            side.synchronize()
+            for s_ in sets:
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    step_calls(s_)
+                graphs.append(g)
+        torch.cuda.synchronize()
+        bs.bs_bandit_init(state, bs.BS_UCB, B, K, w.depths, w.delta)
+
+    def run_step(i):
+        if graphs:
+            graphs[i % ring].replay()
+        else:
+            step_calls(sets[i % ring])
+
+    for i in range(args.warmup):
+        run_step(i)
+    sync_all()
+    n0 = bs.bs_bandit_read(state, bs.BS_UCB, B, K)["n"].copy()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    sync_all()
+    stream = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(args.steps):
+        run_step(args.warmup + i)
+    e1.record(stream)
+    sync_all()
+    ms = e0.elapsed_time(e1)
+    clocks = None
+    if rank == 0:
+        time.sleep(0.15)
+        clocks = sampler.stop()
+    nodes = np.asarray([len(x) for x in w.shapes])
+    dn = bs.bs_bandit_read(state, bs.BS_UCB, B, K)["n"] - n0
+    assert dn.sum() == B * args.steps
+    bytes_timed = float((dn * (nodes + 1)[None, :]).sum()) * V * es
+    ms, bytes_all = reduce_over_ranks(ms, bytes_timed, dev)
+    value = job_rounds_per_s(world, args.steps, ms)
+
+    # kernel pass: events around bs_tree_verify_greedy (statistics kernel in greedy mode + the walk over the nodes)
+    ksteps = min(args.steps, 50)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(ksteps)]
+    y_sum = torch.zeros((), dtype=torch.int64, device=dev)
+    nk0 = bs.bs_bandit_read(state, bs.BS_UCB, B, K)["n"].copy()
+    for i in range(ksteps):
+        s_ = sets[(args.warmup + args.steps + i) % ring]
+        bs.bs_bandit_select(state, bs.BS_UCB, B, K, None, None, arm_d, gam_d)
+        bs.bs_tree_expand_shapes(sp_d, sn_d, arm_d, parent_d, n_d)
+        tok_d.copy_(s_.tokens[arm_d.long(), rows_b])
+        hold_gpu()
+        evs[i][0].record(stream)
+        bs.bs_tree_verify_greedy(s_.target, parent_d, tok_d, n_d, acc, on, otk, ol, ws)
+        evs[i][1].record(stream)
+        bs.bs_bandit_update(state, bs.BS_UCB, B, K, arm_d, ol)
+        y_sum += ol.sum()
+    torch.cuda.synchronize()
+    k_ms = sum(a.elapsed_time(b) for a, b in evs) / ksteps
+    dk = bs.bs_bandit_read(state, bs.BS_UCB, B, K)["n"] - nk0
+    k_bytes = float((dk * (nodes + 1)[None, :]).sum()) * V * es / ksteps
+    mean_y = float(y_sum.item()) / (B * ksteps)
+    assert (bs.bs_get_device_status(ws, B, N, V) == 0).all()
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
+    else:
+        peak, peak_src = FALLBACK_HBM_GBS, "fallback"
+    achieved = k_bytes / (k_ms * 1e-3) / 1e9
+
+    e2e = None
+    if args.e2e_steps > 0:
+        s0 = sets[0]
+        host = {"target": torch.empty(s0.target.shape, dtype=s0.target.dtype, pin_memory=True).copy_(s0.target),
+                "tokens": torch.empty(s0.tokens.shape, dtype=s0.tokens.dtype, pin_memory=True).copy_(s0.tokens)}
+        devb = wl.TreeInputs(target=torch.empty_like(s0.target), tokens=torch.empty_like(s0.tokens),
+                             shape_parent=sp_d, shape_nodes=sn_d)
+        h_tok = torch.empty(otk.shape, dtype=otk.dtype, pin_memory=True)
+        h_len = torch.empty(ol.shape, dtype=ol.dtype, pin_memory=True)
+        h2d = sum(t.numel() * t.element_size() for t in host.values())
+        d2h = h_tok.numel() * 4 + h_len.numel() * 4
+
+        def e2e_step():
+            devb.target.copy_(host["target"], non_blocking=True)
+            devb.tokens.copy_(host["tokens"], non_blocking=True)
+            step_calls(devb)
+            h_tok.copy_(otk, non_blocking=True)
+            h_len.copy_(ol, non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+
+        for _ in range(2):
+            e2e_step()
+        sync_all()
+        a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        b_.record(stream)
+        sync_all()
+        e2e_ms, _ = reduce_over_ranks(a.elapsed_time(b_), 0.0, dev)
+        e2e = {"value": world * args.e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+               "d2h_bytes_per_step": int(d2h), "steps": args.e2e_steps}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        torch.set_num_threads(1)
+        seqs = tree_oracle_inputs(w)
+        n, dt = tree_oracle_sample(seqs, args.cpu_seconds)
+        cpu = {"value": (n / B) / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": f"{n} tree verifications of the first {len(seqs)} sequences in {dt:.1f} s (numpy, one thread; "
+                         f"host has {host_cores()} cores)"}
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {**tree_config(w), "l2": f"ring of {ring} input sets, {ring * set_bytes / 1e6:.0f} MB > 2 x L2",
+                       "launch": "one CUDA graph per step" if graphs else "direct launches",
+                       "path": "select, expand shapes, (token table lookup: torch), tree verify (2 launches), update",
+                       "multi_gpu": "one independent batch per rank, no collective on the data path"},
+            "tokens_per_s": mean_y * B * value, "mean_accepted_len": mean_y,
+            "algorithmic_gbs": bytes_all / (ms * 1e-3) / 1e9,
+            "roofline": {"bound": "hbm", "kernel": "verify_stream_kernel, greedy mode + tree_walk_kernel (bs_tree_verify_greedy)",
+                         "achieved": achieved, "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": ncu_traffic(w.name, k_bytes), "bytes_per_launch": k_bytes, "ms_per_launch": k_ms,
+                         "residual_ms_per_launch": 0.0},
+            "e2e": e2e, "cpu_baseline": cpu, "clocks": clocks, "gpu_launches": 5 * args.steps}))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+OTHER_WORKLOADS = ("llama3_ucb", "llama2_fixed", "llama3_tput", "llama3_tree", "lmhead_llama3", "lmhead_llama3_b128")
 
 
 def other_workloads_summary():
@@ -1000,6 +1236,16 @@ def main():
                 run_lmhead_reference(args, w)
             return
         run_lmhead(args, w)
+        return
+    if args.workload in wl.TREE_WORKLOADS:
+        w = wl.TREE_WORKLOADS[args.workload]
+        if args.batch:
+            w = dataclasses.replace(w, B=args.batch)
+        if args.impl == "reference":
+            if rank == 0:
+                run_tree_reference(args, w)
+            return
+        run_tree(args, w)
         return
     w = wl.WORKLOADS[args.workload]
     if args.batch:

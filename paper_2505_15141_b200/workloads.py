@@ -351,3 +351,82 @@ def make_lmhead_inputs(w: LmHeadWorkload, rnd: int = 1, device="cpu", gamma: Opt
         tok = torch.zeros(B, 0, dtype=torch.int32, device=device)
     gam = np.full(B, G, dtype=np.int32) if gamma is None else np.asarray(gamma, dtype=np.int32)
     return LmHeadInputs(H_t=H_t, W_t=W_t, H_d=H_d, W_d=W_d, tokens=tok.contiguous(), gamma=gam, uniforms=un)
+
+
+# --------------------------------------------------------------------------
+# Inputs of the greedy tree-verification path: tree shapes as arms
+# --------------------------------------------------------------------------
+
+@dataclass(frozen=True)
+class TreeWorkload:
+    name: str
+    B: int
+    V: int
+    dtype: str                      # "bf16" | "f32"
+    shapes: Tuple[Tuple[int, ...], ...]   # per arm: parent of node 1..n (0 = the prompt)
+    p_right: float                  # probability that a drafted node carries the target's arg-max at its parent
+    seed: int
+    delta: float = 0.5
+
+    @property
+    def K(self) -> int:
+        return len(self.shapes)
+
+    @property
+    def Nmax(self) -> int:
+        return max(len(s) for s in self.shapes)
+
+    @property
+    def depths(self) -> Tuple[int, ...]:
+        out = []
+        for s in self.shapes:
+            d = [0]
+            for par in s:
+                d.append(d[par] + 1)
+            out.append(max(d))
+        return tuple(out)
+
+    @property
+    def elem_size(self) -> int:
+        return 2 if self.dtype == "bf16" else 4
+
+
+TREE_WORKLOADS = {
+    # LLaMA-3 vocabulary, 64 sequences, three shapes: a chain of 5, a binary tree of depth 3, a 3 x 3 tree of depth 2
+    "llama3_tree": TreeWorkload("llama3_tree", B=64, V=128256, dtype="bf16",
+                                shapes=((0, 1, 2, 3, 4), (0, 0, 1, 1, 2, 2, 3, 3, 4, 4, 5, 5, 6, 6),
+                                        (0, 0, 0, 1, 1, 1, 2, 2, 2, 3, 3, 3)), p_right=0.75, seed=6),
+    "tiny_tree": TreeWorkload("tiny_tree", B=4, V=1024, dtype="f32",
+                              shapes=((0, 1, 2), (0, 0, 1, 1, 2, 2), (0, 0, 0)), p_right=0.75, seed=7),
+}
+
+
+@dataclass
+class TreeInputs:
+    target: torch.Tensor       # [B, Nmax+1, V]: row n = the target's logits after the path to node n
+    tokens: torch.Tensor       # [K, B, Nmax] int32: the drafted tokens if sequence b uses shape k
+    shape_parent: torch.Tensor  # [K, Nmax] int32
+    shape_nodes: torch.Tensor   # [K] int32
+
+
+def make_tree_inputs(w: TreeWorkload, rnd: int = 1, device="cpu") -> TreeInputs:
+    """Target rows as in the chain workloads (N(0, 3^2) with 5 % of the entries raised by 8).  There is no draft
+    model here: a drafted node carries the target's arg-max at its parent with probability p_right and a uniformly
+    drawn token otherwise, for every shape a sequence might be given (the shape is chosen on the device)."""
+    B, V, N, K = w.B, w.V, w.Nmax, w.K
+    g = torch_generator(w.seed, rnd, device)
+    t = torch.empty(B, N + 1, V, dtype=torch.float32, device=device).normal_(0.0, 3.0, generator=g)
+    t += 8.0 * (torch.rand(B, N + 1, V, generator=g, device=device) < 0.05)
+    t = t.to(torch.bfloat16 if w.dtype == "bf16" else torch.float32)
+    am = t.float().argmax(dim=-1)                                   # [B, N+1]
+    sp = torch.zeros(K, N, dtype=torch.int32)
+    sn = torch.zeros(K, dtype=torch.int32)
+    for k, s in enumerate(w.shapes):
+        sp[k, :len(s)] = torch.tensor(s, dtype=torch.int32)
+        sn[k] = len(s)
+    sp, sn = sp.to(device), sn.to(device)
+    right = torch.rand(K, B, N, generator=g, device=device) < w.p_right
+    rnd_tok = torch.randint(0, V, (K, B, N), generator=g, device=device)
+    at_parent = torch.stack([am.gather(1, sp[k].long().unsqueeze(0).expand(B, N)) for k in range(K)])   # [K, B, N]
+    tok = torch.where(right, at_parent, rnd_tok).to(torch.int32)
+    return TreeInputs(target=t.contiguous(), tokens=tok.contiguous(), shape_parent=sp, shape_nodes=sn)

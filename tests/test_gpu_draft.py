@@ -195,3 +195,37 @@ def test_drafted_walk_equals_plain_walk_and_the_oracle(lib):
     st = lib.bs_get_device_status(ws, B, G, V)
     for b in range(B):
         assert bool(st[b] & lib.BS_DEV_DRAFT_MISSING) == (gamma[b] > 0) and (gamma[b] == 0 or int(acc[b]) == 0)
+
+
+@pytest.mark.parametrize("walk", [False, True])
+def test_a_draft_row_that_cannot_be_sampled_is_reported_by_the_verification(lib, walk):
+    """A draft row with a NaN has no finite normaliser: the drafting pass cannot sample it (it emits token 0) and
+    says so through the drafted-positions word, the verification call that follows reports BS_DEV_NONFINITE for
+    that sequence -- whichever of the two drafted verification entry points is used -- and the other sequences
+    are untouched."""
+    B, G, V, T = 4, 3, 8192, 1.0
+    t, d = _logits(17, B, G, V, torch.float32)
+    d[1, 1, 77] = float("nan")
+    gamma = np.array([3, 3, 2, 3], np.int32); gamma_d = torch.as_tensor(gamma, device=DEV)
+    un = wl.round_uniforms(5, 1, B, G)
+    u_d = torch.as_tensor(un.u_draft, device=DEV)
+    ws = lib.new_workspace(B, G, V, DEV)
+    tok = _draft_all(lib, d, gamma_d, u_d, T, ws)
+    assert 0 <= int(tok[1, 1]) < V
+    acc = torch.full((B,), -1, dtype=torch.int32, device=DEV)
+    p = torch.zeros(B, G, device=DEV); q = torch.zeros(B, G, device=DEV)
+    ot = torch.zeros(B, G + 1, dtype=torch.int32, device=DEV); ol = torch.zeros(B, dtype=torch.int32, device=DEV)
+    ua = torch.as_tensor(un.u_accept, device=DEV); ur = torch.as_tensor(un.u_resample, device=DEV)
+    if walk:
+        lib.bs_verify_walk_drafted(t, d, tok, gamma_d, ua, ur, T, acc, p, q, ot, ol, ws)
+    else:
+        lib.bs_softmax_verify_drafted(t, d, tok, gamma_d, ua, T, acc, p, q, ws)
+        lib.bs_residual_sample(t, d, tok, gamma_d, acc, ur, T, ot, ol, ws)
+    torch.cuda.synchronize()
+    st = lib.bs_get_device_status(ws, B, G, V)
+    assert st[1] & lib.BS_DEV_NONFINITE, st
+    assert (st[[0, 2, 3]] & ~lib.BS_DEV_RESIDUAL_FALLBACK == 0).all(), st
+    # the healthy sequences against the oracle
+    rin = wl.RoundInputs(target=t, draft=d, tokens=tok, gamma=gamma, uniforms=un)
+    out = lib.RoundOutput(acc, p, q, ot, ol, ws)
+    parity.check_round(out, rin, T, parity.Tally(), seqs=[0, 2, 3], where="beside a NaN draft row", walk=walk)

@@ -94,3 +94,25 @@ def test_throughput_workloads_reward_range_and_step_duration():
         # gamma = 0 rounds have one target row per sequence and emit exactly one token
         rnd = wl.make_round(w, 1, np.zeros(w.B, dtype=np.int32), B=min(w.B, 3))
         assert (rnd.gamma == 0).all() and rnd.target.shape[1] == w.Gmax + 1
+
+
+def test_tree_workload_inputs():
+    from oracle import tree as ot
+    w = wl.TREE_WORKLOADS["tiny_tree"]
+    assert w.K == 3 and w.Nmax == 6 and w.depths == (3, 2, 1)
+    a, b = wl.make_tree_inputs(w, 3), wl.make_tree_inputs(w, 3)
+    assert torch.equal(a.target, b.target) and torch.equal(a.tokens, b.tokens)            # seeded
+    assert a.target.shape == (w.B, w.Nmax + 1, w.V) and a.tokens.shape == (w.K, w.B, w.Nmax)
+    assert a.shape_nodes.tolist() == [3, 6, 3] and a.shape_parent[1].tolist() == [0, 0, 1, 1, 2, 2]
+    # parents come before children, and the shapes' depths are what the checker computes
+    for k, s in enumerate(w.shapes):
+        assert all(p < n + 1 for n, p in enumerate(s)) and max(ot.tree_depths(list(s), len(s))) == w.depths[k]
+    # about p_right of the drafted nodes carry the target's arg-max at their parent
+    big = wl.make_tree_inputs(wl.TREE_WORKLOADS["tiny_tree"].__class__("t", B=64, V=512, dtype="f32",
+                              shapes=w.shapes, p_right=0.75, seed=1), 1)
+    am = big.target.argmax(dim=-1)
+    hits = tot = 0
+    for k, s in enumerate(w.shapes):
+        for n, p in enumerate(s):
+            hits += int((big.tokens[k, :, n].long() == am[:, p]).sum()); tot += 64
+    assert 0.68 < hits / tot < 0.83
