@@ -19,9 +19,9 @@
  *    "host".  The library allocates no device memory.  Its only process-wide state is a set of
  *    per-device values looked up on first use and never changed afterwards (the opt-in shared
  *    memory limit, kernel attributes, resident-CTA counts, the device address of the built-in
- *    scratch array of bs_softmax_verify_noalloc) and that scratch array itself; the look-ups are
- *    not locked, so the very first calls on a device should not come from several host threads
- *    at once.
+ *    scratch array of bs_softmax_verify_noalloc) and that scratch array itself; the values are
+ *    held in atomics and every thread that finds one missing looks up the same answer, so calls
+ *    may come from several host threads.
  *  - `stream` is a cudaStream_t passed as void*.  Calls are asynchronous on that stream,
  *    never synchronise, and may be captured in a CUDA graph.
  *  - The return value covers host-side argument checks and launch errors only.  Problems

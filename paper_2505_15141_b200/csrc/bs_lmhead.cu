@@ -29,6 +29,7 @@
 //
 // Every mbarrier wait is bounded (about a second); a wait that gives up sets the abort word,
 // every role leaves its loop, the CTA meets at the final barrier and tensor memory is freed.
+#include <atomic>
 #include "bs_verify_common.cuh"
 #include "bs_pipeline.cuh"
 
@@ -532,7 +533,7 @@ static size_t lm_partial_bytes(int B, int Gmax, int V) {
     return align_up(sizeof(float2) * (size_t)B * (2 * Gmax + 1) * 2 * div_up(V, kLmBN), 256);
 }
 
-static bool g_lm_attr[4][64];
+static std::atomic<bool> g_lm_attr[4][64];
 
 template <int MH, int STAGES, bool GREEDY>
 static bs_status launch_lmhead(const CUtensorMap* tms, const LmParams& lp, const VerifyParams& vp,

@@ -7,6 +7,7 @@
 // The array lives on every GPU that loads the library, for the life of the process, and is shared
 // by all calls: two calls that run at the same time on one GPU would trample each other's row
 // partials and arrival counters.
+#include <atomic>
 #include "bs_common.cuh"
 
 namespace bs {
@@ -17,7 +18,7 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[BS_NOALLOC_SCRA
 
 // Device address of the array, per device.  In host code `g_noalloc_scratch` is only a handle of
 // the symbol: the address a kernel can use has to be asked for, with the device current.
-static void* g_scratch_ptr[64];
+static std::atomic<void*> g_scratch_ptr[64];
 
 static bs_status scratch_address(void** out) {
     int dev = 0;

@@ -22,6 +22,7 @@
 //
 // Every wait (mbarriers, the finisher's poll of the consumers' progress) is bounded; a wait that
 // gives up sets the abort word and the thread leaves.
+#include <atomic>
 #include "bs_residual_level2.cuh"
 #include "bs_pipeline.cuh"
 
@@ -255,8 +256,8 @@ __global__ void __launch_bounds__(kRsThreads, 2) residual_stream_kernel(const Re
     }
 }
 
-static int g_rs_smem[64];          // opt-in shared memory limit per device (0 = not queried)
-static bool g_rs_attr[2][64];
+static std::atomic<int> g_rs_smem[64];          // opt-in shared memory limit per device (0 = not queried)
+static std::atomic<bool> g_rs_attr[2][64];
 
 template <typename T>
 bs_status launch_residual_stream(const ResidParams& p, cudaStream_t st) {

@@ -9,6 +9,7 @@
 // and a scalar tail, reduced to (max, sum exp) with one exp per logit, and written as a
 // partial.  An arrival counter per sequence elects the CTA that merges the partials and runs
 // the accept scan.
+#include <atomic>
 #include "bs_verify_common.cuh"
 
 namespace bs {
@@ -165,15 +166,19 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const VerifyParams p) 
 
 thread_local int g_last_cuda_error = 0;
 
-static int g_occ[4][64];     // resident CTAs per SM per kernel variant, per device (0 = not queried)
-static int g_sms[64];
+static std::atomic<int> g_occ[4][64];     // resident CTAs per SM per kernel variant, per device (0 = not queried)
+static std::atomic<int> g_sms[64];
 
 int sm_count() {
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64) dev = 0;
-    if (!g_sms[dev]) cudaDeviceGetAttribute(&g_sms[dev], cudaDevAttrMultiProcessorCount, dev);
-    return g_sms[dev] > 0 ? g_sms[dev] : 148;
+    int n = g_sms[dev];
+    if (!n) {
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+        g_sms[dev] = n;
+    }
+    return n;
 }
 
 template <typename T, bool GREEDY>

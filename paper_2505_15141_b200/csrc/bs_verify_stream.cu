@@ -22,6 +22,7 @@
 // ticket per sequence; the finisher whose piece completes the count merges all rows of the
 // sequence (one lane per row) and runs the accept scan.  Nobody waits on another CTA.  All waits
 // on mbarriers are bounded; a wait that gives up sets the abort word and the thread leaves.
+#include <atomic>
 #include "bs_verify_common.cuh"
 #include "bs_pipeline.cuh"
 
@@ -333,8 +334,8 @@ __global__ void __launch_bounds__(kStreamThreads, 2) verify_stream_kernel(const 
     }
 }
 
-static int g_stream_smem[64];          // opt-in shared memory limit per device (0 = not queried)
-static bool g_attr_set[4][64];
+static std::atomic<int> g_stream_smem[64];          // opt-in shared memory limit per device (0 = not queried)
+static std::atomic<bool> g_attr_set[4][64];
 
 template <typename T, bool GREEDY>
 bs_status launch_verify_stream(const VerifyParams& p, cudaStream_t st) {

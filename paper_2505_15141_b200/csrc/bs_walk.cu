@@ -19,6 +19,7 @@
 //
 // CTAs of one group wait for one another, so the kernel is launched cooperatively (all CTAs
 // resident).  Every wait is bounded; a wait that gives up sets the abort word and the CTA drains.
+#include <atomic>
 #include "bs_walk_common.cuh"
 
 namespace bs {
@@ -538,7 +539,7 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_kernel(const WalkPa
     }
 }
 
-static int g_wk_blocks[4][64];        // resident CTAs per SM (0 = not queried)
+static std::atomic<int> g_wk_blocks[4][64];        // resident CTAs per SM (0 = not queried)
 
 template <typename T, bool GREEDY>
 static bs_status launch_walk(WalkParams& p, cudaStream_t st) {

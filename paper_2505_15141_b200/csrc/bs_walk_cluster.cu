@@ -22,6 +22,7 @@
 // counter and the decision word lived in the workspace, is what made early exit lose to the two-call path
 // on small batches.  A cluster waits for nobody outside itself, so the launch is an ordinary one.  Every
 // wait is bounded; a wait that gives up sets the abort word and the thread leaves.
+#include <atomic>
 #include "bs_walk_common.cuh"
 
 namespace bs {
@@ -598,8 +599,8 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_cluster_kernel(cons
     }
 }
 
-static int g_cl_smem[64];             // opt-in shared memory limit per device (0 = not queried)
-static int g_cl_max[4][4][64];        // resident clusters per kernel variant and cluster size 2 / 4 / 8 (0 = not queried, -1 = none)
+static std::atomic<int> g_cl_smem[64];             // opt-in shared memory limit per device (0 = not queried)
+static std::atomic<int> g_cl_max[4][4][64];        // resident clusters per kernel variant and cluster size 2 / 4 / 8 (0 = not queried, -1 = none)
 
 template <typename T, bool GREEDY>
 bs_status launch_walk_cluster(WalkParams& p, cudaStream_t st) {
@@ -620,7 +621,7 @@ bs_status launch_walk_cluster(WalkParams& p, cudaStream_t st) {
     if (nst > kWkStages) nst = kWkStages;
     if (nst < 2) return BS_ERR_UNSUPPORTED;
     const size_t smem = (size_t)nst * kSegBytes + extra;
-    static bool attr_set[4][64];
+    static std::atomic<bool> attr_set[4][64];
     if (!attr_set[variant][dev]) {
         if (cudaFuncSetAttribute(verify_walk_cluster_kernel<T, GREEDY>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  g_cl_smem[dev] - 12288) != cudaSuccess)
