@@ -643,6 +643,7 @@ static bs_status run_walk(const void* target_logits, const void* draft_logits, b
     // decision words: the second B words of the per-row counter slot (the first B mark drafted positions)
     p.dec = v.ticket_row + B;
     p.nG = 1;
+    p.look = 0;
     p.drafted = (drafted && !greedy) ? 1 : 0;         // greedy rounds never read draft rows anyway
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // groups of 2, 4 or 8 CTAs as thread-block clusters (hand-offs through distributed shared memory); rows of a

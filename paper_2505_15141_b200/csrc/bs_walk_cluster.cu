@@ -6,29 +6,33 @@
 // interleaves them.  For position k every CTA streams its contiguous share of target row k and draft row k
 // (bulk async copies into a ring of 32 KB stages, 16 consumer warps, online softmax: the pipeline of the
 // row-statistics kernel).  Its finisher warp merges what its consumers produced and sends ONE message per
-// position -- the (max, Z) of its part of either row -- into the mailbox of the cluster's first CTA, the
+// position -- the (max, Z) of its part of either row -- into a mailbox of the cluster's first CTA, the
 // leader of all the cluster's sequences, and arrives on the mailbox's mbarrier there.  The leader's finisher
-// merges the nG messages, tests r <= min{1, P/Q} for the drafted token (the token's two logits were asked
-// for when the previous position was decided) and writes the decision, with the constants of the residual
-// pass if this is the stop, into the shared memory of every CTA of the cluster, arriving on their decision
-// barriers.  Their producers, which wait on those local barriers, stream position k + 1, or -- at the first
-// rejection, or after the bonus row when everything passed -- the row pair of the stop position again (it
-// has just been read: L2) for the residual masses; when every CTA has reported its share of the masses the
-// leader runs the inverse CDF (level 2 of the resampling kernel).  In greedy mode only target rows are
+// merges the nG messages, tests r <= min{1, P/Q} for the drafted token (the two logits at every drafted token
+// were asked for when the kernel started) and writes the decision word of the sequence -- at the stop preceded
+// by the constants of the residual pass -- into the shared memory of every CTA of the cluster.
+//
+// The producers do not wait for a decision before they stream the next position: a sequence may run up to
+// `look` positions ahead of its last decided one (a mailbox per position in flight), so the decision on
+// position k has to be in only before position k + look + 1 is due, and the chain "last byte reduced ->
+// message -> decision -> first copy of the next position" is off the critical path.  What was streamed
+// behind the stop is wasted (at most what the ring holds per CTA, since decisions are quick).  At the first
+// rejection, or after the bonus row when everything passed, the producers stream the row pair of the stop
+// position again (it has just been read: L2) for the residual masses; when every CTA has reported its share
+// the leader runs the inverse CDF (level 2 of the resampling kernel).  In greedy mode only target rows are
 // streamed, the message carries (max, arg-max), and the leader emits the arg-max of the stop row itself.
 //
-// No trip through L2 lies between "the last byte of a position has been reduced" and "the first copy of the
-// next position is issued": that chain, about ten microseconds per position when the partials, the arrival
-// counter and the decision word lived in the workspace, is what made early exit lose to the two-call path
-// on small batches.  A cluster waits for nobody outside itself, so the launch is an ordinary one.  Every
-// wait is bounded; a wait that gives up sets the abort word and the thread leaves.
+// A cluster waits for nobody outside itself, so the launch is an ordinary one.  Every wait is bounded; a
+// wait that gives up sets the abort word and the thread leaves.  Messages of positions behind a stop may
+// arrive after the leader is through with the sequence: every CTA stays until the whole cluster is done.
 #include <atomic>
 #include "bs_walk_common.cuh"
 
 namespace bs {
 
-constexpr int kClMaxSeqs = 32;                                   // sequences of one cluster (one lane of the leader each)
+constexpr int kClMaxSeqs = 16;                                   // sequences of one cluster (one lane of the leader each)
 constexpr int kClMaxCtas = 8;
+constexpr int kClLevels = 4;                                     // mailboxes per sequence: positions that may be in flight at once
 
 struct ClMeta {                                                  // per-stage record, written by the producer
     int type, slot, b, k;
@@ -38,17 +42,16 @@ struct ClMeta {                                                  // per-stage re
     float kt, kd, at, ad;
 };
 struct ClEvent {                                                 // per event handed to the finisher (consumer warp 0)
-    int type, slot, row, flags;
+    int type, slot, row, flags, k;
 };
 struct __align__(16) ClMail {                                    // one CTA's part of a position: target row, draft row
     float mt, zt, md, zd;                                        // greedy: (max, arg-max bits) in mt, zt
 };
-struct __align__(16) ClDec {                                     // the leader's decision on a position
-    unsigned word;         // (positions decided << 1) | accepted
-    float kt, kd, at, ad;  // at the stop: the constants of the residual pass
-    int bonus, pad0, pad1;
+struct __align__(16) ClDec {                                     // what the leader's stop decision carries
+    float kt, kd, at, ad;  // the constants of the residual pass
+    int bonus, pad0, pad1, pad2;
 };
-struct ClPre {                                                   // what the next decision of a sequence will need
+struct __align__(16) ClPre {                                     // what the decision on one position of a sequence needs
     unsigned tw, dw;       // the 4-byte words that hold the target / draft logit at the drafted token
     float2 ds;             // drafted mode: the draft row's statistics
 };
@@ -87,6 +90,21 @@ __device__ __forceinline__ bool cl_try_wait(uint32_t bar, uint32_t parity) {    
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+// The decision word of a sequence: written by the leader into every CTA after whatever the decision carries,
+// polled by that CTA's producer.
+__device__ __forceinline__ void cl_st_release(uint32_t ra, unsigned v) {
+    asm volatile("st.release.cluster.shared::cluster.u32 [%0], %1;" ::"r"(ra), "r"(v) : "memory");
+}
+__device__ __forceinline__ unsigned cl_ld_acquire(const unsigned* local) {
+    unsigned v;
+    asm volatile("ld.acquire.cluster.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(local)) : "memory");
+    return v;
+}
+// Before a CTA exits: nothing written into its shared memory by another CTA of the cluster is still under way
+// (messages of positions behind a stop arrive after the leader has finished with the sequence).
+__device__ __forceinline__ void cl_sync_exit() {
+    asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
+}
 __device__ __forceinline__ void cl_sync_all() {                  // every thread of every CTA of the cluster
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
@@ -110,27 +128,29 @@ template <> __device__ __forceinline__ float value_of<__nv_bfloat16>(unsigned w,
     return __uint_as_float((x & 1) ? (w & 0xffff0000u) : (w << 16));
 }
 
+// The roles leave this function where their work ends; the kernel around it holds the cluster together until
+// every CTA is through.
 template <typename T, bool GREEDY>
-__global__ void __launch_bounds__(kWkThreads, 2) verify_walk_cluster_kernel(const WalkParams p, const int nstages,
-                                                                            const int nclusters) {
+__device__ __forceinline__ void walk_cluster_body(const WalkParams& p, const int nstages, const int nclusters) {
     extern __shared__ __align__(128) unsigned char dsm[];
-    // layout: [nstages * 32 KB ring][tokens 32 x Gmax][uniforms 32 x Gmax]   (the last two used by the leader only)
+    // layout: [nstages * 32 KB ring][tokens 16 x Gmax][uniforms 16 x Gmax][token logits 16 x Gmax]   (the last three
+    // used by the leader only)
     unsigned char* ring = dsm;
     const VerifyParams& v = p.v;
     const int GP = v.Gmax > 0 ? v.Gmax : 1;
     int* s_tok = reinterpret_cast<int*>(dsm + (size_t)nstages * kSegBytes);
     float* s_u = reinterpret_cast<float*>(s_tok + kClMaxSeqs * GP);
+    ClPre* s_pre = reinterpret_cast<ClPre*>(s_u + kClMaxSeqs * GP);
     __shared__ __align__(8) unsigned long long s_full[kWkStages];
     __shared__ __align__(8) unsigned long long s_empty[kWkStages];
     __shared__ __align__(8) unsigned long long s_evbar[kWkRing];
     __shared__ __align__(8) unsigned long long s_evfree[kWkRing];
-    __shared__ __align__(8) unsigned long long s_mailbar[kClMaxSeqs];   // leader: nG messages per position
+    __shared__ __align__(8) unsigned long long s_mailbar[kClMaxSeqs][kClLevels];   // leader: nG messages per position
     __shared__ __align__(8) unsigned long long s_massbar[kClMaxSeqs];   // leader: nG shares of the residual masses
-    __shared__ __align__(8) unsigned long long s_decbar[kClMaxSeqs];    // every CTA: the leader's decision
-    __shared__ ClMail s_mail[kClMaxSeqs][kClMaxCtas];
-    __shared__ ClDec s_dec[kClMaxSeqs];
-    __shared__ ClMail s_acc[kClMaxSeqs];                      // this CTA's part of the position a sequence is at
-    __shared__ ClPre s_pre[kClMaxSeqs];
+    __shared__ ClMail s_mail[kClMaxSeqs][kClLevels][kClMaxCtas];        // position k of a sequence uses level k % kClLevels
+    __shared__ ClDec s_dec[kClMaxSeqs];                       // every CTA: what the stop decision carries
+    __shared__ unsigned s_decword[kClMaxSeqs];                // every CTA: (positions decided << 1) | last one accepted
+    __shared__ ClMail s_acc[kClMaxSeqs];                      // this CTA's part of the position it is streaming
     __shared__ ClMeta s_meta[kWkStages];
     __shared__ ClEvent s_ev[kWkRing];
     __shared__ float2 s_red[kWkRing][kWkWarps];
@@ -156,13 +176,15 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_cluster_kernel(cons
             mbar_init(smem_u32(&s_evfree[s]), 1);
         }
         for (int s = 0; s < kClMaxSeqs; ++s) {
-            mbar_init(smem_u32(&s_mailbar[s]), (uint32_t)nG);
+            for (int l = 0; l < kClLevels; ++l) mbar_init(smem_u32(&s_mailbar[s][l]), (uint32_t)nG);
             mbar_init(smem_u32(&s_massbar[s]), (uint32_t)nG);
-            mbar_init(smem_u32(&s_decbar[s]), 1);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (tid < kClMaxSeqs) s_acc[tid] = ClMail{-INFINITY, GREEDY ? __int_as_float(INT_MAX) : 0.f, -INFINITY, 0.f};
+    if (tid < kClMaxSeqs) {
+        s_acc[tid] = ClMail{-INFINITY, GREEDY ? __int_as_float(INT_MAX) : 0.f, -INFINITY, 0.f};
+        s_decword[tid] = 0u;
+    }
     __syncthreads();
     cl_sync_all();                                            // nobody touches a barrier of a CTA that has not set it up
     pdl_enter();                                              // gamma comes from the kernel before this one
@@ -170,8 +192,8 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_cluster_kernel(cons
     if (warp == kWkWarps) {
         // =============================== producer ===============================
         // Keeps the cluster's sequences moving in this CTA: streams whatever is ready and only sleeps when every
-        // sequence is waiting for the leader's decision.
-        if (lane != 0) return;
+        // sequence is waiting for the leader's decision.  One lane works; the warp meets again before it leaves.
+        if (lane == 0) [&]() {
         int slot = 0;
         uint32_t ph = 0;
         bool ok = true;
@@ -190,51 +212,51 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_cluster_kernel(cons
             if (++slot == nstages) { slot = 0; ph ^= 1u; }
             return true;
         };
-        // s_pstate[s] = k | stage << 8; stage 0: position k to be streamed, 1: waiting for its decision, 2: done
+        // s_pstate[s] = the next position to stream | done << 8.  A position is streamed as soon as the ring takes
+        // it, up to p.look positions past the last decided one: the decision on position k then only has to be in
+        // before position k + look + 1 is due, instead of before k + 1.  What was streamed behind a stop is wasted.
         for (int s = 0; s < nslots; ++s) s_pstate[s] = 0;
         int alive = nslots;
         long long t_last = clock64();
         while (alive > 0 && ok) {
             bool progress = false;
             for (int s = 0; s < nslots && ok; ++s) {
-                int k = s_pstate[s] & 0xff, stg = s_pstate[s] >> 8;
-                if (stg == 2) continue;
+                if (s_pstate[s] >> 8) continue;
+                const int ks = s_pstate[s];
                 const int b = (int)cid + s * nclusters;
                 const int g = clamp_gamma(v.gamma[b], v.Gmax);
-                if (stg == 1) {
-                    // ---- has the leader decided position k? ----
-                    if (!cl_try_wait(smem_u32(&s_decbar[s]), (uint32_t)k & 1u)) continue;
-                    const ClDec d = s_dec[s];
-                    progress = true;
-                    if (k < g && (d.word & 1u)) {              // accepted: on to the next position
-                        k += 1;
-                        stg = 0;
-                    } else {
-                        if (!GREEDY) {
-                            // ---- stop at k: this CTA's share of the residual [P_k - Q_k]_+ (rejected) or of P_k (bonus) ----
-                            const bool bonus = d.bonus != 0;
-                            const T* tp = row_ptr(static_cast<const T*>(v.target), b, v.Gmax + 1, k, v.V);
-                            const T* dp = bonus ? nullptr : row_ptr(static_cast<const T*>(v.draft), b, v.Gmax, k, v.V);
-                            const int rseg = p.r.seg, rnseg = p.r.nseg;
-                            const int j0 = (int)((long long)rnseg * rank / nG), j1 = (int)((long long)rnseg * (rank + 1) / nG);
-                            for (int sg = j0; sg < j1 && ok; ++sg) {
-                                const int e0 = sg * rseg;
-                                const int n = min(rseg, v.V - e0);
-                                ClMeta m;
-                                m.type = kItemMass; m.slot = s; m.b = b; m.k = k; m.row = bonus ? 1 : 0; m.sg = sg;
-                                m.nvec = n / kVec;
-                                m.flags = (sg == j0 ? 1 : 0) | (sg == j1 - 1 ? 2 : 0);
-                                m.kt = d.kt; m.kd = d.kd; m.at = d.at; m.ad = d.ad;
-                                ok = issue(m, tp + e0, bonus ? nullptr : dp + e0, (uint32_t)n * (uint32_t)sizeof(T));
-                            }
+                const unsigned w = cl_ld_acquire(&s_decword[s]);
+                const int nd = (int)(w >> 1);                  // positions decided
+                if (nd > 0 && !(w & 1u)) {
+                    // ---- stop at k = nd - 1: this CTA's share of the residual [P_k - Q_k]_+ (rejected) or of P_k (bonus) ----
+                    const int k = nd - 1;
+                    if (!GREEDY) {
+                        const ClDec d = s_dec[s];
+                        const bool bonus = d.bonus != 0;
+                        const T* tp = row_ptr(static_cast<const T*>(v.target), b, v.Gmax + 1, k, v.V);
+                        const T* dp = bonus ? nullptr : row_ptr(static_cast<const T*>(v.draft), b, v.Gmax, k, v.V);
+                        const int rseg = p.r.seg, rnseg = p.r.nseg;
+                        const int j0 = (int)((long long)rnseg * rank / nG), j1 = (int)((long long)rnseg * (rank + 1) / nG);
+                        for (int sg = j0; sg < j1 && ok; ++sg) {
+                            const int e0 = sg * rseg;
+                            const int n = min(rseg, v.V - e0);
+                            ClMeta m;
+                            m.type = kItemMass; m.slot = s; m.b = b; m.k = k; m.row = bonus ? 1 : 0; m.sg = sg;
+                            m.nvec = n / kVec;
+                            m.flags = (sg == j0 ? 1 : 0) | (sg == j1 - 1 ? 2 : 0);
+                            m.kt = d.kt; m.kd = d.kd; m.at = d.at; m.ad = d.ad;
+                            ok = issue(m, tp + e0, bonus ? nullptr : dp + e0, (uint32_t)n * (uint32_t)sizeof(T));
                         }
-                        --alive;
-                        s_pstate[s] = k | (2 << 8);
-                        continue;
                     }
+                    --alive;
+                    s_pstate[s] = 1 << 8;
+                    progress = true;
+                    continue;
                 }
-                // ---- position k: this CTA's share of target row k and, below gamma, draft row k ----
+                if (ks > g || ks > nd + p.look) continue;      // everything streamed, or far enough ahead of the decisions
+                // ---- position ks: this CTA's share of target row ks and, below gamma, draft row ks ----
                 {
+                    const int k = ks;
                     const int nrows = (!GREEDY && !p.drafted && k < g) ? 2 : 1;
                     const int items = nrows * v.nseg;
                     const int i0 = (int)((long long)items * rank / nG), i1 = (int)((long long)items * (rank + 1) / nG);
@@ -252,7 +274,7 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_cluster_kernel(cons
                         ok = issue(m, rowp + e0, nullptr, (uint32_t)n * (uint32_t)sizeof(T));
                     }
                     progress = true;
-                    s_pstate[s] = k | (1 << 8);
+                    s_pstate[s] = k + 1;
                 }
             }
             if (progress) {
@@ -267,6 +289,8 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_cluster_kernel(cons
         e.type = kItemEnd; e.slot = 0; e.b = 0; e.k = 0; e.row = 0; e.sg = 0; e.nvec = 0; e.flags = 2;
         e.kt = e.kd = 0.f; e.at = e.ad = 1.f;
         issue(e, nullptr, nullptr, 0);
+        }();
+        __syncwarp();
         return;
     }
 
@@ -275,7 +299,7 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_cluster_kernel(cons
         const bool leader = rank == 0;
         int remaining = leader ? nslots : 0;                  // leader: sequences not yet finished
         if (leader) {
-            // ---- every sequence starts at position 0: tokens and uniforms into shared memory, the first two logits asked for ----
+            // ---- tokens and uniforms into shared memory; the two logits at every drafted token asked for ----
             for (int s = 0; s < nslots; ++s) {
                 const int b = (int)cid + s * nclusters;
                 const int graw = v.gamma[b];
@@ -293,23 +317,28 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_cluster_kernel(cons
                 }
             }
             __syncwarp();
-            if (!GREEDY && lane < nslots) {
-                const int s = lane;
-                const int b = (int)cid + s * nclusters;
-                const int g = clamp_gamma(v.gamma[b], v.Gmax);
-                ClPre pre{0u, 0u, make_float2(0.f, 1.f)};
-                if (g > 0) {
-                    const int x = s_tok[s * GP];
+            if (!GREEDY) {
+                // asynchronous 4- and 8-byte copies, waited for before the first decision: by then they have landed
+                for (int i = lane; i < nslots * GP; i += 32) {
+                    const int s = i / GP, j = i - s * GP;
+                    const int b = (int)cid + s * nclusters;
+                    const int g = clamp_gamma(v.gamma[b], v.Gmax);
+                    // a field is written either here or by its copy, never by both
+                    const int x = j < g ? s_tok[i] : -1;
                     if (x >= 0 && x < v.V) {
-                        pre.tw = __ldg(static_cast<const unsigned*>(word_of<T>(row_ptr(static_cast<const T*>(v.target), b, v.Gmax + 1, 0, v.V), x)));
-                        pre.dw = __ldg(static_cast<const unsigned*>(word_of<T>(row_ptr(static_cast<const T*>(v.draft), b, v.Gmax, 0, v.V), x)));
+                        cp_async4(&s_pre[i].tw, word_of<T>(row_ptr(static_cast<const T*>(v.target), b, v.Gmax + 1, j, v.V), x));
+                        cp_async4(&s_pre[i].dw, word_of<T>(row_ptr(static_cast<const T*>(v.draft), b, v.Gmax, j, v.V), x));
+                    } else {
+                        s_pre[i].tw = 0u;
+                        s_pre[i].dw = 0u;
                     }
-                    if (p.drafted) pre.ds = __ldcg(v.row_stats + (size_t)b * v.R + v.Gmax + 1);
+                    if (j < g && p.drafted) cp_async8(&s_pre[i].ds, v.row_stats + (size_t)b * v.R + v.Gmax + 1 + j);
+                    else s_pre[i].ds = make_float2(0.f, 1.f);
                 }
-                s_pre[s] = pre;
             }
             __syncwarp();
         }
+        bool pre_landed = GREEDY;                             // leader: the copies above have been waited for
 
         bool ended = false;
         int ev = 0;
@@ -348,8 +377,9 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_cluster_kernel(cons
                             if (e.flags & 4) {
                                 // the CTA's share of the position is complete: one message to the leader
                                 const ClMail a = s_acc[e.slot];
-                                cl_st_v4(cl_map(&s_mail[e.slot][rank], 0), a.mt, a.zt, a.md, a.zd);
-                                cl_arrive(cl_map(&s_mailbar[e.slot], 0));
+                                const int lv = e.k % kClLevels;
+                                cl_st_v4(cl_map(&s_mail[e.slot][lv][rank], 0), a.mt, a.zt, a.md, a.zd);
+                                cl_arrive(cl_map(&s_mailbar[e.slot][lv], 0));
                                 s_acc[e.slot] = ClMail{-INFINITY, GREEDY ? __int_as_float(INT_MAX) : 0.f, -INFINITY, 0.f};
                             }
                         }
@@ -361,7 +391,10 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_cluster_kernel(cons
             if (leader && remaining > 0) {
                 const int st = lane < nslots ? s_lstate[lane] : 0;
                 bool r = false;
-                if (st == 1) r = cl_try_wait(smem_u32(&s_mailbar[lane]), (uint32_t)s_lk[lane] & 1u);
+                if (st == 1) {
+                    const int kl = s_lk[lane];
+                    r = cl_try_wait(smem_u32(&s_mailbar[lane][kl % kClLevels]), (uint32_t)(kl / kClLevels) & 1u);
+                }
                 else if (st == 2) r = cl_try_wait(smem_u32(&s_massbar[lane]), 0u);
                 unsigned todo = __ballot_sync(0xffffffffu, r);
                 while (todo) {
@@ -391,9 +424,9 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_cluster_kernel(cons
                         continue;
                     }
                     // ---- position k: merge the nG messages, decide ----
-                    cl_try_wait(smem_u32(&s_mailbar[s]), (uint32_t)k & 1u);   // every lane acquires the messages
+                    cl_try_wait(smem_u32(&s_mailbar[s][k % kClLevels]), (uint32_t)(k / kClLevels) & 1u);   // every lane acquires the messages
                     ClMail ml{-INFINITY, GREEDY ? __int_as_float(INT_MAX) : 0.f, -INFINITY, 0.f};
-                    if (lane < nG) ml = s_mail[s][lane];
+                    if (lane < nG) ml = s_mail[s][k % kClLevels][lane];
                     int bits = 0;
                     bool acc = false;
                     float pj = 0.f, qj = 0.f;
@@ -411,9 +444,12 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_cluster_kernel(cons
                         const float Zt = warp_sum(ml.zt * rescale(ml.mt, Mt, v.c));
                         ts = make_float2(Mt, Zt);
                         if (!(Zt > 0.f) || !isfinite(Zt) || !isfinite(Mt)) bits |= BS_DEV_NONFINITE;
-                        if (lane == 0) cp_async_wait_all();            // the logits asked for when k - 1 was decided
-                        __syncwarp();
-                        const ClPre pre = s_pre[s];
+                        if (!pre_landed) {                             // the logits asked for at the start
+                            cp_async_wait_all();
+                            __syncwarp();
+                            pre_landed = true;
+                        }
+                        const ClPre pre = k < g ? s_pre[s * GP + k] : ClPre{0u, 0u, make_float2(0.f, 1.f)};
                         bool missing = false;
                         if (k < g) {
                             if (p.drafted) {
@@ -439,18 +475,20 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_cluster_kernel(cons
                         }
                     }
                     // ---- the decision goes to every CTA of the cluster first: they are what waits ----
+                    const unsigned word = ((unsigned)(k + 1) << 1) | (acc ? 1u : 0u);
                     ClDec d;
-                    d.word = ((unsigned)(k + 1) << 1) | (acc ? 1u : 0u);
-                    d.kt = d.kd = 0.f; d.at = d.ad = 1.f; d.bonus = k >= g; d.pad0 = d.pad1 = 0;
+                    d.kt = d.kd = 0.f; d.at = d.ad = 1.f; d.bonus = k >= g; d.pad0 = d.pad1 = d.pad2 = 0;
                     if (!acc && !GREEDY) {
                         MassFn::fold(ts.x, ts.y, v.c, d.kt, d.at);
                         if (k < g) MassFn::fold(ds.x, ds.y, v.c, d.kd, d.ad);
                     }
                     if (lane < nG) {
-                        const uint32_t ra = cl_map(&s_dec[s], (uint32_t)lane);
-                        cl_st_v4u(ra, d.word, __float_as_uint(d.kt), __float_as_uint(d.kd), __float_as_uint(d.at));
-                        cl_st_v4u(ra + 16u, __float_as_uint(d.ad), (unsigned)d.bonus, 0u, 0u);
-                        cl_arrive(cl_map(&s_decbar[s], (uint32_t)lane));
+                        if (!acc && !GREEDY) {
+                            const uint32_t ra = cl_map(&s_dec[s], (uint32_t)lane);
+                            cl_st_v4(ra, d.kt, d.kd, d.at, d.ad);
+                            cl_st_v4u(ra + 16u, (unsigned)d.bonus, 0u, 0u, 0u);
+                        }
+                        cl_st_release(cl_map(&s_decword[s], (uint32_t)lane), word);   // after what it carries
                     }
                     // ---- then the outputs and what the next decision will need ----
                     if (lane == 0) {
@@ -464,14 +502,6 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_cluster_kernel(cons
                         }
                         if (acc) {
                             s_lk[s] = k + 1;
-                            if (!GREEDY && k + 1 < g) {
-                                const int xn = s_tok[s * GP + k + 1];
-                                if (xn >= 0 && xn < v.V) {
-                                    cp_async4(&s_pre[s].tw, word_of<T>(row_ptr(static_cast<const T*>(v.target), b, v.Gmax + 1, k + 1, v.V), xn));
-                                    cp_async4(&s_pre[s].dw, word_of<T>(row_ptr(static_cast<const T*>(v.draft), b, v.Gmax, k + 1, v.V), xn));
-                                }
-                                if (p.drafted) cp_async8(&s_pre[s].ds, v.row_stats + (size_t)b * v.R + v.Gmax + 1 + k + 1);
-                            }
                         } else {
                             v.accept_len[b] = k;                     // first rejection, or k == gamma: everything passed
                             v.status[b] = bits;
@@ -590,13 +620,20 @@ __global__ void __launch_bounds__(kWkThreads, 2) verify_walk_cluster_kernel(cons
             }
             if (lane == 0) {
                 s_red[rs][warp] = wr;
-                if (warp == 0) s_ev[rs] = ClEvent{m.type, m.slot, m.row, m.flags};
+                if (warp == 0) s_ev[rs] = ClEvent{m.type, m.slot, m.row, m.flags, m.k};
                 mbar_arrive(smem_u32(&s_evbar[rs]));          // release: the writes above are visible to the finisher
             }
             ++ev;
             if (m.type == kItemEnd) return;
         }
     }
+}
+
+template <typename T, bool GREEDY>
+__global__ void __launch_bounds__(kWkThreads, 2) verify_walk_cluster_kernel(const WalkParams p, const int nstages,
+                                                                            const int nclusters) {
+    walk_cluster_body<T, GREEDY>(p, nstages, nclusters);
+    cl_sync_exit();
 }
 
 static std::atomic<int> g_cl_smem[64];             // opt-in shared memory limit per device (0 = not queried)
@@ -615,8 +652,8 @@ bs_status launch_walk_cluster(WalkParams& p, cudaStream_t st) {
     }
     const int variant = (Elem<T>::kDtype == BS_F32 ? 0 : 2) + (GREEDY ? 1 : 0);
     const int GP = p.v.Gmax > 0 ? p.v.Gmax : 1;
-    const size_t extra = (size_t)kClMaxSeqs * GP * (sizeof(int) + sizeof(float));
-    const size_t budget = (size_t)(g_cl_smem[dev] + 1024) / 2 - 12288;          // two CTAs per SM, minus the static part
+    const size_t extra = (size_t)kClMaxSeqs * GP * (sizeof(int) + sizeof(float) + sizeof(ClPre));
+    const size_t budget = (size_t)(g_cl_smem[dev] + 1024) / 2 - 13312;          // two CTAs per SM, minus the static part
     int nst = (int)((budget - extra) / kSegBytes);
     if (nst > kWkStages) nst = kWkStages;
     if (nst < 2) return BS_ERR_UNSUPPORTED;
@@ -624,7 +661,7 @@ bs_status launch_walk_cluster(WalkParams& p, cudaStream_t st) {
     static std::atomic<bool> attr_set[4][64];
     if (!attr_set[variant][dev]) {
         if (cudaFuncSetAttribute(verify_walk_cluster_kernel<T, GREEDY>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 g_cl_smem[dev] - 12288) != cudaSuccess)
+                                 g_cl_smem[dev] - 13312) != cudaSuccess)
             return cuda_status(cudaGetLastError());
         attr_set[variant][dev] = true;
     }
@@ -671,6 +708,7 @@ bs_status launch_walk_cluster(WalkParams& p, cudaStream_t st) {
     const int maxc = max_clusters(nG, cfg);
     const int nclusters = p.v.B < maxc ? p.v.B : maxc;
     p.nG = nG;
+    p.look = kClLevels - 1;
     cfg.gridDim = dim3((unsigned)(nclusters * nG));
     return cuda_status(cudaLaunchKernelEx(&cfg, verify_walk_cluster_kernel<T, GREEDY>, p, nst, nclusters));
 }

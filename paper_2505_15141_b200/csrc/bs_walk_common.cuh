@@ -24,6 +24,7 @@ struct WalkParams {
     uint32_t* dec;         // [B] decision word: (positions decided << 1) | last one accepted
     int nG;                // CTAs per sequence
     int drafted;           // 1: the draft rows' statistics were left by bs_draft_sample: stream target rows only
+    int look;              // cluster kernel: positions a sequence may be streamed past its last decided one
 };
 
 // Per-stage record, written by the producer.
