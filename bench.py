@@ -578,6 +578,27 @@ def run_cuda(args, w):
         peak, peak_src = FALLBACK_HBM_GBS, "fallback"
     achieved = verify_bytes / (verify_ms * 1e-3) / 1e9
 
+    # ---- the same call launched back to back on the rotating input sets, one event pair around the lot: what a
+    # launch takes in a busy stream.  An event pair around ONE short launch (the figure above) also times the
+    # gap before the kernel starts and the event itself, 4-5 us that no kernel change can touch. ----
+    back_to_back = None
+    if not walk and not drafted:
+        nb = min(args.steps, 50)
+        for i in range(3):
+            verify_call(sets[i % ring])
+        a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record(stream)
+        for i in range(nb):
+            verify_call(sets[(3 + i) % ring])
+        b_.record(stream)
+        torch.cuda.synchronize()
+        gm = gamma_d.to(torch.int64)
+        b2b_bytes = float((gm + 1).sum().item() if w.temperature == 0.0 else (2 * gm + 1).sum().item()) * V * es
+        b2b_ms = a.elapsed_time(b_) / nb
+        back_to_back = {"launches": nb, "ms_per_launch": b2b_ms, "bytes_per_launch": b2b_bytes,
+                        "achieved": b2b_bytes / (b2b_ms * 1e-3) / 1e9, "frac": b2b_bytes / (b2b_ms * 1e-3) / 1e9 / peak}
+
     # ---- the same rounds through the early-exit entry point, for comparison (plain runs only) ----
     variants = None
     if not walk and not drafted and w.temperature > 0.0:
@@ -674,10 +695,9 @@ def run_cuda(args, w):
                          "traffic": ncu_traffic(w.name, verify_bytes), "bytes_per_launch": verify_bytes,
                          "nominal_peak": 8000.0, "frac_of_nominal": achieved / 8000.0,
                          "ms_per_launch": verify_ms, "residual_ms_per_launch": resid_ms,
-                         # The second call of the round.  In sampling mode the statistics kernel computes the
-                         # residual masses of most stop rows itself (second touch, out of L2), so what is left
-                         # for bs_residual_sample is the inverse CDF; `stop_row_bytes` are the rows it would
-                         # have to stream if none of that had happened.
+                         "back_to_back": back_to_back,
+                         # The second call of the round; `stop_row_bytes` are the rows it streams again (the row
+                         # pair of a rejected position, or the bonus row alone).
                          "residual": (None if walk or resid_bytes <= 0 else
                                       {"kernel": "residual_stream_kernel (bs_residual_sample)",
                                        "ms_per_launch": resid_ms, "stop_row_bytes": resid_bytes}),
@@ -1190,7 +1210,7 @@ def other_workloads_summary():
             out[name] = {"value": d["value"], "unit": d["unit"], "ms_per_step": d["ms_per_step"],
                          "algorithmic_gbs": d.get("algorithmic_gbs"),
                          "roofline": {k: r.get(k) for k in ("bound", "kernel", "achieved", "peak", "unit", "frac",
-                                                            "ms_per_launch", "residual_ms_per_launch")},
+                                                            "ms_per_launch", "residual_ms_per_launch", "back_to_back")},
                          "variants": d.get("variants")}
         except Exception as e:                                   # the main line must not depend on these
             out[name] = {"error": f"{type(e).__name__}: {e}"[:200]}

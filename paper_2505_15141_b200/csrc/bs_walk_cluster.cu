@@ -665,10 +665,6 @@ bs_status launch_walk_cluster(WalkParams& p, cudaStream_t st) {
             return cuda_status(cudaGetLastError());
         attr_set[variant][dev] = true;
     }
-    // Cluster size: about 3.5 sequences per cluster, so that a long run of accepted drafts keeps a slice of many
-    // CTAs busy instead of one whole CTA.  (A cluster per sequence was tried for small batches -- four CTAs each on
-    // 64 x 128256 bf16 instead of eight CTAs on two sequences -- and gave the same 11 us per position: the two
-    // stages less per CTA and position cost as much as the queueing behind the other sequence's stages saved.)
     auto max_clusters = [&](int nG, cudaLaunchConfig_t& cfg) -> int {
         const int gi = nG == 8 ? 2 : (nG == 4 ? 1 : 0);
         if (!g_cl_max[variant][gi][dev]) {
@@ -693,22 +689,29 @@ bs_status launch_walk_cluster(WalkParams& p, cudaStream_t st) {
     at[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
     cfg.numAttrs = 2;
+    // Cluster size (measured on 64 to 256 sequences of 256 KB and 608 KB rows): four CTAs per sequence unless the
+    // rows are long enough to give eight CTAs four stages each per position AND the batch is small enough for
+    // at most two sequences per cluster (with more, clusters of eight measured 25 to 40 % slower than clusters of
+    // four); two where a row has fewer than four segments.  A cluster holds at most kClMaxSeqs sequences.
     int top = 8;
     while (top > p.v.nseg || top > p.r.nseg) top >>= 1;        // every CTA of a cluster gets a segment of every row
     int nG = 0;
-    const int want = (int)((7LL * 2 * sm_count() + p.v.B) / (2LL * p.v.B));
-    for (int c = want >= 8 ? 8 : (want >= 4 ? 4 : 2); c >= 2 && !nG; c >>= 1) {
-        if (c > top) continue;
+    for (int c = top; c >= 2 && !nG; c >>= 1) {
         at[0].val.clusterDim.x = (unsigned)c;
         const int maxc = max_clusters(c, cfg);
-        if (maxc >= 1 && (p.v.B + maxc - 1) / maxc <= kClMaxSeqs) nG = c;   // else too many sequences per cluster: smaller clusters
+        if (maxc < 1 || (p.v.B + maxc - 1) / maxc > kClMaxSeqs) continue;
+        if (c == 8 && (p.v.nseg < 16 || p.v.B > 2 * maxc)) continue;
+        nG = c;
     }
     if (!nG) return BS_ERR_UNSUPPORTED;
     at[0].val.clusterDim.x = (unsigned)nG;
     const int maxc = max_clusters(nG, cfg);
     const int nclusters = p.v.B < maxc ? p.v.B : maxc;
     p.nG = nG;
-    p.look = kClLevels - 1;
+    // How far a sequence may run ahead of its decisions: all the mailboxes while a cluster has one or two
+    // sequences (the CTAs would idle otherwise), one position once it interleaves several (they keep the CTAs
+    // busy, and what is streamed behind a stop is DRAM bandwidth the other sequences lack).
+    p.look = 2 * p.v.B <= 3 * nclusters ? kClLevels - 1 : 1;
     cfg.gridDim = dim3((unsigned)(nclusters * nG));
     return cuda_status(cudaLaunchKernelEx(&cfg, verify_walk_cluster_kernel<T, GREEDY>, p, nst, nclusters));
 }
