@@ -183,9 +183,11 @@ bs_status bs_softmax_verify_noalloc(const void* target_logits, const void* draft
 
 /* Algorithm 6 from its second line on in the algorithm's own order: position after position,
  * stopping at the first rejection (its "break"), then the resampling step -- bs_softmax_verify
- * followed by bs_residual_sample, but rows behind the first rejected draft are never read: a
+ * followed by bs_residual_sample, but rows behind the first rejected draft are not needed: a
  * sequence that stops at position tau costs 2 (tau + 1) rows (2 gamma + 1 when everything
  * passes) plus a second pass over the rows of the stop position, instead of 2 gamma + 1 + 2.
+ * (The kernel may stream a sequence up to three positions ahead of its last decision, so a few
+ * rows behind the stop can be read all the same; they change no result.)
  *
  *  arguments as bs_softmax_verify and bs_residual_sample (temperature 0 = greedy mode: target rows
  *  only, the emitted token is the arg-max of the stop row, draft logits and uniforms may be NULL)
@@ -193,8 +195,9 @@ bs_status bs_softmax_verify_noalloc(const void* target_logits, const void* draft
  *                (j <= tau_b, j < gamma_b); the entries behind the stop are set to 0 (all of them
  *                in greedy mode)
  *  accept_len, out_tokens, out_len: as the two separate calls
- * The CTAs that share a sequence wait for one another, so the kernel is launched cooperatively
- * and the call fails with BS_ERR_CUDA where that is not possible.  A wait that does not end
+ * The CTAs that share a sequence wait for one another: they form a thread-block cluster, or --
+ * rows of a single 32 KB segment, very large batches -- the kernel is launched cooperatively, and
+ * the call fails with BS_ERR_CUDA where that is not possible.  A wait that does not end
  * within about a second makes bs_get_device_status return BS_ERR_TIMEOUT.
  * Requirement: rows on 16-byte boundaries (V * element size a multiple of 16, base pointers
  * 16-byte aligned), else BS_ERR_UNSUPPORTED. */
