@@ -53,6 +53,34 @@ def test_walk_parity(lib, dtype, B, G, V):
     assert tally.flagged_accept + tally.flagged_token <= 2 + tally.sequences // 100
 
 
+@pytest.mark.parametrize("B,G,V,dtype", [(6, 12, 40000, torch.float32), (330, 12, 40000, torch.float32),
+                                         (3, 31, 65536, torch.bfloat16)])
+def test_walk_long_accepted_runs(lib, B, G, V, dtype):
+    """Runs of up to 32 positions: a sequence is streamed ahead of its decisions through a few mailboxes that
+    are reused every fourth position -- with one sequence per cluster (far ahead) and with several (one ahead).
+    Half of the sequences have q == p, so every draft passes and the bonus row is sampled."""
+    rng = np.random.default_rng(B + G)
+    rnd = _round(rng, B, G, V, dtype, 1.0, sigma=0.25, gamma=rng.integers(G - 2, G + 1, size=B))
+    same = np.arange(B) % 2 == 0
+    rnd.draft[torch.as_tensor(same, device=DEV)] = rnd.target[torch.as_tensor(same, device=DEV), :G]
+    rnd.tokens = wl.draw_draft_tokens(rnd.draft, 1.0, rnd.uniforms.u_draft).contiguous()
+    ws = lib.new_workspace(B, G, V, DEV)
+    tally = parity.Tally()
+    out = _walk(lib, rnd, 1.0, ws)
+    assert (lib.bs_get_device_status(ws, B, G, V) & ~lib.BS_DEV_RESIDUAL_FALLBACK == 0).all()
+    tau = out.accept_len.cpu().numpy()
+    assert (tau[same] == rnd.gamma[same]).all()                          # r <= min{1, 1} always holds
+    assert B < 6 or tau[~same].max() >= 4                                # the mailboxes were reused by a rejecting run too
+    seqs = range(B) if B <= 8 else list(range(0, B, 37)) + [1]
+    parity.check_round(out, rnd, 1.0, tally, seqs=seqs, where=f"walk long runs B={B}", walk=True)
+    ref = parity.gpu_round(lib, rnd, 1.0, ws)                            # the two-call path on the same workspace
+    differ = [b for b in range(B) if int(ref.accept_len[b]) != int(out.accept_len[b])
+              or not torch.equal(ref.out_tokens[b], out.out_tokens[b])]
+    parity.check_round(ref, rnd, 1.0, tally, seqs=differ, where="two-call long runs")
+    parity.check_round(out, rnd, 1.0, tally, seqs=differ, where="walk long runs", walk=True)
+    assert len(differ) <= tally.flagged_accept + tally.flagged_token
+
+
 def test_walk_edge_cases_and_reuse(lib):
     rng = np.random.default_rng(17)
     B, G, V = 8, 6, 3000
