@@ -36,9 +36,11 @@ def _walk(lib, rnd, T, ws=None):
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
-@pytest.mark.parametrize("B,G,V", [(5, 4, 1000), (3, 6, 40000), (40, 3, 8200), (700, 2, 256), (2, 8, 128256)])
+@pytest.mark.parametrize("B,G,V", [(5, 4, 1000), (3, 6, 40000), (40, 3, 8200), (700, 2, 256), (2, 8, 128256),
+                                   (1500, 1, 16504), (2600, 1, 16504)])
 def test_walk_parity(lib, dtype, B, G, V):
-    """One CTA per sequence, several CTAs per sequence, several sequences per CTA; one and many segments."""
+    """One CTA per sequence, several CTAs per sequence, several sequences per CTA; one and many segments; batches
+    that fill the clusters' sequence slots and batches beyond them (the kernel that goes through the workspace)."""
     rng = np.random.default_rng(B * 7 + V)
     tally = parity.Tally()
     for T in (1.0, 0.6):
